@@ -1,0 +1,213 @@
+/*
+ * cpe.h - C ABI of the centroid-positional-encoding decoder for NVIDIA B200 (sm_100a).
+ *
+ * The library turns a dense per-pixel sinusoidal encoding of instance centroids into instance
+ * masks: every participating pixel's embedding is decoded to a centroid estimate, the estimates
+ * vote into an integer centroid map, local maxima of that map become instance centres, and every
+ * participating pixel is assigned to the centre whose encoding is nearest.
+ *
+ * Notation follows the paper: F harmonics per axis (the paper's L), D = 4F channels,
+ * gamma(p) = (sin(2^l pi p), cos(2^l pi p)), l = 0..F-1 (Eq. 2); palettes P_n hold gamma at the bin
+ * positions -1 + 2i/(n+1), i = 1..n (Eq. 9); the vote map has B_w x B_h bins (Sec. 3.2).
+ *
+ * Conventions
+ *   emb       planar [B][4F][H][W], contiguous, element type given by cpe_params.dtype.
+ *             channel c = axis*2F + 2l + t; axis 0 = x (width), 1 = y (height); t = 0 sin, 1 cos
+ *             (Eq. 1-3: concat(gamma(x), gamma(y)), each gamma as (sin, cos) per harmonic).
+ *   fg_mask   [B][H][W] bytes; a pixel participates iff its byte is non-zero.  NULL: all pixels
+ *             participate (the paper's set S is the whole output grid, Eq. 6).
+ *   images of a batch are independent: own vote map, own peak list, labels numbered from 1.
+ *
+ * All pointers named "device" are device memory owned by the caller; nothing in the stream-taking
+ * entry points allocates, frees, synchronises or reads device memory on the host, so they may be
+ * called while the stream is being captured into a CUDA graph.  Return value: 0 (CPE_OK) or a
+ * negative CPE_ERR_* code, reported before any work is enqueued.  Run-time conditions (more peaks
+ * than max_instances, non-finite pixels) are reported in the device status word, never as faults.
+ */
+#ifndef CPE_H_
+#define CPE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* A CUDA stream handle (cudaStream_t / CUstream); 0 is the legacy default stream. */
+typedef struct CUstream_st* cpe_stream_t;
+
+enum { CPE_F32 = 0, CPE_F16 = 1 };
+
+enum {
+  CPE_OK = 0,
+  CPE_ERR_NULL = -1,       /* a required pointer is NULL                                  */
+  CPE_ERR_SIZE = -2,       /* B, H, W < 1, F outside [1,16], bins outside [1,4096], ...    */
+  CPE_ERR_DTYPE = -3,      /* unknown element type                                         */
+  CPE_ERR_ALIGN = -4,      /* emb / outputs not aligned to their element size              */
+  CPE_ERR_WORKSPACE = -5,  /* workspace missing, misaligned (256 B) or too small           */
+  CPE_ERR_PARAM = -6,      /* struct_size mismatch, negative threshold, max_instances < 1  */
+  CPE_ERR_CUDA = -7,       /* a CUDA runtime call failed (see cpe_last_cuda_error)         */
+  CPE_ERR_WHICH = -8,      /* unknown intermediate id, or it was not requested by flags    */
+  CPE_ERR_NOMEM = -9       /* host or device allocation failed (context helpers only)      */
+};
+
+/* cpe_params.flags */
+enum {
+  CPE_FLAG_WRITE_SCORES = 1u  /* also store the best and second-best Eq. 4 distance of every pixel */
+};
+
+/* bits of the device status word */
+enum {
+  CPE_STATUS_PEAK_OVERFLOW = 1u, /* an image had more local maxima than max_instances            */
+  CPE_STATUS_NONFINITE = 2u      /* at least one participating pixel had a non-finite channel    */
+};
+
+/* per-image counters, uint32 [B][CPE_CNT_N] */
+enum {
+  CPE_CNT_VOTING = 0,       /* pixels that cast a vote                                      */
+  CPE_CNT_NONFINITE = 1,    /* participating pixels skipped because a channel was not finite */
+  CPE_CNT_RAW_PEAKS = 2,    /* local maxima found before truncation to max_instances        */
+  CPE_CNT_TRUNCATED = 3,    /* local maxima dropped by the truncation                       */
+  CPE_CNT_TAU_REJECTED = 4, /* pixels whose best distance was not below tau (label 0)       */
+  CPE_CNT_N = 8
+};
+
+/* ids for cpe_get_intermediate */
+enum {
+  CPE_INT_VOTES = 0,        /* uint32 [B][bins_h][bins_w]       hard-vote map                   */
+  CPE_INT_PEAK_CELLS = 1,   /* int32  [B][max_instances]        linear bin cy*bins_w+cx, ascending */
+  CPE_INT_PEAK_VOTES = 2,   /* uint32 [B][max_instances]        votes of each kept peak         */
+  CPE_INT_PEAK_EMB = 3,     /* float  [B][max_instances][4F]    concat(P_w[cx], P_h[cy])        */
+  CPE_INT_PALETTE_W = 4,    /* float  [bins_w][2F]              Eq. 9                           */
+  CPE_INT_PALETTE_H = 5,    /* float  [bins_h][2F]                                              */
+  CPE_INT_BEST_SCORE = 6,   /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
+  CPE_INT_SECOND_SCORE = 7, /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
+  CPE_INT_STATUS = 8,       /* uint32 [1]                                                       */
+  CPE_INT_COUNTERS = 9,     /* uint32 [B][CPE_CNT_N]                                            */
+  CPE_INT_N = 10
+};
+
+/* stages reported by cpe_profile_decode */
+enum {
+  CPE_STAGE_CLEAR = 0,      /* zeroing of the vote map, counters and status                    */
+  CPE_STAGE_DECODE_VOTE = 1,
+  CPE_STAGE_PEAKS = 2,      /* local-maximum test over the vote map                            */
+  CPE_STAGE_COMPACT = 3,    /* ordered peak list, centroids, peak embeddings                   */
+  CPE_STAGE_ASSIGN = 4,     /* assignment and label-map write                                  */
+  CPE_STAGE_N = 5
+};
+
+typedef struct cpe_params {
+  uint32_t struct_size;    /* sizeof(cpe_params)                                               */
+  int32_t dtype;           /* CPE_F32 or CPE_F16 (IEEE binary16) element type of emb           */
+  int32_t bins_w, bins_h;  /* B_w, B_h: vote-map size (Sec. 3.2); each in [1, 4096]            */
+  int32_t levels;          /* harmonics used by the centroid estimate; 0 or >= F means all F   */
+  int32_t vote_threshold;  /* T_v >= 0: a peak needs V > T_v ("predefined threshold", Sec. 3.2) */
+  float tau;               /* Eq. 8: a pixel keeps its label iff d < tau; +inf keeps every one */
+  int32_t max_instances;   /* K_max: capacity per image of the peak / centroid arrays          */
+  uint32_t flags;          /* CPE_FLAG_*                                                       */
+  void* workspace;         /* device memory, 256-byte aligned, owned by the caller             */
+  size_t workspace_bytes;  /* >= cpe_workspace_size(...) for the same B, H, W, F and params    */
+} cpe_params;
+
+/*
+ * Bytes of device workspace that cpe_decode needs for these sizes (0 on invalid arguments).
+ * The workspace holds what the paper keeps resident between stages: the palettes P_w, P_h
+ * (Eq. 9, "stored as model parameters preloaded in memory"), the vote map (Eq. 6, hard-vote
+ * form), the peak indicator (the map H-bar of the local-maxima search) and the peak list.
+ * Only workspace and workspace_bytes of params are ignored.
+ */
+size_t cpe_workspace_size(int B, int H, int W, int F, const cpe_params* params);
+
+/*
+ * One-time set-up of a workspace (Sec. 3.2: palettes are pre-computed once and kept resident):
+ * zeroes it and uploads P_w and P_h, evaluated on the host as (float) sin|cos(pi 2^l pos) in double.
+ * Enqueues on `stream`; must not be called during stream capture.  The workspace is then valid for
+ * cpe_decode calls with the same B, H, W, F, bins, max_instances and flags.
+ */
+int cpe_init_workspace(cpe_stream_t stream, int B, int H, int W, int F, const cpe_params* params);
+
+/*
+ * The decode path ("recover the predicted instance masks from a noisy estimate", Sec. 3.1),
+ * enqueued on `stream` without any host synchronisation:
+ *   1. per participating pixel and axis, a centroid estimate p in [-1,1) by coarse-to-fine phase
+ *      unwrapping of the harmonics; the pixel votes for the nearest Eq. 9 bin (hard-vote form of Eq. 6);
+ *   2. bins that exceed vote_threshold and beat their 8 neighbours (ties: lower linear index) are the
+ *      candidate centroids, listed by ascending linear bin index (Sec. 3.2, local-maxima search);
+ *   3. every participating pixel gets label 1 + argmin_k ||xhat - P_w(a_k)|| + ||yhat - P_h(b_k)||
+ *      (Eq. 4, Eq. 7; lowest k on ties) if that distance is below tau (Eq. 8), else 0.
+ *
+ * emb, fg_mask      device, see Conventions.  emb aligned to its element size (16 bytes and
+ *                   H*W a multiple of 16/elemsize select the vectorised kernels).
+ * out_labels        device int32 [B][H][W]; every element is written (0 = background / rejected).
+ * out_centroids     device float [B][max_instances][2]: (x, y) of each kept peak's bin position in pixel
+ *                   units (pixel centres at integers); rows >= out_count[b] are left untouched.
+ * out_count         device int32 [B]: number of instances kept, min(found, max_instances).
+ */
+int cpe_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+               const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count);
+
+/*
+ * Device address and size of an intermediate inside the workspace (CPE_INT_*); host-only arithmetic.
+ * The contents are those left by the last cpe_decode on that workspace.
+ */
+int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int W, int F, void** device_ptr,
+                         size_t* bytes);
+
+/* Human-readable text for a CPE_ERR_* code; never NULL. */
+const char* cpe_strerror(int code);
+
+/* The CUDA runtime error number behind the calling thread's last CPE_ERR_CUDA (0 if none). */
+int cpe_last_cuda_error(void);
+
+/* ------------------------------------------------------------------ CUDA-graph helper ------- */
+
+/*
+ * "The whole chain on one stream with no host sync between stages": captures one cpe_decode call with
+ * these arguments into a CUDA graph and instantiates it.  The pointers are baked into the graph and
+ * must stay valid.  cpe_graph_launch replays it on a stream.  The handle is host memory owned by the
+ * library until cpe_graph_destroy.
+ */
+typedef struct cpe_graph cpe_graph;
+int cpe_graph_create(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                     const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count,
+                     cpe_graph** out_graph);
+int cpe_graph_launch(cpe_graph* graph, cpe_stream_t stream);
+void cpe_graph_destroy(cpe_graph* graph);
+/* Number of kernel nodes in the captured graph (memset nodes not counted). */
+int cpe_graph_kernel_nodes(const cpe_graph* graph);
+
+/* ------------------------------------------------------------------ per-stage timing -------- */
+
+/*
+ * Runs cpe_decode `iters` times on `stream` with CUDA events recorded between the stages, waits for
+ * the stream, and returns the mean device time of each stage in milliseconds in stage_ms[CPE_STAGE_N].
+ * Synchronises; not capturable.  Same arguments and results as cpe_decode.
+ */
+int cpe_profile_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                       const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count,
+                       int iters, float* stage_ms);
+
+/* ------------------------------------------------------------------ host-buffer front end --- */
+
+/*
+ * End-to-end call for callers whose data lives in host memory.  The context owns its device buffers
+ * (input, mask, outputs, workspace), a stream and a captured graph for fixed B, H, W, F and params
+ * (params->workspace is ignored).  cpe_host_decode copies emb and fg_mask to the device, replays the
+ * graph, copies labels, centroids and counts back and returns when they have arrived.  Host buffers
+ * should be page-locked for full copy bandwidth; pageable memory works.  fg_mask_host may be NULL only
+ * if the context was created with has_mask = 0.
+ */
+typedef struct cpe_host_ctx cpe_host_ctx;
+int cpe_host_ctx_create(int B, int H, int W, int F, const cpe_params* params, int has_mask, cpe_host_ctx** out_ctx);
+int cpe_host_decode(cpe_host_ctx* ctx, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
+                    float* centroids_host, int32_t* count_host);
+/* Bytes moved per cpe_host_decode call in each direction. */
+int cpe_host_ctx_traffic(const cpe_host_ctx* ctx, size_t* h2d_bytes, size_t* d2h_bytes);
+void cpe_host_ctx_destroy(cpe_host_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CPE_H_ */

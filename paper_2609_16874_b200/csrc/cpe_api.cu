@@ -1,0 +1,433 @@
+// C ABI of the decoder: argument checks, workspace layout, launch geometry, CUDA-graph and host-buffer
+// helpers.  Every entry point that takes a stream only enqueues work.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "assign.cuh"
+#include "cpe.h"
+#include "cpe_common.cuh"
+#include "decode_vote.cuh"
+#include "peaks.cuh"
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda = (int)e;
+  return CPE_ERR_CUDA;
+}
+
+#define CPE_CUDA(call)                          \
+  do {                                          \
+    cudaError_t e_ = (call);                    \
+    if (e_ != cudaSuccess) return cuda_fail(e_); \
+  } while (0)
+
+inline size_t elem_size(int dtype) { return dtype == CPE_F32 ? 4 : 2; }
+
+int check_shape(int B, int H, int W, int F, const cpe_params* p) {
+  if (!p) return CPE_ERR_NULL;
+  if (p->struct_size != sizeof(cpe_params)) return CPE_ERR_PARAM;
+  if (p->dtype != CPE_F32 && p->dtype != CPE_F16) return CPE_ERR_DTYPE;
+  if (B < 1 || H < 1 || W < 1 || F < 1 || F > 16) return CPE_ERR_SIZE;
+  if ((long long)H * W > 0x7fffffffLL || B > 65535) return CPE_ERR_SIZE;
+  if (p->bins_w < 1 || p->bins_w > 4096 || p->bins_h < 1 || p->bins_h > 4096) return CPE_ERR_SIZE;
+  if (p->vote_threshold < 0 || p->max_instances < 1 || p->max_instances > (1 << 20)) return CPE_ERR_PARAM;
+  if (p->levels < 0) return CPE_ERR_PARAM;
+  if (p->tau != p->tau) return CPE_ERR_PARAM;  // NaN
+  return CPE_OK;
+}
+
+int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout* L) {
+  int rc = check_shape(B, H, W, F, p);
+  if (rc) return rc;
+  *L = cpe::make_layout(B, H, W, F, p);
+  if (!p->workspace || ((uintptr_t)p->workspace & 255u) || p->workspace_bytes < L->total) return CPE_ERR_WORKSPACE;
+  return CPE_OK;
+}
+
+template <typename T>
+int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                       uint32_t* votes, uint32_t* counters, uint32_t* status) {
+  constexpr int V = cpe::Elem<T>::kVec;
+  const bool vec = ((uintptr_t)emb % 16 == 0) && (HW % V == 0) && (!fg || (uintptr_t)fg % V == 0);
+  const T* e = static_cast<const T*>(emb);
+  const int per = vec ? V : 1;
+  const long long groups = ((long long)HW + per - 1) / per;
+  dim3 grid((unsigned)((groups + cpe::kVoteThreads - 1) / cpe::kVoteThreads), (unsigned)B);
+#define CPE_LAUNCH_VOTE(VEC_, FT_)                                                                             \
+  cpe::decode_vote_kernel<T, VEC_, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, F, p->levels, p->bins_w, \
+                                                                           p->bins_h, votes, counters, status)
+  if (vec) {
+    switch (F) {
+      case 4: CPE_LAUNCH_VOTE(V, 4); break;
+      case 8: CPE_LAUNCH_VOTE(V, 8); break;
+      case 16: CPE_LAUNCH_VOTE(V, 16); break;
+      default: CPE_LAUNCH_VOTE(V, 0); break;
+    }
+  } else {
+    CPE_LAUNCH_VOTE(1, 0);
+  }
+#undef CPE_LAUNCH_VOTE
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
+template <typename T>
+int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                  const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                  uint32_t* counters) {
+  const T* e = static_cast<const T*>(emb);
+  dim3 grid((unsigned)(((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads), (unsigned)B);
+#define CPE_LAUNCH_ASSIGN(FT_)                                                                                  \
+  cpe::assign_kernel<T, FT_><<<grid, cpe::kAssignThreads, 0, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, \
+                                                                  p->tau, labels, best, second, counters)
+  switch (F) {
+    case 4: CPE_LAUNCH_ASSIGN(4); break;
+    case 8: CPE_LAUNCH_ASSIGN(8); break;
+    case 16: CPE_LAUNCH_ASSIGN(16); break;
+    default: CPE_LAUNCH_ASSIGN(0); break;
+  }
+#undef CPE_LAUNCH_ASSIGN
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
+// The chain.  `ev`, when given, holds CPE_STAGE_N + 1 events recorded around the stages.
+int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int H, int W, int F, const cpe_params* p,
+                int32_t* out_labels, float* out_centroids, int32_t* out_count, cudaEvent_t* ev) {
+  if (!emb || !out_labels || !out_centroids || !out_count) return CPE_ERR_NULL;
+  cpe::Layout L;
+  int rc = check_workspace(B, H, W, F, p, &L);
+  if (rc) return rc;
+  if ((uintptr_t)emb % elem_size(p->dtype) || (uintptr_t)out_labels % 4 || (uintptr_t)out_centroids % 4 ||
+      (uintptr_t)out_count % 4)
+    return CPE_ERR_ALIGN;
+  char* ws = static_cast<char*>(p->workspace);
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.status);
+  uint32_t* counters = reinterpret_cast<uint32_t*>(ws + L.counters);
+  uint32_t* votes = reinterpret_cast<uint32_t*>(ws + L.votes);
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(ws + L.bitmap);
+  int32_t* peak_cell = reinterpret_cast<int32_t*>(ws + L.peak_cell);
+  uint32_t* peak_votes = reinterpret_cast<uint32_t*>(ws + L.peak_votes);
+  float* peak_emb = reinterpret_cast<float*>(ws + L.peak_emb);
+  const float* pal_w = reinterpret_cast<const float*>(ws + L.pal_w);
+  const float* pal_h = reinterpret_cast<const float*>(ws + L.pal_h);
+  float* best = (p->flags & CPE_FLAG_WRITE_SCORES) ? reinterpret_cast<float*>(ws + L.best) : nullptr;
+  float* second = (p->flags & CPE_FLAG_WRITE_SCORES) ? reinterpret_cast<float*>(ws + L.second) : nullptr;
+  const int HW = H * W;
+
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_CLEAR], st));
+  CPE_CUDA(cudaMemsetAsync(ws + L.status, 0, L.clear_end - L.status, st));
+
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
+  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, counters, status)
+                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, counters, status);
+  if (rc) return rc;
+
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_PEAKS], st));
+  {
+    const int warps_per_cta = cpe::kPeakThreads / 32;
+    dim3 grid((unsigned)((L.words + warps_per_cta - 1) / warps_per_cta), (unsigned)B);
+    cpe::peaks_bitmap_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
+                                                                 (uint32_t)p->vote_threshold, bitmap);
+    CPE_CUDA(cudaGetLastError());
+  }
+
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_COMPACT], st));
+  cpe::peaks_compact_kernel<<<(unsigned)B, cpe::kCompactThreads, 0, st>>>(
+      bitmap, votes, p->bins_w, p->bins_h, L.words, p->max_instances, F, H, W, pal_w, pal_h, peak_cell, peak_votes,
+      peak_emb, out_centroids, out_count, counters, status);
+  CPE_CUDA(cudaGetLastError());
+
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_ASSIGN], st));
+  rc = p->dtype == CPE_F32
+           ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters)
+           : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters);
+  if (rc) return rc;
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
+  return CPE_OK;
+}
+
+}  // namespace
+
+struct cpe_graph {
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  int kernel_nodes = 0;
+};
+
+struct cpe_host_ctx {
+  int B = 0, H = 0, W = 0, F = 0, has_mask = 0;
+  cpe_params params{};
+  cudaStream_t stream = nullptr;
+  void* d_emb = nullptr;
+  uint8_t* d_fg = nullptr;
+  int32_t* d_labels = nullptr;
+  float* d_centroids = nullptr;
+  int32_t* d_count = nullptr;
+  void* d_ws = nullptr;
+  cpe_graph* graph = nullptr;
+  size_t emb_bytes = 0, fg_bytes = 0, labels_bytes = 0, centroids_bytes = 0, count_bytes = 0;
+};
+
+extern "C" {
+
+size_t cpe_workspace_size(int B, int H, int W, int F, const cpe_params* params) {
+  if (check_shape(B, H, W, F, params) != CPE_OK) return 0;
+  return cpe::make_layout(B, H, W, F, params).total;
+}
+
+int cpe_init_workspace(cpe_stream_t stream, int B, int H, int W, int F, const cpe_params* params) {
+  cpe::Layout L;
+  int rc = check_workspace(B, H, W, F, params, &L);
+  if (rc) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(params->workspace);
+  CPE_CUDA(cudaMemsetAsync(ws, 0, L.total, st));
+  // Eq. 9 positions through Eq. 2, evaluated in double and rounded once to binary32.
+  const double pi = 3.14159265358979323846;
+  for (int axis = 0; axis < 2; ++axis) {
+    const int n = axis == 0 ? params->bins_w : params->bins_h;
+    std::vector<float> pal((size_t)n * 2 * F);
+    for (int i = 1; i <= n; ++i) {
+      const double pos = -1.0 + 2.0 * (double)i / (double)(n + 1);
+      for (int l = 0; l < F; ++l) {
+        const double arg = pi * ldexp(1.0, l) * pos;
+        pal[(size_t)(i - 1) * 2 * F + 2 * l] = (float)sin(arg);
+        pal[(size_t)(i - 1) * 2 * F + 2 * l + 1] = (float)cos(arg);
+      }
+    }
+    // pageable source: the runtime stages the data before returning, so `pal` may go out of scope
+    CPE_CUDA(cudaMemcpyAsync(ws + (axis == 0 ? L.pal_w : L.pal_h), pal.data(), pal.size() * sizeof(float),
+                             cudaMemcpyHostToDevice, st));
+    CPE_CUDA(cudaStreamSynchronize(st));
+  }
+  return CPE_OK;
+}
+
+int cpe_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+               const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count) {
+  return decode_impl(reinterpret_cast<cudaStream_t>(stream), emb, fg_mask, B, H, W, F, params, out_labels,
+                     out_centroids, out_count, nullptr);
+}
+
+int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int W, int F, void** device_ptr,
+                         size_t* bytes) {
+  if (!device_ptr || !bytes) return CPE_ERR_NULL;
+  cpe::Layout L;
+  int rc = check_workspace(B, H, W, F, params, &L);
+  if (rc) return rc;
+  const size_t Kmax = (size_t)params->max_instances, HW = (size_t)H * W;
+  size_t off = 0, sz = 0;
+  switch (which) {
+    case CPE_INT_VOTES: off = L.votes; sz = 4 * (size_t)L.cells * B; break;
+    case CPE_INT_PEAK_CELLS: off = L.peak_cell; sz = 4 * Kmax * B; break;
+    case CPE_INT_PEAK_VOTES: off = L.peak_votes; sz = 4 * Kmax * B; break;
+    case CPE_INT_PEAK_EMB: off = L.peak_emb; sz = 4 * Kmax * 4 * F * B; break;
+    case CPE_INT_PALETTE_W: off = L.pal_w; sz = 4 * (size_t)params->bins_w * 2 * F; break;
+    case CPE_INT_PALETTE_H: off = L.pal_h; sz = 4 * (size_t)params->bins_h * 2 * F; break;
+    case CPE_INT_BEST_SCORE:
+    case CPE_INT_SECOND_SCORE:
+      if (!(params->flags & CPE_FLAG_WRITE_SCORES)) return CPE_ERR_WHICH;
+      off = which == CPE_INT_BEST_SCORE ? L.best : L.second;
+      sz = 4 * HW * B;
+      break;
+    case CPE_INT_STATUS: off = L.status; sz = 4; break;
+    case CPE_INT_COUNTERS: off = L.counters; sz = 4 * (size_t)CPE_CNT_N * B; break;
+    default: return CPE_ERR_WHICH;
+  }
+  *device_ptr = static_cast<char*>(params->workspace) + off;
+  *bytes = sz;
+  return CPE_OK;
+}
+
+const char* cpe_strerror(int code) {
+  switch (code) {
+    case CPE_OK: return "ok";
+    case CPE_ERR_NULL: return "a required pointer is NULL";
+    case CPE_ERR_SIZE: return "a size is out of range (B, H, W >= 1; 1 <= F <= 16; 1 <= bins <= 4096)";
+    case CPE_ERR_DTYPE: return "unknown element type";
+    case CPE_ERR_ALIGN: return "a buffer is not aligned to its element size";
+    case CPE_ERR_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";
+    case CPE_ERR_PARAM: return "invalid cpe_params (struct_size, threshold, max_instances, levels or tau)";
+    case CPE_ERR_CUDA: return "a CUDA runtime call failed";
+    case CPE_ERR_WHICH: return "unknown or unavailable intermediate";
+    case CPE_ERR_NOMEM: return "allocation failed";
+    default: return "unknown error code";
+  }
+}
+
+int cpe_last_cuda_error(void) { return g_last_cuda; }
+
+// ------------------------------------------------------------------------------------ graph helper
+
+int cpe_graph_create(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                     const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count,
+                     cpe_graph** out_graph) {
+  if (!out_graph) return CPE_ERR_NULL;
+  *out_graph = nullptr;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cpe_graph* g = new (std::nothrow) cpe_graph();
+  if (!g) return CPE_ERR_NOMEM;
+  cudaError_t e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) { delete g; return cuda_fail(e); }
+  int rc = decode_impl(st, emb, fg_mask, B, H, W, F, params, out_labels, out_centroids, out_count, nullptr);
+  e = cudaStreamEndCapture(st, &g->graph);
+  if (rc != CPE_OK || e != cudaSuccess) {
+    if (g->graph) cudaGraphDestroy(g->graph);
+    delete g;
+    return rc != CPE_OK ? rc : cuda_fail(e);
+  }
+  e = cudaGraphInstantiate(&g->exec, g->graph, 0);
+  if (e != cudaSuccess) { cudaGraphDestroy(g->graph); delete g; return cuda_fail(e); }
+  size_t n = 0;
+  if (cudaGraphGetNodes(g->graph, nullptr, &n) == cudaSuccess && n) {
+    std::vector<cudaGraphNode_t> nodes(n);
+    if (cudaGraphGetNodes(g->graph, nodes.data(), &n) == cudaSuccess) {
+      for (size_t i = 0; i < n; ++i) {
+        cudaGraphNodeType t;
+        if (cudaGraphNodeGetType(nodes[i], &t) == cudaSuccess && t == cudaGraphNodeTypeKernel) ++g->kernel_nodes;
+      }
+    }
+  }
+  *out_graph = g;
+  return CPE_OK;
+}
+
+int cpe_graph_launch(cpe_graph* graph, cpe_stream_t stream) {
+  if (!graph || !graph->exec) return CPE_ERR_NULL;
+  CPE_CUDA(cudaGraphLaunch(graph->exec, reinterpret_cast<cudaStream_t>(stream)));
+  return CPE_OK;
+}
+
+void cpe_graph_destroy(cpe_graph* graph) {
+  if (!graph) return;
+  if (graph->exec) cudaGraphExecDestroy(graph->exec);
+  if (graph->graph) cudaGraphDestroy(graph->graph);
+  delete graph;
+}
+
+int cpe_graph_kernel_nodes(const cpe_graph* graph) { return graph ? graph->kernel_nodes : 0; }
+
+// ------------------------------------------------------------------------------------ per-stage timing
+
+int cpe_profile_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                       const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count,
+                       int iters, float* stage_ms) {
+  if (!stage_ms) return CPE_ERR_NULL;
+  if (iters < 1) return CPE_ERR_SIZE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int per = CPE_STAGE_N + 1;
+  std::vector<cudaEvent_t> ev((size_t)iters * per, nullptr);
+  int rc = CPE_OK;
+  for (auto& x : ev) {
+    cudaError_t e = cudaEventCreate(&x);
+    if (e != cudaSuccess) { rc = cuda_fail(e); break; }
+  }
+  for (int it = 0; rc == CPE_OK && it < iters; ++it)
+    rc = decode_impl(st, emb, fg_mask, B, H, W, F, params, out_labels, out_centroids, out_count, &ev[(size_t)it * per]);
+  if (rc == CPE_OK) {
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+  }
+  if (rc == CPE_OK) {
+    for (int s = 0; s < CPE_STAGE_N; ++s) {
+      double sum = 0.0;
+      for (int it = 0; it < iters; ++it) {
+        float ms = 0.0f;
+        cudaEventElapsedTime(&ms, ev[(size_t)it * per + s], ev[(size_t)it * per + s + 1]);
+        sum += ms;
+      }
+      stage_ms[s] = (float)(sum / iters);
+    }
+  }
+  for (auto& x : ev)
+    if (x) cudaEventDestroy(x);
+  return rc;
+}
+
+// ------------------------------------------------------------------------------------ host-buffer front end
+
+void cpe_host_ctx_destroy(cpe_host_ctx* c) {
+  if (!c) return;
+  if (c->graph) cpe_graph_destroy(c->graph);
+  cudaFree(c->d_emb);
+  cudaFree(c->d_fg);
+  cudaFree(c->d_labels);
+  cudaFree(c->d_centroids);
+  cudaFree(c->d_count);
+  cudaFree(c->d_ws);
+  if (c->stream) cudaStreamDestroy(c->stream);
+  delete c;
+}
+
+int cpe_host_ctx_create(int B, int H, int W, int F, const cpe_params* params, int has_mask, cpe_host_ctx** out_ctx) {
+  if (!out_ctx) return CPE_ERR_NULL;
+  *out_ctx = nullptr;
+  int rc = check_shape(B, H, W, F, params);
+  if (rc) return rc;
+  cpe_host_ctx* c = new (std::nothrow) cpe_host_ctx();
+  if (!c) return CPE_ERR_NOMEM;
+  c->B = B; c->H = H; c->W = W; c->F = F; c->has_mask = has_mask ? 1 : 0;
+  c->params = *params;
+  const size_t HW = (size_t)H * W;
+  c->emb_bytes = (size_t)B * 4 * F * HW * elem_size(params->dtype);
+  c->fg_bytes = has_mask ? (size_t)B * HW : 0;
+  c->labels_bytes = (size_t)B * HW * 4;
+  c->centroids_bytes = (size_t)B * params->max_instances * 2 * 4;
+  c->count_bytes = (size_t)B * 4;
+  c->params.workspace_bytes = cpe::make_layout(B, H, W, F, params).total;
+  cudaError_t e = cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_emb, c->emb_bytes);
+  if (e == cudaSuccess && has_mask) e = cudaMalloc((void**)&c->d_fg, c->fg_bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_labels, c->labels_bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_centroids, c->centroids_bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_count, c->count_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_ws, c->params.workspace_bytes);
+  if (e != cudaSuccess) {
+    cuda_fail(e);
+    cpe_host_ctx_destroy(c);
+    return e == cudaErrorMemoryAllocation ? CPE_ERR_NOMEM : CPE_ERR_CUDA;
+  }
+  c->params.workspace = c->d_ws;
+  cpe_stream_t s = reinterpret_cast<cpe_stream_t>(c->stream);
+  rc = cpe_init_workspace(s, B, H, W, F, &c->params);
+  if (rc == CPE_OK && cudaMemsetAsync(c->d_centroids, 0, c->centroids_bytes, c->stream) != cudaSuccess) rc = CPE_ERR_CUDA;
+  if (rc == CPE_OK)
+    rc = cpe_graph_create(s, c->d_emb, c->d_fg, B, H, W, F, &c->params, c->d_labels, c->d_centroids, c->d_count,
+                          &c->graph);
+  if (rc != CPE_OK) { cpe_host_ctx_destroy(c); return rc; }
+  *out_ctx = c;
+  return CPE_OK;
+}
+
+int cpe_host_decode(cpe_host_ctx* c, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
+                    float* centroids_host, int32_t* count_host) {
+  if (!c || !emb_host || !labels_host || !centroids_host || !count_host) return CPE_ERR_NULL;
+  if (c->has_mask && !fg_mask_host) return CPE_ERR_NULL;
+  CPE_CUDA(cudaMemcpyAsync(c->d_emb, emb_host, c->emb_bytes, cudaMemcpyHostToDevice, c->stream));
+  if (c->has_mask) CPE_CUDA(cudaMemcpyAsync(c->d_fg, fg_mask_host, c->fg_bytes, cudaMemcpyHostToDevice, c->stream));
+  int rc = cpe_graph_launch(c->graph, reinterpret_cast<cpe_stream_t>(c->stream));
+  if (rc) return rc;
+  CPE_CUDA(cudaMemcpyAsync(labels_host, c->d_labels, c->labels_bytes, cudaMemcpyDeviceToHost, c->stream));
+  CPE_CUDA(cudaMemcpyAsync(centroids_host, c->d_centroids, c->centroids_bytes, cudaMemcpyDeviceToHost, c->stream));
+  CPE_CUDA(cudaMemcpyAsync(count_host, c->d_count, c->count_bytes, cudaMemcpyDeviceToHost, c->stream));
+  CPE_CUDA(cudaStreamSynchronize(c->stream));
+  return CPE_OK;
+}
+
+int cpe_host_ctx_traffic(const cpe_host_ctx* c, size_t* h2d_bytes, size_t* d2h_bytes) {
+  if (!c || !h2d_bytes || !d2h_bytes) return CPE_ERR_NULL;
+  *h2d_bytes = c->emb_bytes + c->fg_bytes;
+  *d2h_bytes = c->labels_bytes + c->centroids_bytes + c->count_bytes;
+  return CPE_OK;
+}
+
+}  // extern "C"

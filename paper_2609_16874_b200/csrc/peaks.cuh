@@ -1,0 +1,140 @@
+// Stage 3: local-maximum test over the vote map (Sec. 3.2, "Local Maxima Search") and ordered
+// compaction of the peaks into a device-side list, with centroids and peak embeddings.
+#pragma once
+
+#include "cpe_common.cuh"
+
+namespace cpe {
+
+constexpr int kPeakThreads = 256;
+constexpr int kCompactThreads = 1024;
+
+// One thread per bin, one warp per 32 consecutive bins: the warp's ballot is one word of the peak
+// indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it beats
+// each existing 8-neighbour: larger count, or equal count and lower linear index.
+__global__ void __launch_bounds__(kPeakThreads)
+peaks_bitmap_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
+                    uint32_t* __restrict__ bitmap) {
+  const int b = blockIdx.y;
+  const int warp = (blockIdx.x * kPeakThreads + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= words) return;  // whole warps leave together
+  const int cells = bins_w * bins_h;
+  const uint32_t* V = votes + (size_t)b * cells;
+  const int lin = warp * 32 + lane;
+  bool peak = false;
+  if (lin < cells) {
+    const uint32_t v = __ldg(V + lin);
+    if (v > T_v) {
+      const int cy = lin / bins_w, cx = lin - cy * bins_w;
+      peak = true;
+#pragma unroll
+      for (int dy = -1; dy <= 1; ++dy) {
+#pragma unroll
+        for (int dx = -1; dx <= 1; ++dx) {
+          if (dx == 0 && dy == 0) continue;
+          const int ny = cy + dy, nx = cx + dx;
+          if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+          const int nlin = ny * bins_w + nx;
+          const uint32_t nv = __ldg(V + nlin);
+          if (nv > v || (nv == v && nlin < lin)) peak = false;
+        }
+      }
+    }
+  }
+  const uint32_t word = __ballot_sync(0xffffffffu, peak);
+  if (lane == 0) bitmap[(size_t)b * words + warp] = word;
+}
+
+// One CTA per image.  Ordered compaction without atomics or sorting: every thread counts the set bits
+// of its contiguous slice of the bitmap, an exclusive block scan gives each slice its first output slot,
+// and the slices are written out in order, so the list is ascending in the linear bin index and, when
+// there are more than K_max peaks, exactly the first K_max are kept.  Then the centroids (bin positions
+// of Eq. 9 in pixel units) and the peak embeddings concat(P_w[cx], P_h[cy]) are gathered.
+__global__ void __launch_bounds__(kCompactThreads)
+peaks_compact_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ votes, int bins_w, int bins_h,
+                     int words, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
+                     const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell,
+                     uint32_t* __restrict__ peak_votes, float* __restrict__ peak_emb,
+                     float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
+                     uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
+  const int b = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int cells = bins_w * bins_h;
+  const uint32_t* bm = bitmap + (size_t)b * words;
+  const uint32_t* V = votes + (size_t)b * cells;
+  int32_t* pc = peak_cell + (size_t)b * K_max;
+  uint32_t* pv = peak_votes + (size_t)b * K_max;
+
+  const int per = (words + kCompactThreads - 1) / kCompactThreads;
+  const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+  int local = 0;
+  for (int w = w0; w < w1; ++w) local += __popc(bm[w]);
+
+  // exclusive scan over the block
+  __shared__ int s_warp[kCompactThreads / 32];
+  __shared__ int s_total;
+  int incl = local;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) s_warp[wid] = incl;
+  __syncthreads();
+  if (wid == 0) {
+    int v = s_warp[lane];
+    int inc2 = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc2, d);
+      if (lane >= d) inc2 += t;
+    }
+    s_warp[lane] = inc2 - v;  // exclusive prefix of the warp totals
+    if (lane == 31) s_total = inc2;
+  }
+  __syncthreads();
+  int slot = s_warp[wid] + incl - local;
+  const int total = s_total;
+
+  for (int w = w0; w < w1 && slot < K_max; ++w) {
+    uint32_t bits = bm[w];
+    while (bits && slot < K_max) {
+      const int bit = __ffs(bits) - 1;
+      bits &= bits - 1;
+      const int lin = w * 32 + bit;
+      pc[slot] = lin;
+      pv[slot] = V[lin];
+      ++slot;
+    }
+  }
+  const int count = min(total, K_max);
+  if (tid == 0) {
+    out_count[b] = count;
+    counters[b * CPE_CNT_N + CPE_CNT_RAW_PEAKS] = (uint32_t)total;
+    counters[b * CPE_CNT_N + CPE_CNT_TRUNCATED] = (uint32_t)(total - count);
+    if (total > K_max) atomicOr(status, (uint32_t)CPE_STATUS_PEAK_OVERFLOW);
+  }
+  __syncthreads();  // the list written above is read below by other threads of this CTA
+
+  const int D = 4 * F;
+  float* pe = peak_emb + (size_t)b * K_max * D;
+  for (int i = tid; i < count * D; i += kCompactThreads) {
+    const int k = i / D, c = i - k * D;
+    const int lin = pc[k];
+    const int cy = lin / bins_w, cx = lin - cy * bins_w;
+    pe[i] = (c < 2 * F) ? pal_w[cx * 2 * F + c] : pal_h[cy * 2 * F + (c - 2 * F)];
+  }
+  for (int k = tid; k < count; k += kCompactThreads) {
+    const int lin = pc[k];
+    const int cy = lin / bins_w, cx = lin - cy * bins_w;
+    // bin position -1 + 2i/(n+1), i = c+1 (Eq. 9); pixel centres sit at x = -1 + (2 col + 1)/W
+    const double x = -1.0 + 2.0 * (double)(cx + 1) / (double)(bins_w + 1);
+    const double y = -1.0 + 2.0 * (double)(cy + 1) / (double)(bins_h + 1);
+    float* o = out_centroids + ((size_t)b * K_max + k) * 2;
+    o[0] = (float)(((x + 1.0) * (double)W - 1.0) * 0.5);
+    o[1] = (float)(((y + 1.0) * (double)H - 1.0) * 0.5);
+  }
+}
+
+}  // namespace cpe

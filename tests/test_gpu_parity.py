@@ -1,0 +1,189 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.  All tests need a B200."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_16874_b200 import binding as cb
+from paper_2609_16874_b200 import workloads as wl
+
+from gpu_util import check_case, compare_front, compare_labels, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+# Reduced copies of the five configurations: same recipe, sizes the oracle finishes in seconds, several CTAs
+# per kernel, with and without a ragged tail (H*W not a multiple of the vector width -> scalar-load kernels).
+SMALL = [
+    ("c1", dict()),                                                        # the real c1: 128x128
+    ("c1", dict(H=67, W=93)),                                              # odd sizes: scalar path
+    ("c2", dict(H=192, W=256, K=12)),
+    ("c2", dict(H=131, W=77, K=6, bins_w=48, bins_h=40)),
+    ("c3", dict(H=256, W=384, K=24, bins_w=96, bins_h=64)),
+    ("c3", dict(H=99, W=121, K=8, bins_w=64, bins_h=32)),
+    ("c4", dict(B=3, H=160, W=168, K=30, bins_w=40, bins_h=40)),
+    ("c5", dict(H=256, W=256, K=40, bins_w=128, bins_h=128)),
+]
+
+
+@pytest.mark.parametrize("name,over", SMALL, ids=[f"{n}-{i}" for i, (n, _) in enumerate(SMALL)])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_small_configs_match_oracle(name, over, mode):
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 0)
+    gpu, ora, rep = check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, mode=mode)
+    assert ora["count"].min() >= 1
+    assert gpu["status"] == 0
+    print(name, over, "near ties:", rep)
+
+
+@pytest.mark.parametrize("F,dtype", [(1, np.float32), (2, np.float16), (3, np.float32), (5, np.float16), (12, np.float32)])
+def test_other_harmonic_counts(F, dtype):
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=64, W=80, K=5, F=F, bins_w=16, bins_h=16,
+                    dtype="f32" if dtype == np.float32 else "f16", sigma=0.02)
+    fr = wl.make_frame(cfg, 2)
+    check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)
+
+
+def test_no_mask_all_pixels_participate():
+    cfg = wl.scaled(wl.CONFIGS["c1"], H=64, W=64)
+    fr = wl.make_frame(cfg, 1)
+    gpu, ora, _ = check_case(fr["emb"], None, cfg.bins_w, cfg.bins_h)
+    assert ora["counters"][0, oracle.CNT_VOTING] == 64 * 64
+
+
+def test_empty_foreground_and_no_peaks():
+    cfg = wl.scaled(wl.CONFIGS["c3"], H=64, W=128, K=4, bins_w=32, bins_h=16)
+    fr = wl.make_frame(cfg, 0)
+    fg = np.zeros_like(fr["fg"])
+    gpu, ora, _ = check_case(fr["emb"], fg, cfg.bins_w, cfg.bins_h)
+    assert gpu["count"][0] == 0 and (gpu["labels"] == 0).all() and gpu["votes"].sum() == 0
+    # foreground too small for any bin to pass the threshold: votes exist, no peak, all labels 0
+    fg[0, :2, :3] = 1
+    gpu, ora, _ = check_case(fr["emb"], fg, cfg.bins_w, cfg.bins_h)
+    assert gpu["count"][0] == 0 and (gpu["labels"] == 0).all() and gpu["votes"].sum() == 6
+
+
+def test_nonfinite_pixels_are_skipped_and_counted():
+    for dtype in ("f32", "f16"):
+        cfg = wl.scaled(wl.CONFIGS["c2"], H=96, W=96, K=5, dtype=dtype, bins_w=32, bins_h=32)
+        fr = wl.make_frame(cfg, 0)
+        emb = fr["emb"].copy()
+        ys, xs = np.nonzero(fr["fg"][0])
+        rng = np.random.default_rng(0)
+        pick = rng.choice(ys.size, 40, replace=False)
+        for i, j in enumerate(pick):
+            emb[0, rng.integers(0, cfg.D), ys[j], xs[j]] = [np.nan, np.inf, -np.inf][i % 3]
+        gpu, ora, _ = check_case(emb, fr["fg"], cfg.bins_w, cfg.bins_h)
+        assert gpu["counters"][0, cb.CPE_CNT_NONFINITE] == 40
+        assert gpu["status"] & cb.CPE_STATUS_NONFINITE
+        assert (gpu["labels"][0, ys[pick], xs[pick]] == 0).all()
+
+
+def test_peak_overflow_keeps_first_k_max():
+    cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=160, W=160, K=30, bins_w=40, bins_h=40)
+    fr = wl.make_frame(cfg, 0)
+    gpu, ora, _ = check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, K_max=7)
+    assert (gpu["count"] == 7).all() and gpu["status"] & cb.CPE_STATUS_PEAK_OVERFLOW
+    assert (gpu["counters"][:, cb.CPE_CNT_TRUNCATED] > 0).all()
+
+
+def test_tau_rejection_and_levels():
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=128, W=128, K=6, bins_w=32, bins_h=32, sigma=0.1)
+    fr = wl.make_frame(cfg, 0)
+    ora = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)
+    tau = float(np.median(ora["best"][np.isfinite(ora["best"])]))
+    gpu, ora2, _ = check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, tau=tau)
+    assert 0 < gpu["counters"][0, cb.CPE_CNT_TAU_REJECTED] < fr["fg"].sum()
+    for levels in (1, 3, 6):
+        check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, levels=levels)
+
+
+def test_threshold_and_tie_rules_on_constructed_votes():
+    # Noise-free encodings of centroids on bin positions give an exactly known vote map; equal-area
+    # neighbours make a two-bin plateau, which must resolve to the lower linear index on both sides.
+    H, W, F, bw, bh = 64, 64, 4, 16, 16
+    inst = np.zeros((H, W), np.int32)
+    inst[0:16, 0:16] = 1
+    inst[0:16, 16:32] = 2          # same area as 1, adjacent bins -> tie
+    inst[32:64, 0:32] = 3
+    inst[40:43, 40:43] = 4         # 9 pixels: above T_v = 8
+    inst[50:52, 50:54] = 5         # 8 pixels: not above
+    bins = [(3, 3), (4, 3), (10, 12), (13, 2), (8, 8)]
+    cents = np.array([[-1 + 2 * (cx + 1) / (bw + 1), -1 + 2 * (cy + 1) / (bh + 1)] for cx, cy in bins])
+    emb = wl.encode(inst, cents, F, 0.0, None, np.float32)[None]
+    fg = (inst > 0).astype(np.uint8)[None]
+    gpu, ora, _ = check_case(emb, fg, bw, bh, T_v=8)
+    assert gpu["count"][0] == 3
+    assert gpu["peak_cell"][0, :3].tolist() == sorted([3 * bw + 3, 12 * bw + 10, 2 * bw + 13])
+
+
+def test_host_front_end_matches_device_path():
+    cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=96, W=104, K=10, bins_w=24, bins_h=24)
+    fr = wl.make_frame(cfg, 0)
+    ora = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    hd = cb.HostDecoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    labels = np.full((cfg.B, cfg.H, cfg.W), -1, np.int32)
+    cents = np.zeros((cfg.B, cfg.K_max, 2), np.float32)
+    count = np.zeros(cfg.B, np.int32)
+    for _ in range(2):
+        hd.decode(fr["emb"], fr["fg"], labels, cents, count)
+        assert np.array_equal(count, ora["count"])
+        rep = compare_labels(labels, None, None, ora["labels"], ora["best"], ora["second"])
+    assert hd.h2d_bytes == fr["emb"].nbytes + fr["fg"].nbytes
+    assert hd.d2h_bytes == labels.nbytes + cents.nbytes + count.nbytes
+    hd.close()
+
+
+def test_profile_entry_point_reports_all_stages():
+    import torch
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=128, W=128, K=6, bins_w=32, bins_h=32)
+    fr = wl.make_frame(cfg, 0)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h)
+    ms = dec.profile(torch.from_numpy(fr["emb"]).cuda(), torch.from_numpy(fr["fg"]).cuda(), iters=3)
+    assert set(ms) == set(cb.CPE_STAGE_NAMES) and all(v > 0 for v in ms.values())
+    ora = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, want_scores=True)
+    compare_labels(dec.labels.cpu().numpy(), None, None, ora["labels"], ora["best"], ora["second"])
+    dec.close()
+
+
+# ---------------------------------------------------------------- the five configurations at full size
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+def test_full_size_configs(name):
+    """Full-size inputs in the launch configuration the benchmark times (graph replay): votes, peaks, counts and
+    centroids against the full oracle; labels and scores on sampled pixels the oracle scores one by one; label-map
+    properties on every pixel."""
+    cfg = wl.CONFIGS[name]
+    fr = wl.make_frame(cfg, 0)
+    emb, fg = fr["emb"], fr["fg"]
+    gpu = run_gpu(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, True, "graph")
+    ov = oracle.votes(emb, fg, cfg.bins_w, cfg.bins_h)
+    ora = {"votes": ov["votes"], "counters": ov["counters"], "count": np.zeros(cfg.B, np.int32),
+           "peak_cell": np.full((cfg.B, cfg.K_max), -1, np.int32), "peak_votes": np.zeros((cfg.B, cfg.K_max), np.uint32),
+           "centroids": np.zeros((cfg.B, cfg.K_max, 2), np.float32)}
+    for b in range(cfg.B):
+        cells, pv, raw = oracle.peaks(ov["votes"][b], cfg.T_v, cfg.K_max)
+        n = len(cells)
+        ora["count"][b] = n
+        ora["peak_cell"][b, :n], ora["peak_votes"][b, :n] = cells, pv
+        ora["counters"][b, oracle.CNT_RAW_PEAKS], ora["counters"][b, oracle.CNT_TRUNCATED] = raw, raw - n
+        for k, lin in enumerate(cells):
+            ora["centroids"][b, k] = oracle.centroid_px(lin % cfg.bins_w, lin // cfg.bins_w, cfg.bins_w, cfg.bins_h,
+                                                        cfg.H, cfg.W)
+    compare_front(gpu, ora, cfg.F, cfg.bins_w, cfg.bins_h)
+    rng = np.random.default_rng(99)
+    n_sample = {"c1": cfg.H * cfg.W, "c2": 60000, "c3": 40000, "c4": 8000, "c5": 12000}[name]
+    near = excused = 0
+    for b in range(cfg.B):
+        n = int(ora["count"][b])
+        idx = np.sort(rng.choice(cfg.H * cfg.W, min(n_sample, cfg.H * cfg.W), replace=False)).astype(np.int64)
+        res = oracle.assign_image(emb[b], fg[b], cfg.bins_w, cfg.bins_h, ora["peak_cell"][b, :n], cfg.tau, idx=idx)
+        rep = compare_labels(gpu["labels"][b].ravel()[idx], gpu["best"][b].ravel()[idx],
+                             gpu["second"][b].ravel()[idx], res["labels"], res["best"], res["second"])
+        near += rep["near_tie_pixels"]
+        excused += rep["excused_mismatches"]
+        lab = gpu["labels"][b]
+        assert ((lab > 0) == (fg[b] > 0)).all()          # tau = inf: labels partition the foreground
+        assert lab.max() <= n and lab.min() >= 0
+    assert gpu["status"] == 0
+    print(f"{name}: peaks {ora['count'].tolist()}, sampled near-tie pixels {near}, excused label differences {excused}")
