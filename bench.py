@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the CPE decode path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1..c5] [--impl ours|reference]
+
+One "step" is one pass of the whole decode path (clear, decode+vote, peaks, compaction, assignment+labels)
+over one batch of the chosen workload, replayed as one CUDA graph.  Prints ONE JSON line (rank 0).
+
+  value       whole-job megapixels/s, inputs resident in HBM, device time (CUDA events on the launching
+              stream), max over ranks; weak scaling: every rank decodes its own frames, no collective.
+  e2e         the same metric through the host-buffer entry point (pinned host memory in, host memory out),
+              copies inside the timed region.
+  roofline    the dominant kernel against the measured HBM copy bandwidth (MEASURED_PEAKS.json).
+  cpu_baseline  the CPU oracle, as it stands, on this machine's host cores (rank 0, N = 1).
+
+`--impl reference` times the CPU oracle itself (there is no other reference implementation of this path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_16874_b200 import distributed as dist_util  # noqa: E402
+from paper_2609_16874_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode_megapixels_per_s"
+UNIT = "MP/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (None: not captured for that workload).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed region runs (reading only)."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._active = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            if self._active.is_set():
+                try:
+                    mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                    try:
+                        r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                    except Exception:
+                        r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                    self.samples.append(mhz)
+                    for bit, name in self.REASONS.items():
+                        if r & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def window(self, on: bool):
+        (self._active.set if on else self._active.clear)()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=1.0)
+        return {"sm_mhz": (float(np.median(self.samples)) if self.samples else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def algorithmic_bytes(cfg, fg_pixels: int):
+    """Bytes each kernel must move per launch: participating pixels' embeddings once per pass, the mask once per
+    pass, the label map once; vote map / peak lists are negligible and counted where they are touched."""
+    P, D, esz = cfg.pixels, cfg.D, cfg.esz
+    cells = cfg.B * cfg.bins_w * cfg.bins_h
+    return {
+        "clear": 4 * cells,
+        "decode_vote": fg_pixels * D * esz + P,
+        "peaks": 4 * cells + cells // 8,
+        "compact": cells // 8,
+        "assign": fg_pixels * D * esz + P + 4 * P,
+    }
+
+
+def frames_needed(cfg):
+    """Rotate over enough distinct frames that the inputs of consecutive steps cannot all sit in L2."""
+    return max(1, min(8, math.ceil(2.2 * L2_BYTES / cfg.emb_bytes)))
+
+
+# ----------------------------------------------------------------------------------------- CPU oracle timing
+
+def time_oracle(cfg, frame, budget_s: float, threads: int):
+    """Seconds per full batch for the oracle as it stands: the vote and peak steps on the whole batch, the
+    assignment on a sample of pixels (scaled up linearly: its cost is per pixel)."""
+    import oracle
+    oracle.set_threads(threads)
+    emb, fg = frame["emb"], frame["fg"]
+    t0 = time.perf_counter()
+    ov = oracle.votes(emb, fg, cfg.bins_w, cfg.bins_h)
+    peaks = [oracle.peaks(ov["votes"][b], cfg.T_v, cfg.K_max)[0] for b in range(cfg.B)]
+    t_front = time.perf_counter() - t0
+    HW = cfg.H * cfg.W
+    # calibrate the per-pixel assignment cost on a small sample, then size the real sample to the budget
+    rng = np.random.default_rng(0)
+    n_cal = min(HW, 4096)
+    idx = np.sort(rng.choice(HW, n_cal, replace=False)).astype(np.int64)
+    t0 = time.perf_counter()
+    oracle.assign_image(emb[0], fg[0], cfg.bins_w, cfg.bins_h, peaks[0], cfg.tau, idx=idx)
+    per_px = max((time.perf_counter() - t0) / n_cal, 1e-9)
+    n = int(min(HW, max(n_cal, budget_s / per_px / cfg.B)))
+    t_assign = 0.0
+    for b in range(cfg.B):
+        idx = None if n >= HW else np.sort(rng.choice(HW, n, replace=False)).astype(np.int64)
+        t0 = time.perf_counter()
+        oracle.assign_image(emb[b], fg[b], cfg.bins_w, cfg.bins_h, peaks[b], cfg.tau, idx=idx)
+        t_assign += (time.perf_counter() - t0) * (HW / min(n, HW))
+    sample = (f"votes+peaks on the full batch; assignment on {min(n, HW)} of {HW} pixels per image"
+              + (" (all)" if n >= HW else ", scaled to the image"))
+    return t_front + t_assign, sample
+
+
+def run_reference(args, cfg):
+    """`--impl reference`: the CPU oracle, timed on the host cores, on the same workload and metric."""
+    rank, _, world = dist_util.env_world()
+    if rank != 0:
+        return
+    import oracle
+    threads = oracle.max_threads()
+    frame = wl.make_frame(cfg, 0)
+    total_steps = args.steps + args.warmup
+    budget = max(0.05, min(2.0, 90.0 / max(1, total_steps)))
+    times, sample = [], ""
+    for i in range(total_steps):
+        t, sample = time_oracle(cfg, frame, budget, threads)
+        if i >= args.warmup:
+            times.append(t)
+    sec = float(np.mean(times))
+    value = cfg.pixels / sec / 1e6
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.describe(), "name": cfg.name, "timing": "host wall clock; the oracle is CPU code"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------- the GPU arm
+
+def run_ours(args, cfg):
+    import torch
+    from paper_2609_16874_b200 import binding as cb
+
+    rank, local_rank, world = dist_util.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    dev = torch.device("cuda", local_rank if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist_util.init("nccl", dev)
+    K, Wm = args.steps, args.warmup
+
+    # inputs: this rank's own frames (weak scaling), resident in HBM before anything is timed
+    n_frames = frames_needed(cfg)
+    frame_ids = dist_util.frames_for_rank(rank, world, n_frames)
+    frames = [wl.make_frame(cfg, f) for f in frame_ids]
+    d_emb = [torch.from_numpy(f["emb"]).to(dev) for f in frames]
+    d_fg = [torch.from_numpy(f["fg"]).to(dev) for f in frames]
+    fg_pixels = [int(f["fg"].sum()) for f in frames]
+    flush = None
+    if n_frames * cfg.emb_bytes < 2 * L2_BYTES:
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max,
+                     device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    with torch.cuda.stream(stream):
+        graphs = [dec.capture(d_emb[i], d_fg[i], stream=stream) for i in range(n_frames)]
+        kernel_nodes = cb.cpe_graph_kernel_nodes(graphs[0])
+
+        def step(i, ev0=None, ev1=None):
+            if flush is not None:
+                flush.fill_(i & 0xff)                     # evicts L2 between steps; outside the event pair
+            if ev0 is not None:
+                ev0.record(stream)
+            dec.replay(graphs[i % n_frames], stream=stream)
+            if ev1 is not None:
+                ev1.record(stream)
+
+        # bring the clocks up (idle parts sit at a few hundred MHz), then the W warm-up steps
+        t_end = time.perf_counter() + (0.0 if args.quick else 0.4)
+        i = 0
+        while time.perf_counter() < t_end:
+            step(i)
+            i += 1
+            if i % 64 == 0:
+                stream.synchronize()
+        for i in range(Wm):
+            step(i)
+        stream.synchronize()
+
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        dist_util.barrier()
+        torch.cuda.synchronize(dev)
+        sampler.window(True)
+        for i in range(K):
+            step(i, *ev[i])
+        stream.synchronize()
+        torch.cuda.synchronize(dev)
+        sampler.window(False)
+        dist_util.barrier()
+        step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+        span_ms = ev[0][0].elapsed_time(ev[-1][1])
+
+        # per-stage device times of the same frames (events between the kernels; outside the graph)
+        stage_ms = {k: 0.0 for k in cb.CPE_STAGE_NAMES}
+        reps = max(3, min(20, K // max(1, n_frames)))
+        for i in range(n_frames):
+            if flush is not None:
+                flush.fill_(1)
+            ms = dec.profile(d_emb[i], d_fg[i], iters=reps if flush is None else 1, stream=stream)
+            for k, v in ms.items():
+                stage_ms[k] += v / n_frames
+    clocks = sampler.stop()
+
+    # sum of the per-step device times: excludes the L2 flush, includes every kernel and gap inside a step
+    total_ms = float(step_ms.sum())
+    t_max, px_total = dist_util.reduce_measurement(total_ms, float(cfg.pixels) * K, device=dev)
+    value = px_total / (t_max * 1e-3) / 1e6
+    p50, p95 = float(np.percentile(step_ms, 50)), float(np.percentile(step_ms, 95))
+
+    # ---- end to end through the host-buffer entry point (rank-local wall clock, max over ranks)
+    if args.quick:
+        print(json.dumps({"quick": True, "name": cfg.name, "p50_ms": p50, "value": value, "stage_ms": stage_ms}))
+        dec.close()
+        dist_util.shutdown()
+        return
+    hd = cb.HostDecoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    h_emb = [torch.from_numpy(f["emb"]).pin_memory() for f in frames]
+    h_fg = [torch.from_numpy(f["fg"]).pin_memory() for f in frames]
+    h_lab = torch.empty((cfg.B, cfg.H, cfg.W), dtype=torch.int32).pin_memory()
+    h_cen = torch.empty((cfg.B, cfg.K_max, 2), dtype=torch.float32).pin_memory()
+    h_cnt = torch.empty((cfg.B,), dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(K, int(3.0 / max(1e-4, cfg.emb_bytes / 20e9))))
+    for i in range(min(3, Wm)):
+        hd.decode(h_emb[i % n_frames], h_fg[i % n_frames], h_lab, h_cen, h_cnt)
+    dist_util.barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        hd.decode(h_emb[i % n_frames], h_fg[i % n_frames], h_lab, h_cen, h_cnt)
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    dist_util.barrier()
+    e_max, e_px = dist_util.reduce_measurement(e2e_ms, float(cfg.pixels) * e2e_steps, device=dev)
+    e2e_value = e_px / (e_max * 1e-3) / 1e6
+    count_last = h_cnt.numpy().copy()
+    h2d, d2h = hd.h2d_bytes, hd.d2h_bytes
+    hd.close()
+
+    all_clocks = dist_util.gather_objects(clocks)
+    if rank != 0:
+        dist_util.shutdown()
+        return
+
+    peak_gbs, peak_src = measured_peaks()
+    alg = algorithmic_bytes(cfg, int(np.mean(fg_pixels)))
+    dominant = max(stage_ms, key=lambda k: stage_ms[k])
+    achieved = alg[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
+    one_read_us = cfg.emb_bytes / (peak_gbs * 1e9) * 1e6
+    alg_total = sum(alg.values())
+    roofline = {
+        "bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+        "frac": achieved / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, dominant)),
+        "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[dominant],
+        "kernel_ms": stage_ms[dominant],
+        "stage_ms": stage_ms,
+        "stage_frac_of_peak": {k: (alg[k] / (v * 1e-3) / 1e9 / peak_gbs if v > 0 else None) for k, v in stage_ms.items()},
+        "end_to_end": {
+            "p50_ms": p50,
+            "one_read_embedding_roofline_us": one_read_us,
+            "frac_of_one_read_roofline": one_read_us / (p50 * 1e3),
+            "algorithmic_bytes": alg_total,
+            "frac_of_algorithmic_bytes_roofline": alg_total / (peak_gbs * 1e9) / (p50 * 1e-3),
+        },
+    }
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        threads = oracle.max_threads()
+        sec, sample = time_oracle(cfg, frames[0], 12.0, threads)
+        sec1, _ = time_oracle(cfg, frames[0], 4.0, 1)
+        cpu = {"value": cfg.pixels / sec / 1e6, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+               "single_thread_value": cfg.pixels / sec1 / 1e6}
+
+    worst = [c for c in all_clocks if c.get("sm_mhz")]
+    clk = dict(clocks)
+    if worst:
+        clk["sm_mhz"] = float(min(c["sm_mhz"] for c in worst))
+        clk["reasons"] = sorted(set(r for c in all_clocks for r in c.get("reasons", [])))
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": t_max / K, "p50_ms": p50, "p95_ms": p95, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": cfg.describe(), "name": cfg.name, "frames_per_rank": n_frames,
+            "l2": ("inputs rotate over %d frames, %.0f MB > L2" % (n_frames, n_frames * cfg.emb_bytes / 1e6)
+                   if flush is None else "a 252 MB buffer is rewritten between steps, outside the timed events"),
+            "launch": "one CUDA graph replay per step (%d kernels + 1 memset node)" % kernel_nodes,
+            "timing": "sum of per-step CUDA-event times on the launching stream; span of the region %.3f ms" % span_ms,
+            "parallelism": "independent frames per rank, no collective",
+            "instances_found_last_step": count_last.tolist(),
+        },
+        "clocks": clk,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e_max / e2e_steps,
+                "timing": "host wall clock around the synchronous host-buffer call, pinned buffers"},
+        "gpu_launches": kernel_nodes * K,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    dec.close()
+    dist_util.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="profiling runs: no clock pre-heat, no host-buffer leg, no CPU baseline (few launches)")
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup)
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -55,26 +55,39 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
 template <typename T>
 int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                        uint32_t* votes, uint32_t* counters, uint32_t* status) {
-  constexpr int V = cpe::Elem<T>::kVec;
-  const bool vec = ((uintptr_t)emb % 16 == 0) && (HW % V == 0) && (!fg || (uintptr_t)fg % V == 0);
   const T* e = static_cast<const T*>(emb);
-  const int per = vec ? V : 1;
-  const long long groups = ((long long)HW + per - 1) / per;
-  dim3 grid((unsigned)((groups + cpe::kVoteThreads - 1) / cpe::kVoteThreads), (unsigned)B);
-#define CPE_LAUNCH_VOTE(VEC_, FT_)                                                                             \
-  cpe::decode_vote_kernel<T, VEC_, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, F, p->levels, p->bins_w, \
-                                                                           p->bins_h, votes, counters, status)
+  constexpr int V = cpe::Elem<T>::kVec;
+  // 128-bit plane loads: every plane of every image must start on a 16-byte boundary
+  const bool vec = ((uintptr_t)emb % 16 == 0) && (HW % V == 0) && (!fg || (uintptr_t)fg % V == 0) &&
+                   (F == 4 || F == 8 || F == 16);
   if (vec) {
+    const long long groups = (long long)HW / V;
+    dim3 grid((unsigned)((groups + cpe::kVecGroups - 1) / cpe::kVecGroups), (unsigned)B);
+#define CPE_LAUNCH_VOTE(FT_)                                                                                   \
+  cpe::decode_vote_vec_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,      \
+                                                                         p->bins_h, votes, counters, status)
     switch (F) {
-      case 4: CPE_LAUNCH_VOTE(V, 4); break;
-      case 8: CPE_LAUNCH_VOTE(V, 8); break;
-      case 16: CPE_LAUNCH_VOTE(V, 16); break;
-      default: CPE_LAUNCH_VOTE(V, 0); break;
+      case 4: CPE_LAUNCH_VOTE(4); break;
+      case 8: CPE_LAUNCH_VOTE(8); break;
+      default: CPE_LAUNCH_VOTE(16); break;
     }
-  } else {
-    CPE_LAUNCH_VOTE(1, 0);
-  }
 #undef CPE_LAUNCH_VOTE
+  } else {
+    // 64-bit mask loads need every image's mask to start on an 8-byte boundary
+    const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
+    dim3 grid((unsigned)(((long long)HW + cpe::kVoteSpan - 1) / cpe::kVoteSpan), (unsigned)B);
+#define CPE_LAUNCH_VOTE(FT_)                                                                                       \
+  cpe::decode_vote_scalar_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, F, p->levels, p->bins_w,    \
+                                                                            p->bins_h, vec_mask, votes, counters, \
+                                                                            status)
+    switch (F) {
+      case 4: CPE_LAUNCH_VOTE(4); break;
+      case 8: CPE_LAUNCH_VOTE(8); break;
+      case 16: CPE_LAUNCH_VOTE(16); break;
+      default: CPE_LAUNCH_VOTE(0); break;
+    }
+#undef CPE_LAUNCH_VOTE
+  }
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }

@@ -1,6 +1,13 @@
 // Stage 1+2: per-pixel centroid estimate and hard-vote accumulation (hard-vote form of Eq. 6 on the
-// Eq. 9 bins).  HBM-bound: each participating pixel's 4F channel values are read once with 128-bit
-// loads from the channel planes; groups of pixels that do not participate are never fetched.
+// Eq. 9 bins).
+//
+// A CTA owns a span of consecutive pixels.  It first compacts the span's participating pixels into a
+// shared-memory list (mask bytes read with 64-bit loads), then walks that list with all lanes busy:
+// lane i of a warp decodes the i-th participating pixel, so background pixels cost neither arithmetic
+// nor embedding traffic (32-byte sectors that hold no participating pixel are never requested), and
+// consecutive lanes read consecutive addresses of each channel plane.  Votes are aggregated per warp
+// (one bin per warp is the common case), cached per CTA in a small shared-memory (bin -> count) table
+// and flushed with one global atomic per distinct bin per CTA.
 #pragma once
 
 #include "cpe_common.cuh"
@@ -8,6 +15,8 @@
 namespace cpe {
 
 constexpr int kVoteThreads = 256;
+constexpr int kVoteSpan = 2048;       // pixels per CTA (8 per thread in the mask pass)
+constexpr int kVotePix = 2;           // pixels decoded per thread per sweep of the list (independent chains)
 constexpr int kHashSlots = 512;       // per-CTA (bin -> count) cache in shared memory
 constexpr int kHashProbes = 16;
 constexpr uint32_t kHashEmpty = 0xffffffffu;
@@ -28,13 +37,66 @@ __device__ __forceinline__ void vote_cache_add(uint32_t* keys, uint32_t* cnts, u
   atomicAdd(&votes_img[cell], n);
 }
 
-// One thread owns VEC consecutive pixels (one 128-bit load per channel plane when VEC is the vector
-// width).  FT > 0 fixes F at compile time.
-template <typename T, int VEC, int FT>
+// Compacts the participating pixels of the CTA's span into s_list (offsets within the span, ascending).
+// Returns the number of entries.  `fg` may be NULL (all pixels participate).  Uses s_scan[9] as scratch.
+__device__ __forceinline__ int compact_span(const uint8_t* __restrict__ fg_img, long long span0, int HW, bool vec_mask,
+                                            uint16_t* s_list, int* s_scan) {
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const long long p0 = span0 + (long long)tid * 8;
+  uint32_t bits = 0;  // bit j: pixel p0 + j participates
+  if (p0 < HW) {
+    if (!fg_img) {
+      const long long left = HW - p0;
+      bits = left >= 8 ? 0xffu : ((1u << (int)left) - 1u);
+    } else if (vec_mask && p0 + 8 <= HW) {
+      const uint2 w = __ldg(reinterpret_cast<const uint2*>(fg_img + p0));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        bits |= (((w.x >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+        bits |= (((w.y >> (8 * j)) & 0xffu) ? 1u : 0u) << (4 + j);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (p0 + j < HW && __ldg(fg_img + p0 + j)) bits |= 1u << j;
+    }
+  }
+  const int mine = __popc(bits);
+  int incl = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) s_scan[wid] = incl;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+#pragma unroll
+    for (int w = 0; w < kVoteThreads / 32; ++w) {
+      const int t = s_scan[w];
+      s_scan[w] = run;
+      run += t;
+    }
+    s_scan[kVoteThreads / 32] = run;
+  }
+  __syncthreads();
+  int slot = s_scan[wid] + incl - mine;
+  while (bits) {
+    const int j = __ffs(bits) - 1;
+    bits &= bits - 1;
+    s_list[slot++] = (uint16_t)(tid * 8 + j);
+  }
+  __syncthreads();
+  return s_scan[kVoteThreads / 32];
+}
+
+// Scalar-load variant: any F, any alignment, any H*W.  FT > 0 fixes F at compile time.
+template <typename T, int FT>
 __global__ void __launch_bounds__(kVoteThreads)
-decode_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
-                   int bins_w, int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ counters,
-                   uint32_t* __restrict__ status) {
+decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
+                   int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
+                   uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
   const int b = blockIdx.y;
@@ -42,130 +104,286 @@ decode_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, in
   const int lane = tid & 31;
   const size_t plane = (size_t)HW;
   const T* e = emb + (size_t)b * 4 * F * plane;
+  const uint8_t* fg_img = fg ? fg + (size_t)b * plane : nullptr;
   uint32_t* votes_img = votes + (size_t)b * bins_w * bins_h;
+  const long long span0 = (long long)blockIdx.x * kVoteSpan;
 
   __shared__ uint32_t s_keys[kHashSlots];
   __shared__ uint32_t s_cnts[kHashSlots];
+  __shared__ uint16_t s_list[kVoteSpan];
+  __shared__ int s_scan[kVoteThreads / 32 + 1];
   __shared__ uint32_t s_nonfinite, s_voting;
   for (int i = tid; i < kHashSlots; i += kVoteThreads) {
     s_keys[i] = kHashEmpty;
     s_cnts[i] = 0;
   }
   if (tid == 0) s_nonfinite = s_voting = 0;
-  __syncthreads();
 
-  const long long n0 = ((long long)blockIdx.x * kVoteThreads + tid) * VEC;
-  bool take[VEC];
-  bool any = false;
+  const int n_active = compact_span(fg_img, span0, HW, vec_mask != 0, s_list, s_scan);  // has __syncthreads
+
+  const float half_w = (float)(bins_w + 1) * 0.5f, half_h = (float)(bins_h + 1) * 0.5f;
+  uint32_t nonfinite = 0, voted = 0;
+
+  // all threads of a warp run the same number of sweeps (warp collectives inside)
+  for (int base = 0; base < n_active; base += kVoteThreads * kVotePix) {
+    bool have[kVotePix];
+    const T* src[kVotePix];
 #pragma unroll
-  for (int j = 0; j < VEC; ++j) take[j] = false;
-  if (n0 < HW) {
-    if (fg) {
-      const uint8_t* m = fg + (size_t)b * plane + n0;
-      if constexpr (VEC == 8) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2*>(m));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          take[j] = ((w.x >> (8 * j)) & 0xffu) != 0;
-          take[4 + j] = ((w.y >> (8 * j)) & 0xffu) != 0;
-        }
-      } else if constexpr (VEC == 4) {
-        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(m));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) take[j] = ((w >> (8 * j)) & 0xffu) != 0;
-      } else {
-        take[0] = __ldg(m) != 0;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < VEC; ++j) take[j] = true;
+    for (int q = 0; q < kVotePix; ++q) {
+      const int i = base + q * kVoteThreads + tid;
+      have[q] = i < n_active;
+      const int off = have[q] ? (int)s_list[i] : 0;
+      src[q] = e + span0 + off;
     }
+    float p[kVotePix][2];
+    float fin[kVotePix];
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) any |= take[j];
-  }
-
-  int cell[VEC];
-#pragma unroll
-  for (int j = 0; j < VEC; ++j) cell[j] = -1;
-  uint32_t nonfinite = 0;
-
-  if (any) {
-    float p[2][VEC];
-    bool ok[VEC];
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) ok[j] = true;
+    for (int q = 0; q < kVotePix; ++q) fin[q] = 0.0f;
 #pragma unroll
     for (int axis = 0; axis < 2; ++axis) {
-      const T* ea = e + (size_t)axis * 2 * F * plane + n0;
-#pragma unroll 2
-      for (int l = 0; l < F; ++l) {
-        float s[VEC], c[VEC];
-        load_elems<T, VEC>(ea + (size_t)(2 * l) * plane, s);
-        load_elems<T, VEC>(ea + (size_t)(2 * l + 1) * plane, c);
-        const float scale = pow2f(l), inv = pow2f(-l);
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-          ok[j] = ok[j] && pair_finite(s[j], c[j]);
+      for (int l = 0; l < (FT > 0 ? FT : 16); ++l) {
+        if (FT == 0 && l >= F) break;
+        const size_t ch = ((size_t)axis * 2 * F + 2 * l) * plane;
+        float s[kVotePix], c[kVotePix];
+#pragma unroll
+        for (int q = 0; q < kVotePix; ++q) {
+          s[q] = have[q] ? Elem<T>::load1(src[q] + ch) : 0.0f;
+          c[q] = have[q] ? Elem<T>::load1(src[q] + ch + plane) : 1.0f;
+        }
+#pragma unroll
+        for (int q = 0; q < kVotePix; ++q) {
+          fin[q] = fold_finite(fin[q], s[q], c[q]);
           if (l < Fu) {
-            const float u = atan2_ht(s[j], c[j]);
-            p[axis][j] = (l == 0) ? u : refine(p[axis][j], u, scale, inv);
+            const float u = atan2_ht(s[q], c[q]);
+            p[q][axis] = (l == 0) ? u : refine_scaled(p[q][axis], u);
           }
         }
       }
     }
-    const float half_w = (float)(bins_w + 1) * 0.5f, half_h = (float)(bins_h + 1) * 0.5f;
+    const float unscale = pow2f(1 - Fu);
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-      if (take[j]) {
-        if (ok[j]) {
-          const int cx = cell_of(wrap_unit(p[0][j]), half_w, bins_w);
-          const int cy = cell_of(wrap_unit(p[1][j]), half_h, bins_h);
-          cell[j] = cy * bins_w + cx;
+    for (int q = 0; q < kVotePix; ++q) {
+      int cell = -1;
+      if (have[q]) {
+        if (fin[q] == fin[q]) {
+          const int cx = cell_of(wrap_unit(__fmul_rn(p[q][0], unscale)), half_w, bins_w);
+          const int cy = cell_of(wrap_unit(__fmul_rn(p[q][1], unscale)), half_h, bins_h);
+          cell = cy * bins_w + cx;
+          ++voted;
         } else {
           ++nonfinite;
         }
       }
-    }
-  }
-
-  // Warp-aggregated insertion into the CTA's cache.  Fast path: the whole warp votes for one bin.
-  {
-    int first = -1;
-    uint32_t mine = 0;
-    bool uniform = true;
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-      if (cell[j] >= 0) {
-        if (first < 0) first = cell[j];
-        uniform = uniform && (cell[j] == first);
-        ++mine;
-      }
-    }
-    const uint32_t voters = __ballot_sync(0xffffffffu, mine > 0);
-    if (voters) {
-      const uint32_t warp_votes = __reduce_add_sync(0xffffffffu, mine);
-      if (lane == 0) atomicAdd(&s_voting, warp_votes);
-      const int leader = __ffs(voters) - 1;
-      const int ref = __shfl_sync(0xffffffffu, first, leader);
-      const bool warp_uniform = __all_sync(0xffffffffu, mine == 0 || (uniform && first == ref));
-      if (warp_uniform) {
-        if (lane == leader) vote_cache_add(s_keys, s_cnts, (uint32_t)ref, warp_votes, votes_img);
-      } else {
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-          const int key = cell[j];
-          const uint32_t same = __match_any_sync(0xffffffffu, key);
-          if (key >= 0 && lane == __ffs(same) - 1)
-            vote_cache_add(s_keys, s_cnts, (uint32_t)key, (uint32_t)__popc(same), votes_img);
+      // warp-aggregated insertion; fast path: every voting lane of the warp names the same bin
+      const uint32_t voters = __ballot_sync(0xffffffffu, cell >= 0);
+      if (voters) {
+        const int leader = __ffs(voters) - 1;
+        const int ref = __shfl_sync(0xffffffffu, cell, leader);
+        if (__all_sync(0xffffffffu, cell < 0 || cell == ref)) {
+          if (lane == leader) vote_cache_add(s_keys, s_cnts, (uint32_t)ref, (uint32_t)__popc(voters), votes_img);
+        } else {
+          const uint32_t same = __match_any_sync(0xffffffffu, cell);
+          if (cell >= 0 && lane == __ffs(same) - 1)
+            vote_cache_add(s_keys, s_cnts, (uint32_t)cell, (uint32_t)__popc(same), votes_img);
         }
       }
     }
-    const uint32_t bad = __reduce_add_sync(0xffffffffu, nonfinite);
-    if (bad && lane == 0) atomicAdd(&s_nonfinite, bad);
+  }
+  const uint32_t wv = __reduce_add_sync(0xffffffffu, voted);
+  const uint32_t wb = __reduce_add_sync(0xffffffffu, nonfinite);
+  if (lane == 0) {
+    if (wv) atomicAdd(&s_voting, wv);
+    if (wb) atomicAdd(&s_nonfinite, wb);
   }
   __syncthreads();
 
   // Flush: one global atomic per distinct bin per CTA.
+  for (int i = tid; i < kHashSlots; i += kVoteThreads) {
+    const uint32_t k = s_keys[i];
+    if (k != kHashEmpty) atomicAdd(&votes_img[k], s_cnts[i]);
+  }
+  if (tid == 0 && s_voting) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_VOTING], s_voting);
+  if (tid == 0 && s_nonfinite) {
+    atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_NONFINITE], s_nonfinite);
+    atomicOr(status, (uint32_t)CPE_STATUS_NONFINITE);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Vector-load variant (the fast path): needs 16-byte aligned planes (emb 16-byte aligned, H*W a
+// multiple of the vector width) and F fixed at compile time.
+//
+// The unit of work is (group, axis): VEC consecutive pixels (one 128-bit load per channel plane) and
+// one of the two coordinate axes.  A CTA compacts the groups of its span that hold at least one
+// participating pixel, then each thread takes one (group, axis) item: it issues all 2F plane loads of
+// its axis at once (the only long-latency step), runs the coarse-to-fine estimate for its VEC pixels,
+// swaps results with its partner lane (same group, other axis) and turns half of the pixels into bins.
+constexpr int kVecGroups = 256;      // groups per CTA
+constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight together (2 loads each)
+
+template <typename T, int FT>
+__global__ void __launch_bounds__(kVoteThreads, 3)
+decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
+                       int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ counters,
+                       uint32_t* __restrict__ status) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int F = FT;
+  const int Fu = (levels > 0 && levels < F) ? levels : F;
+  const int b = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const size_t plane = (size_t)HW;
+  const T* e = emb + (size_t)b * 4 * F * plane;
+  uint32_t* votes_img = votes + (size_t)b * bins_w * bins_h;
+  const long long span0 = (long long)blockIdx.x * kVecGroups * VEC;
+
+  __shared__ uint32_t s_keys[kHashSlots];
+  __shared__ uint32_t s_cnts[kHashSlots];
+  __shared__ uint16_t s_grp[kVecGroups];   // low 8 bits: group index in the span; high 8 bits: participation bits
+  __shared__ int s_scan[kVoteThreads / 32 + 1];
+  __shared__ uint32_t s_nonfinite, s_voting;
+  for (int i = tid; i < kHashSlots; i += kVoteThreads) {
+    s_keys[i] = kHashEmpty;
+    s_cnts[i] = 0;
+  }
+  if (tid == 0) s_nonfinite = s_voting = 0;
+
+  // ---- which groups of the span hold a participating pixel (thread t looks at group t)
+  uint32_t bits = 0;
+  {
+    const long long p0 = span0 + (long long)tid * VEC;
+    if (p0 < HW) {  // H*W is a multiple of VEC: a group is never cut by the end of the image
+      if (!fg) {
+        bits = (1u << VEC) - 1u;
+      } else {
+        const uint8_t* m = fg + (size_t)b * plane + p0;
+        if constexpr (VEC == 8) {
+          const uint2 w = __ldg(reinterpret_cast<const uint2*>(m));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            bits |= (((w.x >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+            bits |= (((w.y >> (8 * j)) & 0xffu) ? 1u : 0u) << (4 + j);
+          }
+        } else {
+          const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(m));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) bits |= (((w >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+        }
+      }
+    }
+  }
+  const uint32_t act = __ballot_sync(0xffffffffu, bits != 0);
+  if (lane == 0) s_scan[wid] = __popc(act);
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+#pragma unroll
+    for (int w = 0; w < kVoteThreads / 32; ++w) {
+      const int t = s_scan[w];
+      s_scan[w] = run;
+      run += t;
+    }
+    s_scan[kVoteThreads / 32] = run;
+  }
+  __syncthreads();
+  if (bits) s_grp[s_scan[wid] + __popc(act & ((1u << lane) - 1u))] = (uint16_t)(tid | (bits << 8));
+  __syncthreads();
+  const int n_items = 2 * s_scan[kVoteThreads / 32];
+
+  const float half_w = (float)(bins_w + 1) * 0.5f, half_h = (float)(bins_h + 1) * 0.5f;
+  uint32_t nonfinite = 0, voted = 0;
+
+  for (int base = 0; base < n_items; base += kVoteThreads) {   // warp-uniform trip count
+    const int i = base + tid;
+    const bool have = i < n_items;
+    const uint32_t ent = have ? (uint32_t)s_grp[i >> 1] : 0u;
+    const int axis = i & 1;                    // lanes 2j and 2j+1 share a group
+    const uint32_t take = ent >> 8;
+    const T* src = e + span0 + (size_t)(ent & 0xffu) * VEC + (size_t)axis * 2 * F * plane;
+
+    float p[VEC];
+    uint32_t okbits = (1u << VEC) - 1u;
+    if (have) {
+      float fin[VEC];
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) fin[j] = 0.0f;
+      // the plane loads of up to 8 harmonics (16 x 128 bits) are in flight together, kept raw in registers
+      constexpr int LB = F < kVecLevelBatch ? F : kVecLevelBatch;
+#pragma unroll
+      for (int l0 = 0; l0 < F; l0 += LB) {
+        uint4 raw[2 * LB];
+#pragma unroll
+        for (int i = 0; i < 2 * LB; ++i)
+          raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + i) * plane));
+#pragma unroll
+        for (int ll = 0; ll < LB; ++ll) {
+          const int l = l0 + ll;
+          float s[VEC], c[VEC];
+          unpack_vec<T>(raw[2 * ll], s);
+          unpack_vec<T>(raw[2 * ll + 1], c);
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) {
+            fin[j] = fold_finite(fin[j], s[j], c[j]);
+            if (l < Fu) {
+              const float u = atan2_ht(s[j], c[j]);
+              p[j] = (l == 0) ? u : refine_scaled(p[j], u);
+            }
+          }
+        }
+      }
+      const float unscale = pow2f(1 - Fu);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        p[j] = __fmul_rn(p[j], unscale);
+        if (fin[j] != fin[j]) okbits &= ~(1u << j);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) p[j] = 0.0f;
+    }
+    // swap with the partner lane: afterwards every lane knows both coordinates of its half of the pixels
+    const uint32_t ok_other = __shfl_xor_sync(0xffffffffu, okbits, 1);
+    const uint32_t ok_both = okbits & ok_other;
+    float other[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) other[j] = __shfl_xor_sync(0xffffffffu, p[j], 1);
+#pragma unroll
+    for (int jj = 0; jj < VEC / 2; ++jj) {
+      const int j = axis * (VEC / 2) + jj;       // axis-0 lane finishes the first half, axis-1 lane the second
+      float px = axis == 0 ? p[jj] : other[VEC / 2 + jj];
+      float py = axis == 0 ? other[jj] : p[VEC / 2 + jj];
+      int cell = -1;
+      if (have && ((take >> j) & 1u)) {
+        if ((ok_both >> j) & 1u) {
+          const int cx = cell_of(wrap_unit(px), half_w, bins_w);
+          const int cy = cell_of(wrap_unit(py), half_h, bins_h);
+          cell = cy * bins_w + cx;
+          ++voted;
+        } else {
+          ++nonfinite;
+        }
+      }
+      const uint32_t voters = __ballot_sync(0xffffffffu, cell >= 0);
+      if (voters) {
+        const int leader = __ffs(voters) - 1;
+        const int ref = __shfl_sync(0xffffffffu, cell, leader);
+        if (__all_sync(0xffffffffu, cell < 0 || cell == ref)) {
+          if (lane == leader) vote_cache_add(s_keys, s_cnts, (uint32_t)ref, (uint32_t)__popc(voters), votes_img);
+        } else {
+          const uint32_t same = __match_any_sync(0xffffffffu, cell);
+          if (cell >= 0 && lane == __ffs(same) - 1)
+            vote_cache_add(s_keys, s_cnts, (uint32_t)cell, (uint32_t)__popc(same), votes_img);
+        }
+      }
+    }
+  }
+  const uint32_t wv = __reduce_add_sync(0xffffffffu, voted);
+  const uint32_t wb = __reduce_add_sync(0xffffffffu, nonfinite);
+  if (lane == 0) {
+    if (wv) atomicAdd(&s_voting, wv);
+    if (wb) atomicAdd(&s_nonfinite, wb);
+  }
+  __syncthreads();
   for (int i = tid; i < kHashSlots; i += kVoteThreads) {
     const uint32_t k = s_keys[i];
     if (k != kHashEmpty) atomicAdd(&votes_img[k], s_cnts[i]);
