@@ -54,7 +54,9 @@ enum {
 
 /* cpe_params.flags */
 enum {
-  CPE_FLAG_WRITE_SCORES = 1u  /* also store the best and second-best Eq. 4 distance of every pixel */
+  CPE_FLAG_WRITE_SCORES = 1u, /* also store the best and second-best Eq. 4 distance of every pixel */
+  CPE_FLAG_EXACT_ASSIGN = 2u  /* score every (pixel, peak) pair in binary32 on the plain ALUs instead of
+                                 filtering with the tensor cores first; same results, for cross-checking */
 };
 
 /* bits of the device status word */

@@ -5,10 +5,12 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
 #include "assign.cuh"
+#include "assign_mma.cuh"
 #include "cpe.h"
 #include "cpe_common.cuh"
 #include "decode_vote.cuh"
@@ -93,9 +95,9 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
 }
 
 template <typename T>
-int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                  const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                  uint32_t* counters) {
+int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                        const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                        uint32_t* counters) {
   const T* e = static_cast<const T*>(emb);
   dim3 grid((unsigned)(((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads), (unsigned)B);
 #define CPE_LAUNCH_ASSIGN(FT_)                                                                                  \
@@ -110,6 +112,58 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
 #undef CPE_LAUNCH_ASSIGN
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
+}
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+template <typename T, int KA, bool WANT2>
+int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                        const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                        uint32_t* counters) {
+  const int cap_limit = KA == 16 ? cpe::kAmPeakCap : 320;
+  const int peak_cap = std::min(cap_limit, (p->max_instances + 7) & ~7);
+  const int smem = cpe::am_smem_layout(KA, peak_cap).total;
+  auto kern = cpe::assign_mma_kernel<T, KA, WANT2>;
+  static bool configured = false;   // per instantiation; the attribute is sticky for the process
+  if (!configured) {
+    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+    configured = true;
+  }
+  const int n_spans = (HW + cpe::kAmSpan - 1) / cpe::kAmSpan;
+  const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
+  dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
+  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
+  const int need_exact = p->tau < INFINITY ? 1 : 0;
+  kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
+                                            peak_cap, vec_mask, labels, best, second, counters);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
+template <typename T>
+int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                  const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                  uint32_t* counters) {
+  if (p->flags & CPE_FLAG_EXACT_ASSIGN)
+    return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
+  const T* e = static_cast<const T*>(emb);
+  const bool want2 = best != nullptr;
+  if (F <= 8) {
+    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters)
+                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
+  }
+  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters)
+               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
 }
 
 // The chain.  `ev`, when given, holds CPE_STAGE_N + 1 events recorded around the stages.

@@ -8,12 +8,14 @@ MARGIN = 1e-5      # label differences are excused where the oracle's top-2 dist
 REL = 1e-4         # relative tolerance of float scores and centroids
 
 
-def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, scores=True, mode="direct"):
+def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, scores=True, mode="direct",
+            exact_assign=False):
     import torch
     B, D, H, W = emb.shape
     F = D // 4
     dtype = "f32" if emb.dtype == np.float32 else "f16"
-    dec = cb.Decoder(B, H, W, F, dtype, bins_w, bins_h, T_v, float(tau), K_max, levels, write_scores=scores)
+    dec = cb.Decoder(B, H, W, F, dtype, bins_w, bins_h, T_v, float(tau), K_max, levels, write_scores=scores,
+                     exact_assign=exact_assign)
     d_emb = torch.from_numpy(emb).cuda()
     d_fg = None if fg is None else torch.from_numpy(np.ascontiguousarray(fg, np.uint8)).cuda()
     if mode == "direct":
@@ -92,4 +94,9 @@ def check_case(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0,
     rep = compare_labels(gpu["labels"], gpu["best"], gpu["second"], ora["labels"], ora["best"], ora["second"])
     if rep["excused_mismatches"] == 0:
         assert np.array_equal(gpu["counters"][:, cb.CPE_CNT_TAU_REJECTED], ora["counters"][:, oracle.CNT_TAU_REJECTED])
+    # the production configuration: no score output (the filter may then decide a pixel without re-scoring it)
+    fast = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, levels, False, mode)
+    compare_front(fast, ora, F, bins_w, bins_h)
+    rep2 = compare_labels(fast["labels"], None, None, ora["labels"], ora["best"], ora["second"])
+    rep["excused_mismatches_no_scores"] = rep2["excused_mismatches"]
     return gpu, ora, rep

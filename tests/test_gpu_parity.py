@@ -117,6 +117,40 @@ def test_threshold_and_tie_rules_on_constructed_votes():
     assert gpu["peak_cell"][0, :3].tolist() == sorted([3 * bw + 3, 12 * bw + 10, 2 * bw + 13])
 
 
+@pytest.mark.parametrize("name,over", [("c2", dict(H=192, W=256, K=12)), ("c5", dict(H=256, W=256, K=40, bins_w=128, bins_h=128)),
+                                       ("c3", dict(H=99, W=121, K=8, bins_w=64, bins_h=32))])
+def test_exact_all_pairs_assignment_agrees(name, over):
+    # the plain-ALU kernel that scores every (pixel, peak) pair and the tensor-core filtered kernel must agree bit for bit
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 1)
+    a = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, exact_assign=True)
+    b = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, exact_assign=False)
+    c = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, exact_assign=False, scores=False)
+    assert np.array_equal(a["labels"], b["labels"]) and np.array_equal(a["labels"], c["labels"])
+    assert np.array_equal(a["best"].view(np.uint32), b["best"].view(np.uint32))
+    assert np.array_equal(a["second"].view(np.uint32), b["second"].view(np.uint32))
+    ora = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)
+    compare_labels(a["labels"], a["best"], a["second"], ora["labels"], ora["best"], ora["second"])
+
+
+def test_many_peaks_and_fp32_out_of_half_range():
+    # more peaks than fit the resident peak operand (several peak chunks), and binary32 pixels too large for binary16
+    rng = np.random.default_rng(5)
+    H, W, F, bw, bh = 96, 128, 4, 64, 48
+    K = 600
+    cells = np.sort(rng.choice(bw // 2 * (bh // 2), K, replace=False))
+    cx, cy = 2 * (cells % (bw // 2)), 2 * (cells // (bw // 2))          # no two peaks adjacent
+    inst = np.zeros((H, W), np.int32)
+    inst.ravel()[:] = (np.arange(H * W) // 20) % K + 1                     # 20 pixels per run: every bin gets > T_v votes
+    cents = np.stack([-1 + 2 * (cx + 1) / (bw + 1), -1 + 2 * (cy + 1) / (bh + 1)], 1)
+    emb = wl.encode(inst, cents, F, 0.02, rng, np.float32)[None]
+    emb[0, 3, 5, 7] = 1e5
+    emb[0, 9, 50, 60] = -7e4
+    fg = np.ones((1, H, W), np.uint8)
+    gpu, ora, rep = check_case(emb, fg, bw, bh, T_v=8, K_max=1024)
+    assert ora["count"][0] == K
+
+
 def test_host_front_end_matches_device_path():
     cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=96, W=104, K=10, bins_w=24, bins_h=24)
     fr = wl.make_frame(cfg, 0)
