@@ -274,7 +274,9 @@ def run_ours(args, cfg):
 
     # ---- end to end through the host-buffer entry point (rank-local wall clock, max over ranks)
     if args.quick:
-        print(json.dumps({"quick": True, "name": cfg.name, "p50_ms": p50, "value": value, "stage_ms": stage_ms}))
+        cnt = dec.intermediate(cb.CPE_INT_COUNTERS).cpu().numpy().sum(0).tolist()
+        print(json.dumps({"quick": True, "name": cfg.name, "p50_ms": p50, "value": value, "stage_ms": stage_ms,
+                          "counters": cnt}))
         dec.close()
         dist_util.shutdown()
         return

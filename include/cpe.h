@@ -62,7 +62,9 @@ enum {
 /* bits of the device status word */
 enum {
   CPE_STATUS_PEAK_OVERFLOW = 1u, /* an image had more local maxima than max_instances            */
-  CPE_STATUS_NONFINITE = 2u      /* at least one participating pixel had a non-finite channel    */
+  CPE_STATUS_NONFINITE = 2u,     /* at least one participating pixel had a non-finite channel    */
+  CPE_STATUS_INTERNAL = 4u       /* an index self-check failed (site code in bits 8..15); the access was
+                                    skipped.  Never set by a correct build: please report it.      */
 };
 
 /* per-image counters, uint32 [B][CPE_CNT_N] */
@@ -72,6 +74,9 @@ enum {
   CPE_CNT_RAW_PEAKS = 2,    /* local maxima found before truncation to max_instances        */
   CPE_CNT_TRUNCATED = 3,    /* local maxima dropped by the truncation                       */
   CPE_CNT_TAU_REJECTED = 4, /* pixels whose best distance was not below tau (label 0)       */
+  CPE_CNT_FILTER_PAIRS = 5, /* (pixel, peak) pairs that survived the tensor-core filter     */
+  CPE_CNT_RESCORED = 6,     /* pixels decided by exact re-scoring of several candidates     */
+  CPE_CNT_FULL_SCORED = 7,  /* pixels for which every peak was scored exactly               */
   CPE_CNT_N = 8
 };
 

@@ -22,8 +22,9 @@ CPE_ERR_NULL, CPE_ERR_SIZE, CPE_ERR_DTYPE, CPE_ERR_ALIGN, CPE_ERR_WORKSPACE = -1
 CPE_ERR_PARAM, CPE_ERR_CUDA, CPE_ERR_WHICH, CPE_ERR_NOMEM = -6, -7, -8, -9
 CPE_FLAG_WRITE_SCORES = 1
 CPE_FLAG_EXACT_ASSIGN = 2
-CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE = 1, 2
-CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED, CPE_CNT_N = 0, 1, 2, 3, 4, 8
+CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL = 1, 2, 4
+CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
+CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8
 (CPE_INT_VOTES, CPE_INT_PEAK_CELLS, CPE_INT_PEAK_VOTES, CPE_INT_PEAK_EMB, CPE_INT_PALETTE_W, CPE_INT_PALETTE_H,
  CPE_INT_BEST_SCORE, CPE_INT_SECOND_SCORE, CPE_INT_STATUS, CPE_INT_COUNTERS) = range(10)
 CPE_STAGE_NAMES = ("clear", "decode_vote", "peaks", "compact", "assign")

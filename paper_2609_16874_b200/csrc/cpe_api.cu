@@ -129,23 +129,29 @@ int sm_count() {
 template <typename T, int KA, bool WANT2>
 int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                         const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                        uint32_t* counters) {
-  const int cap_limit = KA == 16 ? cpe::kAmPeakCap : 320;
-  const int peak_cap = std::min(cap_limit, (p->max_instances + 7) & ~7);
-  const int smem = cpe::am_smem_layout(KA, peak_cap).total;
+                        uint32_t* counters, uint32_t* status) {
+  // small inputs get short spans so that there are enough CTAs to fill the GPU
+  const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
+  // as many peaks resident in shared memory as leave room for two CTAs per SM
+  int peak_cap = (p->max_instances + 7) & ~7;
+  const int budget = 110 * 1024;
+  const int fixed = cpe::am_smem_layout(KA, 0, span).total;
+  peak_cap = std::max(8, std::min(peak_cap, ((budget - fixed) / ((2 * KA + 8) * 2)) & ~7));
+  const int smem = cpe::am_smem_layout(KA, peak_cap, span).total;
   auto kern = cpe::assign_mma_kernel<T, KA, WANT2>;
   static bool configured = false;   // per instantiation; the attribute is sticky for the process
   if (!configured) {
     CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
     configured = true;
   }
-  const int n_spans = (HW + cpe::kAmSpan - 1) / cpe::kAmSpan;
+  const int n_spans = (HW + span - 1) / span;
   const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
   dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
   const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
-  const int need_exact = p->tau < INFINITY ? 1 : 0;
+  int need_exact = p->tau < INFINITY ? 1 : 0;
+  if (const char* ph = getenv("CPE_DEBUG_PHASE")) need_exact |= (atoi(ph) & 0xf) << 8;   // timing experiments
   kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
-                                            peak_cap, vec_mask, labels, best, second, counters);
+                                            peak_cap, span, vec_mask, labels, best, second, counters, status);
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -153,17 +159,32 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
 template <typename T>
 int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                   const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                  uint32_t* counters) {
+                  uint32_t* counters, uint32_t* status) {
   if (p->flags & CPE_FLAG_EXACT_ASSIGN)
     return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
   const T* e = static_cast<const T*>(emb);
   const bool want2 = best != nullptr;
   if (F <= 8) {
-    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters)
-                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
+    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status)
+                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status);
   }
-  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters)
-               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
+  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status)
+               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status);
+}
+
+// CPE_DEBUG_SYNC=1 in the environment: wait after every stage and name the stage whose kernel failed
+// (never inside stream capture).
+int debug_stage_check(cudaStream_t st, const char* stage) {
+  static const bool on = getenv("CPE_DEBUG_SYNC") != nullptr;
+  if (!on) return CPE_OK;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone) return CPE_OK;
+  cudaError_t e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    fprintf(stderr, "[cpe] stage %s failed: %s\n", stage, cudaGetErrorString(e));
+    return cuda_fail(e);
+  }
+  return CPE_OK;
 }
 
 // The chain.  `ev`, when given, holds CPE_STAGE_N + 1 events recorded around the stages.
@@ -197,6 +218,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, counters, status)
                            : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, counters, status);
   if (rc) return rc;
+  if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_PEAKS], st));
   {
@@ -212,12 +234,14 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
       bitmap, votes, p->bins_w, p->bins_h, L.words, p->max_instances, F, H, W, pal_w, pal_h, peak_cell, peak_votes,
       peak_emb, out_centroids, out_count, counters, status);
   CPE_CUDA(cudaGetLastError());
+  if ((rc = debug_stage_check(st, "peaks"))) return rc;
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_ASSIGN], st));
   rc = p->dtype == CPE_F32
-           ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters)
-           : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters);
+           ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters, status)
+           : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters, status);
   if (rc) return rc;
+  if ((rc = debug_stage_check(st, "assign"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
   return CPE_OK;
 }

@@ -53,6 +53,7 @@ def compare_front(gpu, ora, F, bins_w, bins_h):
     """Palettes, votes, peak list, counts, centroids, counters: bit-exact except the float centroids."""
     assert np.array_equal(gpu["pal_w"].view(np.uint32), oracle.palette(bins_w, F).view(np.uint32))
     assert np.array_equal(gpu["pal_h"].view(np.uint32), oracle.palette(bins_h, F).view(np.uint32))
+    assert not (gpu["status"] & cb.CPE_STATUS_INTERNAL), hex(gpu["status"])      # no index self-check fired
     assert np.array_equal(gpu["votes"], ora["votes"]), "vote map differs"
     assert np.array_equal(gpu["count"], ora["count"]), (gpu["count"], ora["count"])
     Pw, Ph = oracle.palette(bins_w, F), oracle.palette(bins_h, F)
