@@ -55,11 +55,16 @@ enum {
 /* cpe_params.flags */
 enum {
   CPE_FLAG_WRITE_SCORES = 1u, /* also store the best and second-best Eq. 4 distance of every pixel */
-  CPE_FLAG_EXACT_ASSIGN = 2u  /* score every (pixel, peak) pair in binary32 on the plain ALUs instead of
+  CPE_FLAG_EXACT_ASSIGN = 2u, /* score every (pixel, peak) pair in binary32 on the plain ALUs instead of
                                  filtering with the tensor cores first; same results, for cross-checking */
+  CPE_FLAG_FILTER_ASSIGN = 8u,/* use the tensor-core filtered kernel for every image, however few peaks it has
+                                 (by default images with few peaks take the all-pairs kernel); same results   */
+  CPE_FLAG_KEEP_VOTES = 4u    /* leave the vote map readable after the decode (CPE_INT_VOTES).  Without it the
+                                 last kernel of a decode re-zeroes the map for the next decode, which saves the
+                                 clearing pass at the start; with it every decode starts with that pass.       */
 };
 
-/* bits of the device status word */
+/* bits of the per-image device status words */
 enum {
   CPE_STATUS_PEAK_OVERFLOW = 1u, /* an image had more local maxima than max_instances            */
   CPE_STATUS_NONFINITE = 2u,     /* at least one participating pixel had a non-finite channel    */
@@ -82,7 +87,7 @@ enum {
 
 /* ids for cpe_get_intermediate */
 enum {
-  CPE_INT_VOTES = 0,        /* uint32 [B][bins_h][bins_w]       hard-vote map                   */
+  CPE_INT_VOTES = 0,        /* uint32 [B][bins_h][bins_w]       hard-vote map (CPE_FLAG_KEEP_VOTES)  */
   CPE_INT_PEAK_CELLS = 1,   /* int32  [B][max_instances]        linear bin cy*bins_w+cx, ascending */
   CPE_INT_PEAK_VOTES = 2,   /* uint32 [B][max_instances]        votes of each kept peak         */
   CPE_INT_PEAK_EMB = 3,     /* float  [B][max_instances][4F]    concat(P_w[cx], P_h[cy])        */
@@ -90,18 +95,18 @@ enum {
   CPE_INT_PALETTE_H = 5,    /* float  [bins_h][2F]                                              */
   CPE_INT_BEST_SCORE = 6,   /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
   CPE_INT_SECOND_SCORE = 7, /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
-  CPE_INT_STATUS = 8,       /* uint32 [1]                                                       */
+  CPE_INT_STATUS = 8,       /* uint32 [B]                       CPE_STATUS_* bits of each image      */
   CPE_INT_COUNTERS = 9,     /* uint32 [B][CPE_CNT_N]                                            */
   CPE_INT_N = 10
 };
 
 /* stages reported by cpe_profile_decode */
 enum {
-  CPE_STAGE_CLEAR = 0,      /* zeroing of the vote map, counters and status                    */
+  CPE_STAGE_CLEAR = 0,      /* zeroing of the vote map (only with CPE_FLAG_KEEP_VOTES; else ~0)  */
   CPE_STAGE_DECODE_VOTE = 1,
-  CPE_STAGE_PEAKS = 2,      /* local-maximum test over the vote map                            */
-  CPE_STAGE_COMPACT = 3,    /* ordered peak list, centroids, peak embeddings                   */
-  CPE_STAGE_ASSIGN = 4,     /* assignment and label-map write                                  */
+  CPE_STAGE_PEAKS = 2,      /* local-maximum test, ordered peak list, centroids, peak embeddings */
+  CPE_STAGE_COMPACT = 3,    /* (merged into CPE_STAGE_PEAKS; reported as ~0)                     */
+  CPE_STAGE_ASSIGN = 4,     /* assignment and label-map write                                    */
   CPE_STAGE_N = 5
 };
 

@@ -22,6 +22,8 @@ CPE_ERR_NULL, CPE_ERR_SIZE, CPE_ERR_DTYPE, CPE_ERR_ALIGN, CPE_ERR_WORKSPACE = -1
 CPE_ERR_PARAM, CPE_ERR_CUDA, CPE_ERR_WHICH, CPE_ERR_NOMEM = -6, -7, -8, -9
 CPE_FLAG_WRITE_SCORES = 1
 CPE_FLAG_EXACT_ASSIGN = 2
+CPE_FLAG_KEEP_VOTES = 4
+CPE_FLAG_FILTER_ASSIGN = 8
 CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL = 1, 2, 4
 CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
 CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8
@@ -210,14 +212,15 @@ class Decoder:
     """Holds the parameter struct, the workspace and the output tensors for one problem shape on one device."""
 
     def __init__(self, B, H, W, F, dtype, bins_w, bins_h, vote_threshold=8, tau=math.inf, max_instances=1024,
-                 levels=0, write_scores=False, device="cuda:0", exact_assign=False):
+                 levels=0, write_scores=False, device="cuda:0", exact_assign=False, keep_votes=False, filter_assign=False):
         import torch
         self.torch = torch
         self.B, self.H, self.W, self.F = B, H, W, F
         self.device = torch.device(device)
         code = {"f32": CPE_F32, "f16": CPE_F16, torch.float32: CPE_F32, torch.float16: CPE_F16}[dtype]
         self.emb_dtype = torch.float32 if code == CPE_F32 else torch.float16
-        flags = (CPE_FLAG_WRITE_SCORES if write_scores else 0) | (CPE_FLAG_EXACT_ASSIGN if exact_assign else 0)
+        flags = ((CPE_FLAG_WRITE_SCORES if write_scores else 0) | (CPE_FLAG_EXACT_ASSIGN if exact_assign else 0) |
+                 (CPE_FLAG_KEEP_VOTES if keep_votes else 0) | (CPE_FLAG_FILTER_ASSIGN if filter_assign else 0))
         self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances, flags)
         n = cpe_workspace_size(B, H, W, F, self.params)
         if n == 0:
@@ -286,7 +289,7 @@ class Decoder:
             CPE_INT_PALETTE_H: (torch.float32, (bh, 2 * self.F)),
             CPE_INT_BEST_SCORE: (torch.float32, (self.B, self.H, self.W)),
             CPE_INT_SECOND_SCORE: (torch.float32, (self.B, self.H, self.W)),
-            CPE_INT_STATUS: (torch.int32, (1,)),
+            CPE_INT_STATUS: (torch.int32, (self.B,)),
             CPE_INT_COUNTERS: (torch.int32, (self.B, CPE_CNT_N)),
         }
         dt, shape = shapes[which]

@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kAssignThreads)
 assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int K_max,
               const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau,
               int32_t* __restrict__ labels, float* __restrict__ best, float* __restrict__ second,
-              uint32_t* __restrict__ counters) {
+              uint32_t* __restrict__ counters, uint32_t* __restrict__ votes, int cells, int k_limit) {
   constexpr int DT = FT > 0 ? 4 * FT : 64;
   const int F = FT > 0 ? FT : F_rt;
   const int D = 4 * F;
@@ -65,11 +65,14 @@ assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW,
   const long long n = (long long)blockIdx.x * kAssignThreads + tid;
   const size_t plane = (size_t)HW;
   const int K = count_ptr[b];
+  if (K > k_limit) return;   // this image is left to the tensor-core kernel launched next to this one
   const float* pk_img = peak_emb + (size_t)b * K_max * D;
 
   __shared__ __align__(16) float s_pk[kPeakChunk * 64];
   __shared__ uint32_t s_rejected;
   if (tid == 0) s_rejected = 0;
+  // the vote map has no reader left: leave it zero for the next decode (votes == NULL keeps it)
+  if (votes) zero_votes_share(votes + (size_t)b * cells, cells, (int)blockIdx.x, (int)gridDim.x);
 
   bool act = n < HW;
   if (act && fg) act = __ldg(fg + (size_t)b * plane + n) != 0;

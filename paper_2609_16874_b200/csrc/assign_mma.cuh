@@ -109,7 +109,8 @@ __global__ void __launch_bounds__(kAmThreads, 2)
 assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
                   const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
                   int peak_cap, int span, int vec_mask, int32_t* __restrict__ labels, float* __restrict__ best,
-                  float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
+                  float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
+                  uint32_t* __restrict__ votes, int cells, int k_min) {
   constexpr int PKP = 2 * KA + 8;     // peak row pitch in halves
   constexpr int KS = KA / 16;         // k-steps per axis
   extern __shared__ __align__(16) unsigned char smem[];
@@ -135,12 +136,16 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int g = lane >> 2, t4 = lane & 3;
+  uint32_t* status = status_all + b;
+  // the vote map has no reader left: leave it zero for the next decode (votes == NULL keeps it)
+  if (votes) zero_votes_share(votes + (size_t)b * cells, cells, (int)blockIdx.x, (int)gridDim.x);
   const size_t plane = (size_t)HW;
   const int D = 4 * F;
   const T* e_img = emb + (size_t)b * D * plane;
   const uint8_t* fg_img = fg ? fg + (size_t)b * plane : nullptr;
   const float* pk_img = peak_emb + (size_t)b * K_max * D;
   const int K = count_ptr[b];
+  if (K < k_min) return;     // few peaks: this image is done by the plain all-pairs kernel launched next to this one
   const float inf = __int_as_float(0x7f800000);
   const int n_spans = (HW + span - 1) / span;
   const int n_pchunks = K > 0 ? (K + peak_cap - 1) / peak_cap : 0;

@@ -56,7 +56,7 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
 
 template <typename T>
 int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                       uint32_t* votes, uint32_t* counters, uint32_t* status) {
+                       uint32_t* votes, uint32_t* acc) {
   const T* e = static_cast<const T*>(emb);
   constexpr int V = cpe::Elem<T>::kVec;
   // 128-bit plane loads: every plane of every image must start on a 16-byte boundary
@@ -67,7 +67,7 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
     dim3 grid((unsigned)((groups + cpe::kVecGroups - 1) / cpe::kVecGroups), (unsigned)B);
 #define CPE_LAUNCH_VOTE(FT_)                                                                                   \
   cpe::decode_vote_vec_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,      \
-                                                                         p->bins_h, votes, counters, status)
+                                                                         p->bins_h, votes, acc)
     switch (F) {
       case 4: CPE_LAUNCH_VOTE(4); break;
       case 8: CPE_LAUNCH_VOTE(8); break;
@@ -80,8 +80,7 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
     dim3 grid((unsigned)(((long long)HW + cpe::kVoteSpan - 1) / cpe::kVoteSpan), (unsigned)B);
 #define CPE_LAUNCH_VOTE(FT_)                                                                                       \
   cpe::decode_vote_scalar_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, F, p->levels, p->bins_w,    \
-                                                                            p->bins_h, vec_mask, votes, counters, \
-                                                                            status)
+                                                                            p->bins_h, vec_mask, votes, acc)
     switch (F) {
       case 4: CPE_LAUNCH_VOTE(4); break;
       case 8: CPE_LAUNCH_VOTE(8); break;
@@ -97,12 +96,13 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
 template <typename T>
 int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                         const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                        uint32_t* counters) {
+                        uint32_t* counters, uint32_t* votes_to_zero, int cells, int k_limit) {
   const T* e = static_cast<const T*>(emb);
   dim3 grid((unsigned)(((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads), (unsigned)B);
 #define CPE_LAUNCH_ASSIGN(FT_)                                                                                  \
   cpe::assign_kernel<T, FT_><<<grid, cpe::kAssignThreads, 0, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, \
-                                                                  p->tau, labels, best, second, counters)
+                                                                  p->tau, labels, best, second, counters, votes_to_zero, cells, \
+                                                                  k_limit)
   switch (F) {
     case 4: CPE_LAUNCH_ASSIGN(4); break;
     case 8: CPE_LAUNCH_ASSIGN(8); break;
@@ -129,7 +129,7 @@ int sm_count() {
 template <typename T, int KA, bool WANT2>
 int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                         const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                        uint32_t* counters, uint32_t* status) {
+                        uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min) {
   // small inputs get short spans so that there are enough CTAs to fill the GPU
   const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
   // as many peaks resident in shared memory as leave room for two CTAs per SM
@@ -151,7 +151,8 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   int need_exact = p->tau < INFINITY ? 1 : 0;
   if (const char* ph = getenv("CPE_DEBUG_PHASE")) need_exact |= (atoi(ph) & 0xf) << 8;   // timing experiments
   kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
-                                            peak_cap, span, vec_mask, labels, best, second, counters, status);
+                                            peak_cap, span, vec_mask, labels, best, second, counters, status, votes_to_zero,
+                                            cells, k_min);
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -159,17 +160,30 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
 template <typename T>
 int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                   const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                  uint32_t* counters, uint32_t* status) {
+                  uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells) {
   if (p->flags & CPE_FLAG_EXACT_ASSIGN)
-    return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters);
+    return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                  votes_to_zero, cells, 0x7fffffff);
+  // The number of peaks is only known on the device.  Two kernels are enqueued and every image is done by
+  // exactly one of them: all pairs on the plain ALUs when an image has few peaks (the fixed cost of the
+  // tensor-core filter does not pay), the filtered kernel otherwise.  The other kernel's CTAs exit at once.
+  const int k_limit = (p->flags & CPE_FLAG_FILTER_ASSIGN) ? 0 : (F <= 8 ? 32 : 16);
+  int rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
+                                  cells, k_limit);
+  if (rc) return rc;
   const T* e = static_cast<const T*>(emb);
   const bool want2 = best != nullptr;
+  const int k_min = k_limit + 1;
   if (F <= 8) {
-    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status)
-                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status);
+    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                                    status, votes_to_zero, cells, k_min)
+                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                     counters, status, votes_to_zero, cells, k_min);
   }
-  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status)
-               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, status);
+  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                                  status, votes_to_zero, cells, k_min)
+               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                   counters, status, votes_to_zero, cells, k_min);
 }
 
 // CPE_DEBUG_SYNC=1 in the environment: wait after every stage and name the stage whose kernel failed
@@ -211,12 +225,16 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   float* second = (p->flags & CPE_FLAG_WRITE_SCORES) ? reinterpret_cast<float*>(ws + L.second) : nullptr;
   const int HW = H * W;
 
+  uint32_t* acc = reinterpret_cast<uint32_t*>(ws + L.acc);
+  const bool keep_votes = (p->flags & CPE_FLAG_KEEP_VOTES) != 0;
+
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_CLEAR], st));
-  CPE_CUDA(cudaMemsetAsync(ws + L.status, 0, L.clear_end - L.status, st));
+  // Normally the map is already zero (cpe_init_workspace, then the previous decode's last kernel).
+  if (keep_votes) CPE_CUDA(cudaMemsetAsync(ws + L.votes, 0, L.votes_end - L.votes, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
-  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, counters, status)
-                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, counters, status);
+  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, acc)
+                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, acc);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
@@ -224,22 +242,21 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   {
     const int warps_per_cta = cpe::kPeakThreads / 32;
     dim3 grid((unsigned)((L.words + warps_per_cta - 1) / warps_per_cta), (unsigned)B);
-    cpe::peaks_bitmap_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
-                                                                 (uint32_t)p->vote_threshold, bitmap);
+    cpe::peaks_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
+                                                          (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W,
+                                                          pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids,
+                                                          out_count, acc, counters, status);
     CPE_CUDA(cudaGetLastError());
   }
-
-  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_COMPACT], st));
-  cpe::peaks_compact_kernel<<<(unsigned)B, cpe::kCompactThreads, 0, st>>>(
-      bitmap, votes, p->bins_w, p->bins_h, L.words, p->max_instances, F, H, W, pal_w, pal_h, peak_cell, peak_votes,
-      peak_emb, out_centroids, out_count, counters, status);
-  CPE_CUDA(cudaGetLastError());
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_COMPACT], st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_ASSIGN], st));
-  rc = p->dtype == CPE_F32
-           ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters, status)
-           : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second, counters, status);
+  uint32_t* votes_to_zero = keep_votes ? nullptr : votes;
+  rc = p->dtype == CPE_F32 ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second,
+                                                  counters, status, votes_to_zero, L.cells)
+                           : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best,
+                                                   second, counters, status, votes_to_zero, L.cells);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "assign"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
@@ -318,7 +335,11 @@ int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int 
   const size_t Kmax = (size_t)params->max_instances, HW = (size_t)H * W;
   size_t off = 0, sz = 0;
   switch (which) {
-    case CPE_INT_VOTES: off = L.votes; sz = 4 * (size_t)L.cells * B; break;
+    case CPE_INT_VOTES:
+      if (!(params->flags & CPE_FLAG_KEEP_VOTES)) return CPE_ERR_WHICH;
+      off = L.votes;
+      sz = 4 * (size_t)L.cells * B;
+      break;
     case CPE_INT_PEAK_CELLS: off = L.peak_cell; sz = 4 * Kmax * B; break;
     case CPE_INT_PEAK_VOTES: off = L.peak_votes; sz = 4 * Kmax * B; break;
     case CPE_INT_PEAK_EMB: off = L.peak_emb; sz = 4 * Kmax * 4 * F * B; break;
@@ -330,7 +351,7 @@ int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int 
       off = which == CPE_INT_BEST_SCORE ? L.best : L.second;
       sz = 4 * HW * B;
       break;
-    case CPE_INT_STATUS: off = L.status; sz = 4; break;
+    case CPE_INT_STATUS: off = L.status; sz = 4 * (size_t)B; break;
     case CPE_INT_COUNTERS: off = L.counters; sz = 4 * (size_t)CPE_CNT_N * B; break;
     default: return CPE_ERR_WHICH;
   }

@@ -96,7 +96,7 @@ template <typename T, int FT>
 __global__ void __launch_bounds__(kVoteThreads)
 decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
                    int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
-                   uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
+                   uint32_t* __restrict__ acc) {
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
   const int b = blockIdx.y;
@@ -203,11 +203,8 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
     const uint32_t k = s_keys[i];
     if (k != kHashEmpty) atomicAdd(&votes_img[k], s_cnts[i]);
   }
-  if (tid == 0 && s_voting) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_VOTING], s_voting);
-  if (tid == 0 && s_nonfinite) {
-    atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_NONFINITE], s_nonfinite);
-    atomicOr(status, (uint32_t)CPE_STATUS_NONFINITE);
-  }
+  if (tid == 0 && s_voting) atomicAdd(&acc[b * kAccStride + kAccVoting], s_voting);
+  if (tid == 0 && s_nonfinite) atomicAdd(&acc[b * kAccStride + kAccNonfinite], s_nonfinite);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -225,8 +222,7 @@ constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight 
 template <typename T, int FT>
 __global__ void __launch_bounds__(kVoteThreads, 3)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
-                       int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ counters,
-                       uint32_t* __restrict__ status) {
+                       int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int F = FT;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
@@ -388,11 +384,8 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
     const uint32_t k = s_keys[i];
     if (k != kHashEmpty) atomicAdd(&votes_img[k], s_cnts[i]);
   }
-  if (tid == 0 && s_voting) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_VOTING], s_voting);
-  if (tid == 0 && s_nonfinite) {
-    atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_NONFINITE], s_nonfinite);
-    atomicOr(status, (uint32_t)CPE_STATUS_NONFINITE);
-  }
+  if (tid == 0 && s_voting) atomicAdd(&acc[b * kAccStride + kAccVoting], s_voting);
+  if (tid == 0 && s_nonfinite) atomicAdd(&acc[b * kAccStride + kAccNonfinite], s_nonfinite);
 }
 
 }  // namespace cpe

@@ -1,78 +1,86 @@
 // Stage 3: local-maximum test over the vote map (Sec. 3.2, "Local Maxima Search") and ordered
-// compaction of the peaks into a device-side list, with centroids and peak embeddings.
+// compaction of the peaks into a device-side list, with centroids and peak embeddings - one kernel.
 #pragma once
 
 #include "cpe_common.cuh"
 
 namespace cpe {
 
-constexpr int kPeakThreads = 256;
-constexpr int kCompactThreads = 1024;
+constexpr int kPeakThreads = 1024;   // wide CTAs: the last one of an image does the whole compaction
 
-// One thread per bin, one warp per 32 consecutive bins: the warp's ballot is one word of the peak
-// indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it beats
-// each existing 8-neighbour: larger count, or equal count and lower linear index.
+// Phase 1 (every CTA): one thread per bin, one warp per 32 consecutive bins; the warp's ballot is one word
+// of the peak indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it
+// beats each existing 8-neighbour: larger count, or equal count and lower linear index.
+//
+// Phase 2 (the last CTA of each image to finish phase 1; found with a ticket counter, no waiting): ordered
+// compaction without atomics or sorting.  Every thread counts the set bits of its contiguous slice of the
+// bitmap, an exclusive block scan gives each slice its first output slot, and the slices are written out in
+// order, so the list is ascending in the linear bin index and, when there are more than K_max peaks, exactly
+// the first K_max are kept.  Then the centroids (bin positions of Eq. 9 in pixel units) and the peak
+// embeddings concat(P_w[cx], P_h[cy]) are gathered, and the image's counters and status word are written.
 __global__ void __launch_bounds__(kPeakThreads)
-peaks_bitmap_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
-                    uint32_t* __restrict__ bitmap) {
+peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
+             uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
+             const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
+             float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
+             uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
   const int b = blockIdx.y;
-  const int warp = (blockIdx.x * kPeakThreads + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (warp >= words) return;  // whole warps leave together
-  const int cells = bins_w * bins_h;
-  const uint32_t* V = votes + (size_t)b * cells;
-  const int lin = warp * 32 + lane;
-  bool peak = false;
-  if (lin < cells) {
-    const uint32_t v = __ldg(V + lin);
-    if (v > T_v) {
-      const int cy = lin / bins_w, cx = lin - cy * bins_w;
-      peak = true;
-#pragma unroll
-      for (int dy = -1; dy <= 1; ++dy) {
-#pragma unroll
-        for (int dx = -1; dx <= 1; ++dx) {
-          if (dx == 0 && dy == 0) continue;
-          const int ny = cy + dy, nx = cx + dx;
-          if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
-          const int nlin = ny * bins_w + nx;
-          const uint32_t nv = __ldg(V + nlin);
-          if (nv > v || (nv == v && nlin < lin)) peak = false;
-        }
-      }
-    }
-  }
-  const uint32_t word = __ballot_sync(0xffffffffu, peak);
-  if (lane == 0) bitmap[(size_t)b * words + warp] = word;
-}
-
-// One CTA per image.  Ordered compaction without atomics or sorting: every thread counts the set bits
-// of its contiguous slice of the bitmap, an exclusive block scan gives each slice its first output slot,
-// and the slices are written out in order, so the list is ascending in the linear bin index and, when
-// there are more than K_max peaks, exactly the first K_max are kept.  Then the centroids (bin positions
-// of Eq. 9 in pixel units) and the peak embeddings concat(P_w[cx], P_h[cy]) are gathered.
-__global__ void __launch_bounds__(kCompactThreads)
-peaks_compact_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ votes, int bins_w, int bins_h,
-                     int words, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
-                     const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell,
-                     uint32_t* __restrict__ peak_votes, float* __restrict__ peak_emb,
-                     float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
-                     uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
-  const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int cells = bins_w * bins_h;
-  const uint32_t* bm = bitmap + (size_t)b * words;
   const uint32_t* V = votes + (size_t)b * cells;
+  uint32_t* bm = bitmap + (size_t)b * words;
+
+  // ---- phase 1
+  {
+    const int warp = (blockIdx.x * kPeakThreads + tid) >> 5;
+    if (warp < words) {  // whole warps take this branch together
+      const int lin = warp * 32 + lane;
+      bool peak = false;
+      if (lin < cells) {
+        const uint32_t v = __ldg(V + lin);
+        if (v > T_v) {
+          const int cy = lin / bins_w, cx = lin - cy * bins_w;
+          peak = true;
+#pragma unroll
+          for (int dy = -1; dy <= 1; ++dy) {
+#pragma unroll
+            for (int dx = -1; dx <= 1; ++dx) {
+              if (dx == 0 && dy == 0) continue;
+              const int ny = cy + dy, nx = cx + dx;
+              if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+              const int nlin = ny * bins_w + nx;
+              const uint32_t nv = __ldg(V + nlin);
+              if (nv > v || (nv == v && nlin < lin)) peak = false;
+            }
+          }
+        }
+      }
+      const uint32_t word = __ballot_sync(0xffffffffu, peak);
+      if (lane == 0) bm[warp] = word;
+    }
+  }
+
+  // ---- which CTA of this image is the last one?
+  __shared__ int s_last;
+  __threadfence();          // this CTA's bitmap words are visible device-wide before its ticket is taken
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t ticket = atomicAdd(&acc[b * kAccStride + kAccTicket], 1u);
+    s_last = ticket == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();          // and the other CTAs' words are visible to this one
+
+  // ---- phase 2
   int32_t* pc = peak_cell + (size_t)b * K_max;
   uint32_t* pv = peak_votes + (size_t)b * K_max;
-
-  const int per = (words + kCompactThreads - 1) / kCompactThreads;
+  const int per = (words + kPeakThreads - 1) / kPeakThreads;
   const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
   int local = 0;
-  for (int w = w0; w < w1; ++w) local += __popc(bm[w]);
+  for (int w = w0; w < w1; ++w) local += __popc(__ldcg(bm + w));
 
-  // exclusive scan over the block
-  __shared__ int s_warp[kCompactThreads / 32];
+  __shared__ int s_warp[kPeakThreads / 32];
   __shared__ int s_total;
   int incl = local;
 #pragma unroll
@@ -82,23 +90,22 @@ peaks_compact_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __rest
   }
   if (lane == 31) s_warp[wid] = incl;
   __syncthreads();
-  if (wid == 0) {
-    int v = s_warp[lane];
-    int inc2 = v;
+  if (tid == 0) {
+    int run = 0;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, inc2, d);
-      if (lane >= d) inc2 += t;
+    for (int w = 0; w < kPeakThreads / 32; ++w) {
+      const int t = s_warp[w];
+      s_warp[w] = run;
+      run += t;
     }
-    s_warp[lane] = inc2 - v;  // exclusive prefix of the warp totals
-    if (lane == 31) s_total = inc2;
+    s_total = run;
   }
   __syncthreads();
   int slot = s_warp[wid] + incl - local;
   const int total = s_total;
 
   for (int w = w0; w < w1 && slot < K_max; ++w) {
-    uint32_t bits = bm[w];
+    uint32_t bits = __ldcg(bm + w);
     while (bits && slot < K_max) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
@@ -111,21 +118,34 @@ peaks_compact_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __rest
   const int count = min(total, K_max);
   if (tid == 0) {
     out_count[b] = count;
-    counters[b * CPE_CNT_N + CPE_CNT_RAW_PEAKS] = (uint32_t)total;
-    counters[b * CPE_CNT_N + CPE_CNT_TRUNCATED] = (uint32_t)(total - count);
-    if (total > K_max) atomicOr(status, (uint32_t)CPE_STATUS_PEAK_OVERFLOW);
+    // fold the voting kernel's accumulators into this image's counters, and leave them zero for the next decode
+    const uint32_t voting = acc[b * kAccStride + kAccVoting], nonfinite = acc[b * kAccStride + kAccNonfinite];
+    acc[b * kAccStride + kAccVoting] = 0u;
+    acc[b * kAccStride + kAccNonfinite] = 0u;
+    acc[b * kAccStride + kAccTicket] = 0u;
+    uint32_t* cnt = counters + b * CPE_CNT_N;
+    cnt[CPE_CNT_VOTING] = voting;
+    cnt[CPE_CNT_NONFINITE] = nonfinite;
+    cnt[CPE_CNT_RAW_PEAKS] = (uint32_t)total;
+    cnt[CPE_CNT_TRUNCATED] = (uint32_t)(total - count);
+    cnt[CPE_CNT_TAU_REJECTED] = 0u;     // the assignment kernel adds to these four
+    cnt[CPE_CNT_FILTER_PAIRS] = 0u;
+    cnt[CPE_CNT_RESCORED] = 0u;
+    cnt[CPE_CNT_FULL_SCORED] = 0u;
+    status[b] = (nonfinite ? (uint32_t)CPE_STATUS_NONFINITE : 0u) |
+                (total > K_max ? (uint32_t)CPE_STATUS_PEAK_OVERFLOW : 0u);
   }
   __syncthreads();  // the list written above is read below by other threads of this CTA
 
   const int D = 4 * F;
   float* pe = peak_emb + (size_t)b * K_max * D;
-  for (int i = tid; i < count * D; i += kCompactThreads) {
+  for (int i = tid; i < count * D; i += kPeakThreads) {
     const int k = i / D, c = i - k * D;
     const int lin = pc[k];
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     pe[i] = (c < 2 * F) ? pal_w[cx * 2 * F + c] : pal_h[cy * 2 * F + (c - 2 * F)];
   }
-  for (int k = tid; k < count; k += kCompactThreads) {
+  for (int k = tid; k < count; k += kPeakThreads) {
     const int lin = pc[k];
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     // bin position -1 + 2i/(n+1), i = c+1 (Eq. 9); pixel centres sit at x = -1 + (2 col + 1)/W

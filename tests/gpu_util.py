@@ -9,13 +9,13 @@ REL = 1e-4         # relative tolerance of float scores and centroids
 
 
 def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, scores=True, mode="direct",
-            exact_assign=False):
+            exact_assign=False, keep_votes=True, filter_assign=False):
     import torch
     B, D, H, W = emb.shape
     F = D // 4
     dtype = "f32" if emb.dtype == np.float32 else "f16"
     dec = cb.Decoder(B, H, W, F, dtype, bins_w, bins_h, T_v, float(tau), K_max, levels, write_scores=scores,
-                     exact_assign=exact_assign)
+                     exact_assign=exact_assign, keep_votes=keep_votes, filter_assign=filter_assign)
     d_emb = torch.from_numpy(emb).cuda()
     d_fg = None if fg is None else torch.from_numpy(np.ascontiguousarray(fg, np.uint8)).cuda()
     if mode == "direct":
@@ -33,13 +33,13 @@ def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, sc
         "labels": dec.labels.cpu().numpy(),
         "centroids": dec.centroids.cpu().numpy(),
         "count": dec.count.cpu().numpy(),
-        "votes": dec.intermediate(cb.CPE_INT_VOTES).cpu().numpy().view(np.uint32),
+        "votes": dec.intermediate(cb.CPE_INT_VOTES).cpu().numpy().view(np.uint32) if keep_votes else None,
         "peak_cell": dec.intermediate(cb.CPE_INT_PEAK_CELLS).cpu().numpy(),
         "peak_votes": dec.intermediate(cb.CPE_INT_PEAK_VOTES).cpu().numpy().view(np.uint32),
         "peak_emb": dec.intermediate(cb.CPE_INT_PEAK_EMB).cpu().numpy(),
         "pal_w": dec.intermediate(cb.CPE_INT_PALETTE_W).cpu().numpy(),
         "pal_h": dec.intermediate(cb.CPE_INT_PALETTE_H).cpu().numpy(),
-        "status": int(dec.intermediate(cb.CPE_INT_STATUS).cpu().numpy()[0]),
+        "status": int(np.bitwise_or.reduce(dec.intermediate(cb.CPE_INT_STATUS).cpu().numpy())),
         "counters": dec.intermediate(cb.CPE_INT_COUNTERS).cpu().numpy().astype(np.int64),
     }
     if scores:
@@ -54,7 +54,8 @@ def compare_front(gpu, ora, F, bins_w, bins_h):
     assert np.array_equal(gpu["pal_w"].view(np.uint32), oracle.palette(bins_w, F).view(np.uint32))
     assert np.array_equal(gpu["pal_h"].view(np.uint32), oracle.palette(bins_h, F).view(np.uint32))
     assert not (gpu["status"] & cb.CPE_STATUS_INTERNAL), hex(gpu["status"])      # no index self-check fired
-    assert np.array_equal(gpu["votes"], ora["votes"]), "vote map differs"
+    if gpu["votes"] is not None:
+        assert np.array_equal(gpu["votes"], ora["votes"]), "vote map differs"
     assert np.array_equal(gpu["count"], ora["count"]), (gpu["count"], ora["count"])
     Pw, Ph = oracle.palette(bins_w, F), oracle.palette(bins_h, F)
     for b in range(len(ora["count"])):
@@ -96,8 +97,17 @@ def check_case(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0,
     if rep["excused_mismatches"] == 0:
         assert np.array_equal(gpu["counters"][:, cb.CPE_CNT_TAU_REJECTED], ora["counters"][:, oracle.CNT_TAU_REJECTED])
     # the production configuration: no score output (the filter may then decide a pixel without re-scoring it)
-    fast = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, levels, False, mode)
+    fast = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, levels, False, mode, keep_votes=False)
     compare_front(fast, ora, F, bins_w, bins_h)
     rep2 = compare_labels(fast["labels"], None, None, ora["labels"], ora["best"], ora["second"])
     rep["excused_mismatches_no_scores"] = rep2["excused_mismatches"]
+    # the tensor-core filtered kernel forced on, with and without scores (images with few peaks would
+    # otherwise take the all-pairs kernel)
+    for sc in (True, False):
+        filt = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, levels, sc, mode, keep_votes=False, filter_assign=True)
+        compare_front(filt, ora, F, bins_w, bins_h)
+        compare_labels(filt["labels"], filt.get("best"), filt.get("second"), ora["labels"], ora["best"], ora["second"])
+        if sc:   # both kernels compute the same binary32 scores
+            assert np.array_equal(filt["best"].view(np.uint32), gpu["best"].view(np.uint32))
+            assert np.array_equal(filt["second"].view(np.uint32), gpu["second"].view(np.uint32))
     return gpu, ora, rep

@@ -70,7 +70,7 @@ def test_argument_errors_are_reported_before_any_launch():
 
 
 def test_intermediate_addresses_are_inside_the_workspace_and_disjoint():
-    p = cb.make_params(cb.CPE_F32, 64, 48, flags=cb.CPE_FLAG_WRITE_SCORES, max_instances=100)
+    p = cb.make_params(cb.CPE_F32, 64, 48, flags=cb.CPE_FLAG_WRITE_SCORES | cb.CPE_FLAG_KEEP_VOTES, max_instances=100)
     base = 1 << 20
     p.workspace = base
     p.workspace_bytes = cb.cpe_workspace_size(2, 30, 50, 8, p)
@@ -88,6 +88,7 @@ def test_intermediate_addresses_are_inside_the_workspace_and_disjoint():
     assert cb.cpe_get_intermediate(p, 99, 2, 30, 50, 8)[0] == cb.CPE_ERR_WHICH
     p.flags = 0
     assert cb.cpe_get_intermediate(p, cb.CPE_INT_BEST_SCORE, 2, 30, 50, 8)[0] == cb.CPE_ERR_WHICH
+    assert cb.cpe_get_intermediate(p, cb.CPE_INT_VOTES, 2, 30, 50, 8)[0] == cb.CPE_ERR_WHICH
 
 
 def test_strerror_covers_every_code():
