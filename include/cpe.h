@@ -49,7 +49,8 @@ enum {
   CPE_ERR_PARAM = -6,      /* struct_size mismatch, negative threshold, max_instances < 1  */
   CPE_ERR_CUDA = -7,       /* a CUDA runtime call failed (see cpe_last_cuda_error)         */
   CPE_ERR_WHICH = -8,      /* unknown intermediate id, or it was not requested by flags    */
-  CPE_ERR_NOMEM = -9       /* host or device allocation failed (context helpers only)      */
+  CPE_ERR_NOMEM = -9,      /* host or device allocation failed (context helpers only)      */
+  CPE_ERR_STATIC_LIMIT = -10 /* the problem needs more scratch than cpe_decode_static has       */
 };
 
 /* cpe_params.flags */
@@ -218,6 +219,37 @@ int cpe_host_decode(cpe_host_ctx* ctx, const void* emb_host, const uint8_t* fg_m
 /* Bytes moved per cpe_host_decode call in each direction. */
 int cpe_host_ctx_traffic(const cpe_host_ctx* ctx, size_t* h2d_bytes, size_t* d2h_bytes);
 void cpe_host_ctx_destroy(cpe_host_ctx* ctx);
+
+/* ------------------------------------------------------------------ decode without any allocation --- */
+
+/*
+ * (No counterpart in the paper: an integration variant of cpe_decode.)
+ *
+ * For callers that cannot give the library a workspace because they must not allocate device memory at
+ * all: plug-ins that run inside another engine's enqueue call, code on a real-time path, processes whose
+ * memory pool is fixed at start-up.  cpe_decode_static is cpe_decode with the workspace replaced by a
+ * scratch array that is part of the library image itself (a file-scope __device__ array of
+ * CPE_STATIC_SCRATCH_BYTES bytes; every GPU that loads the library holds it until the process exits).
+ * The caller still passes the inputs and the three outputs; params->workspace and workspace_bytes are
+ * ignored, CPE_FLAG_WRITE_SCORES is not available, and cpe_get_intermediate does not apply.
+ *
+ * It calls no cudaMalloc, cudaFree or any other allocating routine, on the host or on the device.
+ *
+ * Limits and rules
+ *   - The scratch needed (what cpe_workspace_size reports for the same arguments) must not exceed
+ *     CPE_STATIC_SCRATCH_BYTES, and bins_w, bins_h must not exceed CPE_STATIC_MAX_BINS; otherwise the
+ *     call returns CPE_ERR_STATIC_LIMIT and enqueues nothing.
+ *   - The first call on a device, and any call whose sizes or parameters (B, F, bins, max_instances) differ
+ *     from the previous call on that device, also sets the scratch up: it looks up the array's device address, uploads the palettes
+ *     and waits for the stream.  Make such a call before starting a stream capture, not inside one.
+ *   - All calls on a device share the one array, which keeps what the last call left in it; every call
+ *     clears the parts that must start at zero.  Two calls that overlap on the GPU (different streams)
+ *     would race on it: keep them on one stream, or order them yourself.
+ */
+#define CPE_STATIC_SCRATCH_BYTES (8u << 20)
+#define CPE_STATIC_MAX_BINS 1024
+int cpe_decode_static(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                      const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,9 @@ from . import build as _build
 CPE_F32, CPE_F16 = 0, 1
 CPE_OK = 0
 CPE_ERR_NULL, CPE_ERR_SIZE, CPE_ERR_DTYPE, CPE_ERR_ALIGN, CPE_ERR_WORKSPACE = -1, -2, -3, -4, -5
-CPE_ERR_PARAM, CPE_ERR_CUDA, CPE_ERR_WHICH, CPE_ERR_NOMEM = -6, -7, -8, -9
+CPE_ERR_PARAM, CPE_ERR_CUDA, CPE_ERR_WHICH, CPE_ERR_NOMEM, CPE_ERR_STATIC_LIMIT = -6, -7, -8, -9, -10
+CPE_STATIC_SCRATCH_BYTES = 8 << 20
+CPE_STATIC_MAX_BINS = 1024
 CPE_FLAG_WRITE_SCORES = 1
 CPE_FLAG_EXACT_ASSIGN = 2
 CPE_FLAG_KEEP_VOTES = 4
@@ -36,6 +38,7 @@ EXPORTS = (
     "cpe_workspace_size", "cpe_init_workspace", "cpe_decode", "cpe_get_intermediate", "cpe_strerror",
     "cpe_last_cuda_error", "cpe_graph_create", "cpe_graph_launch", "cpe_graph_destroy", "cpe_graph_kernel_nodes",
     "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
+    "cpe_decode_static",
 )
 
 
@@ -116,6 +119,8 @@ def load() -> ctypes.CDLL:
     lib.cpe_host_ctx_traffic.restype = ci
     lib.cpe_host_ctx_destroy.argtypes = [vp]
     lib.cpe_host_ctx_destroy.restype = None
+    lib.cpe_decode_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, pp, vp, vp, vp]
+    lib.cpe_decode_static.restype = ci
     _lib = lib
     return lib
 
@@ -147,6 +152,12 @@ def cpe_init_workspace(stream, B, H, W, F, params: cpe_params) -> int:
 def cpe_decode(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_labels, out_centroids, out_count) -> int:
     return int(load().cpe_decode(stream, emb, fg_mask or None, B, H, W, F, ctypes.byref(params), out_labels,
                                  out_centroids, out_count))
+
+
+def cpe_decode_static(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_labels, out_centroids, out_count) -> int:
+    """``cpe_decode`` on the library's built-in scratch array: no workspace, no allocation (see ``cpe.h``)."""
+    return int(load().cpe_decode_static(stream, emb, fg_mask or None, B, H, W, F, ctypes.byref(params), out_labels,
+                                        out_centroids, out_count))
 
 
 def cpe_get_intermediate(params: cpe_params, which, B, H, W, F):

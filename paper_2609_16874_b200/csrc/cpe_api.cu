@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -372,6 +373,7 @@ const char* cpe_strerror(int code) {
     case CPE_ERR_CUDA: return "a CUDA runtime call failed";
     case CPE_ERR_WHICH: return "unknown or unavailable intermediate";
     case CPE_ERR_NOMEM: return "allocation failed";
+    case CPE_ERR_STATIC_LIMIT: return "the problem needs more scratch (or more bins) than cpe_decode_static provides";
     default: return "unknown error code";
   }
 }
@@ -543,3 +545,83 @@ int cpe_host_ctx_traffic(const cpe_host_ctx* c, size_t* h2d_bytes, size_t* d2h_b
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------ decode without allocation
+
+// The scratch of cpe_decode_static lives in the library image.  In host code this name is only a handle for
+// cudaGetSymbolAddress: it is not a device address and must never be handed to a kernel as one.
+static __device__ __align__(256) unsigned char g_static_scratch[CPE_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+struct StaticSlot {
+  void* ptr = nullptr;                 // device address of g_static_scratch on this device
+  int F = 0, bins_w = 0, bins_h = 0;   // palettes currently uploaded ...
+  size_t off_w = 0, off_h = 0;         // ... and where (the layout moves with B, bins and max_instances)
+};
+StaticSlot g_static_slot[64];
+// host staging for one palette: static storage, so the set-up allocates nothing either
+float g_static_palette[CPE_STATIC_MAX_BINS * 32];
+std::mutex g_static_mutex;
+
+}  // namespace
+
+extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W,
+                                 int F, const cpe_params* params, int32_t* out_labels, float* out_centroids,
+                                 int32_t* out_count) {
+  int rc = check_shape(B, H, W, F, params);
+  if (rc) return rc;
+  if (!emb || !out_labels || !out_centroids || !out_count) return CPE_ERR_NULL;
+  cpe_params p = *params;
+  if (p.flags & CPE_FLAG_WRITE_SCORES) return CPE_ERR_STATIC_LIMIT;
+  p.flags |= CPE_FLAG_KEEP_VOTES;   // the vote map is cleared at the start of every call instead of at the end
+  p.workspace = nullptr;
+  p.workspace_bytes = 0;
+  const cpe::Layout L = cpe::make_layout(B, H, W, F, &p);
+  if (L.total > (size_t)CPE_STATIC_SCRATCH_BYTES || p.bins_w > CPE_STATIC_MAX_BINS || p.bins_h > CPE_STATIC_MAX_BINS)
+    return CPE_ERR_STATIC_LIMIT;
+
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int dev = 0;
+  CPE_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CPE_ERR_SIZE;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSlot& slot = g_static_slot[dev];
+  if (!slot.ptr) {
+    // once per device, with that device current: the device address behind the symbol
+    void* ptr = nullptr;
+    CPE_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    slot.ptr = ptr;
+  }
+  char* ws = static_cast<char*>(slot.ptr);
+  if (slot.F != F || slot.bins_w != p.bins_w || slot.bins_h != p.bins_h || slot.off_w != L.pal_w ||
+      slot.off_h != L.pal_h) {
+    // Eq. 9 positions through Eq. 2, in double, rounded once to binary32 (as cpe_init_workspace does)
+    const double pi = 3.14159265358979323846;
+    for (int axis = 0; axis < 2; ++axis) {
+      const int n = axis == 0 ? p.bins_w : p.bins_h;
+      for (int i = 1; i <= n; ++i) {
+        const double pos = -1.0 + 2.0 * (double)i / (double)(n + 1);
+        for (int l = 0; l < F; ++l) {
+          const double arg = pi * ldexp(1.0, l) * pos;
+          g_static_palette[(size_t)(i - 1) * 2 * F + 2 * l] = (float)sin(arg);
+          g_static_palette[(size_t)(i - 1) * 2 * F + 2 * l + 1] = (float)cos(arg);
+        }
+      }
+      CPE_CUDA(cudaMemcpyAsync(ws + (axis == 0 ? L.pal_w : L.pal_h), g_static_palette,
+                               sizeof(float) * (size_t)n * 2 * F, cudaMemcpyHostToDevice, st));
+      CPE_CUDA(cudaStreamSynchronize(st));   // the staging buffer is reused for the other axis
+    }
+    slot.F = F;
+    slot.bins_w = p.bins_w;
+    slot.bins_h = p.bins_h;
+    slot.off_w = L.pal_w;
+    slot.off_h = L.pal_h;
+  }
+  // what must start at zero: the voting accumulators and the peak kernel's ticket (the vote map is cleared by
+  // the decode itself because of CPE_FLAG_KEEP_VOTES); an earlier call with other sizes may have left anything
+  CPE_CUDA(cudaMemsetAsync(ws + L.acc, 0, L.votes - L.acc, st));
+  p.workspace = slot.ptr;
+  p.workspace_bytes = CPE_STATIC_SCRATCH_BYTES;
+  return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
+}
