@@ -14,24 +14,33 @@ namespace cpe {
 constexpr int kAssignThreads = 256;
 constexpr int kPeakChunk = 32;  // peaks staged in shared memory per pass
 
+// `bound`: the caller only needs to know d if d < bound.  sqrt(sx) alone already bounds d from below, so when
+// sqrt(sx) >= bound the y half is skipped and +inf is returned (the peak cannot beat `bound`; on equality it
+// would lose the tie to the earlier peak anyway).  Whenever a finite value is returned it is the full score.
 template <int D>
-__device__ __forceinline__ float score_direct(const float (&e)[D], const float* __restrict__ pk) {
+__device__ __forceinline__ float score_direct(const float (&e)[D], const float* __restrict__ pk, float bound) {
   float sx = 0.0f, sy = 0.0f;
 #pragma unroll
   for (int c = 0; c < D / 2; c += 4) {
     const float4 a = *reinterpret_cast<const float4*>(pk + c);
-    const float4 g = *reinterpret_cast<const float4*>(pk + D / 2 + c);
     float t;
     t = __fsub_rn(e[c + 0], a.x); sx = __fmaf_rn(t, t, sx);
     t = __fsub_rn(e[c + 1], a.y); sx = __fmaf_rn(t, t, sx);
     t = __fsub_rn(e[c + 2], a.z); sx = __fmaf_rn(t, t, sx);
     t = __fsub_rn(e[c + 3], a.w); sx = __fmaf_rn(t, t, sx);
+  }
+  const float dx = __fsqrt_rn(sx);
+  if (!(dx < bound)) return __int_as_float(0x7f800000);
+#pragma unroll
+  for (int c = 0; c < D / 2; c += 4) {
+    const float4 g = *reinterpret_cast<const float4*>(pk + D / 2 + c);
+    float t;
     t = __fsub_rn(e[D / 2 + c + 0], g.x); sy = __fmaf_rn(t, t, sy);
     t = __fsub_rn(e[D / 2 + c + 1], g.y); sy = __fmaf_rn(t, t, sy);
     t = __fsub_rn(e[D / 2 + c + 2], g.z); sy = __fmaf_rn(t, t, sy);
     t = __fsub_rn(e[D / 2 + c + 3], g.w); sy = __fmaf_rn(t, t, sy);
   }
-  return __fadd_rn(__fsqrt_rn(sx), __fsqrt_rn(sy));
+  return __fadd_rn(dx, __fsqrt_rn(sy));
 }
 
 // Generic-F version of the same arithmetic (any F in [1,16]); e lives in local memory.
@@ -103,7 +112,8 @@ assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW,
     if (act) {
       for (int kk = 0; kk < kn; ++kk) {
         float d;
-        if constexpr (FT > 0) d = score_direct<DT>(e, s_pk + kk * DT);
+        // only distances below the current runner-up (or best, when no scores are stored) matter
+        if constexpr (FT > 0) d = score_direct<DT>(e, s_pk + kk * DT, best ? d2 : d1);
         else d = score_direct_rt(e, s_pk + kk * D, F);
         if (d < d1) { d2 = d1; d1 = d; k1 = k0 + kk; }
         else if (d < d2) { d2 = d; }

@@ -33,18 +33,20 @@ constexpr int kAmTilePitch = kAmMT + 8;     // halves; +8 keeps ldmatrix rows on
 constexpr int kAmQueue = 128;               // queued (pixel, peak) pairs per warp and tile
 
 struct AmSmem {
-  int list, lab, tile, peaks, cs, cxlo, d2x, d2y, flag, best, second, u1, u2, nc, ck, queue, scan, total;
+  int list, lab, tile, tile2, peaks, rowoff, glist, gbits, d2x, d2y, flag, best, second, u1, u2, nc, ck, queue, scan, total;
 };
 
-__host__ __device__ inline AmSmem am_smem_layout(int KA, int peak_cap, int span) {
+__host__ __device__ inline AmSmem am_smem_layout(int KA, int peak_cap, int span, int two_tiles) {
   AmSmem s;
   int off = 0;
   s.list = off;   off += span * 2;
   s.lab = off;    off += span * 4;
   s.tile = off;   off += 2 * KA * kAmTilePitch * 2;
+  s.tile2 = off;  off += two_tiles ? 2 * KA * kAmTilePitch * 2 : 0;
   s.peaks = off;  off += peak_cap * (2 * KA + 8) * 2;
-  s.cs = off;     off += kAmMT * 4;
-  s.cxlo = off;   off += kAmMT * 4;
+  s.rowoff = off; off += kAmMT * 2;
+  s.glist = off;  off += 256 * 2;
+  s.gbits = off;  off += 256;
   s.d2x = off;    off += kAmMT * 4;
   s.d2y = off;    off += kAmMT * 4;
   s.flag = off;   off += kAmMT * 4;
@@ -56,7 +58,7 @@ __host__ __device__ inline AmSmem am_smem_layout(int KA, int peak_cap, int span)
   s.u1 = off;     off += kAmMT * 8;
   s.u2 = off;     off += kAmMT * 8;
   s.queue = off;  off += (kAmThreads / 32) * kAmQueue * 16;
-  s.scan = off;   off += 64;
+  s.scan = off;   off += 128;   // block-scan scratch (16 ints) and the warps' queue counters (8 ints)
   s.total = off;
   return s;
 }
@@ -108,19 +110,22 @@ template <typename T, int KA, bool WANT2>
 __global__ void __launch_bounds__(kAmThreads, 2)
 assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
                   const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
-                  int peak_cap, int span, int vec_mask, int32_t* __restrict__ labels, float* __restrict__ best,
+                  int peak_cap, int span, int vec_mask, int vec_gather, int32_t* __restrict__ labels, float* __restrict__ best,
                   float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
                   uint32_t* __restrict__ votes, int cells, int k_min) {
   constexpr int PKP = 2 * KA + 8;     // peak row pitch in halves
   constexpr int KS = KA / 16;         // k-steps per axis
   extern __shared__ __align__(16) unsigned char smem[];
-  const AmSmem L = am_smem_layout(KA, peak_cap, span);
+  const int two_tiles = (vec_gather && sizeof(T) == 2 && KA == 16) ? 1 : 0;   // prefetch the next tile while this one is swept
+  const AmSmem L = am_smem_layout(KA, peak_cap, span, two_tiles);
   uint16_t* s_list = reinterpret_cast<uint16_t*>(smem + L.list);
   int32_t* s_lab = reinterpret_cast<int32_t*>(smem + L.lab);
-  __half* s_tile = reinterpret_cast<__half*>(smem + L.tile);
+  __half* s_tile0 = reinterpret_cast<__half*>(smem + L.tile);
+  __half* s_tile = s_tile0;                                            // the tile being swept
   __half* s_pk = reinterpret_cast<__half*>(smem + L.peaks);
-  float* s_cs = reinterpret_cast<float*>(smem + L.cs);
-  float* s_cxlo = reinterpret_cast<float*>(smem + L.cxlo);
+  uint16_t* s_rowoff = reinterpret_cast<uint16_t*>(smem + L.rowoff);   // row -> pixel offset in the span, 0xffff: no pixel
+  uint16_t* s_glist = reinterpret_cast<uint16_t*>(smem + L.glist);     // participating 8-pixel groups of the span
+  uint8_t* s_gbits = reinterpret_cast<uint8_t*>(smem + L.gbits);       // which of a group's 8 pixels participate
   float* s_d2x = reinterpret_cast<float*>(smem + L.d2x);
   float* s_d2y = reinterpret_cast<float*>(smem + L.d2y);
   uint32_t* s_flag = reinterpret_cast<uint32_t*>(smem + L.flag);
@@ -156,7 +161,8 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
   const int ppt = span / kAmThreads;   // pixels per thread in the mask pass: 8 or 2
 
   // zero the tile once: padding rows (channels beyond 2F of each axis) must stay zero
-  for (int i = tid; i < 2 * KA * kAmTilePitch / 2; i += kAmThreads) reinterpret_cast<uint32_t*>(s_tile)[i] = 0u;
+  for (int i = tid; i < (1 + two_tiles) * 2 * KA * kAmTilePitch / 2; i += kAmThreads)
+    reinterpret_cast<uint32_t*>(s_tile0)[i] = 0u;
 
   // peak operand: row k = [-2 ex (2F), 0.., -2 ey (2F), 0..] in binary16 (the factor -2 is exact)
   auto load_peaks = [&](int pc) {
@@ -231,44 +237,119 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
       }
       __syncthreads();
       int slot = s_scan[wid] + incl - mine;
-      while (bits) {
-        const int j = __ffs(bits) - 1;
-        bits &= bits - 1;
+      uint32_t rest = bits;
+      while (rest) {
+        const int j = __ffs(rest) - 1;
+        rest &= rest - 1;
         s_list[slot++] = (uint16_t)(tid * ppt + j);
       }
+      const int n_act = s_scan[kAmThreads / 32];
       __syncthreads();
+      if (vec_gather) {
+        // second compaction, of whole 8-pixel groups (thread t owns group t of the span)
+        const uint32_t gm = __ballot_sync(0xffffffffu, bits != 0);
+        if (lane == 0) s_scan[wid] = __popc(gm);
+        __syncthreads();
+        if (tid == 0) {
+          int run = 0;
+#pragma unroll
+          for (int w = 0; w < kAmThreads / 32; ++w) {
+            const int v = s_scan[w];
+            s_scan[w] = run;
+            run += v;
+          }
+          s_scan[kAmThreads / 32 + 1] = run;
+        }
+        __syncthreads();
+        if (bits) {
+          const int gi = s_scan[wid] + __popc(gm & ((1u << lane) - 1u));
+          s_glist[gi] = (uint16_t)tid;
+          s_gbits[gi] = (uint8_t)bits;
+        }
+        if (tid == 0) s_scan[kAmThreads / 32] = n_act;
+        __syncthreads();
+      }
     }
     const int n_active = s_scan[kAmThreads / 32];
+    const int n_groups = vec_gather ? s_scan[kAmThreads / 32 + 1] : 0;
+    const int n_chunks = K > 0 ? (vec_gather ? (n_groups + 31) / 32 : (n_active + kAmMT - 1) / kAmMT) : 0;
 
-    for (int chunk0 = 0; chunk0 < n_active && K > 0; chunk0 += kAmMT) {
-      const int nrows = min(kAmMT, n_active - chunk0);
+    // Asynchronous 16-byte copies of one tile (32 groups x 4F channels) straight into shared memory.
+    auto issue_gather = [&](int ci, __half* dst_tile) {
+      if constexpr (sizeof(T) == 2) {
+        const int ng = min(32, n_groups - ci * 32);
+        for (int i = tid; i < ng * D; i += kAmThreads) {
+          const int gl = i % ng, c = i / ng;               // consecutive lanes -> consecutive groups of one channel
+          const int grp = s_glist[ci * 32 + gl];
+          const int axis = c >= 2 * F ? 1 : 0;
+          const __half* dst = dst_tile + (size_t)(axis * KA + (c - axis * 2 * F)) * kAmTilePitch + gl * 8;
+          const T* src = e_img + (size_t)c * plane + span0 + grp * 8;
+          const uint32_t d32 = (uint32_t)__cvta_generic_to_shared(dst);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d32), "l"(src));
+        }
+      }
+      asm volatile("cp.async.commit_group;\n" ::);
+    };
+    if (vec_gather && sizeof(T) == 2 && n_chunks > 0) issue_gather(0, s_tile0);
+
+    for (int ci = 0; ci < n_chunks; ++ci) {
+      const int chunk0 = ci * kAmMT;
       __syncthreads();   // the previous tile and its row state are no longer read
-      // ---- gather: thread j copies pixel j of the tile, all channels (binary32 inputs are rounded to binary16)
+      // ---- gather
       {
-        if (tid < nrows && am_ok((int)s_list[chunk0 + tid] < span_len, 1u, status)) {
-          const T* src = e_img + span0 + (int)s_list[chunk0 + tid];
-          constexpr int FMAX = KA / 2;       // F <= FMAX for this instantiation
-#pragma unroll
-          for (int axis = 0; axis < 2; ++axis) {
-            const T* sa = src + (size_t)axis * 2 * F * plane;
-            __half* ta = s_tile + (size_t)axis * KA * kAmTilePitch + tid;
-            // every plane load of this axis is issued before the first value is stored
-            __half hv[2 * FMAX];
-#pragma unroll
-            for (int c = 0; c < 2 * FMAX; ++c) {
-              hv[c] = __ushort_as_half((unsigned short)0);
-              if (c < 2 * F) {
-                if constexpr (sizeof(T) == 2)
-                  hv[c] = __ushort_as_half(__ldg(reinterpret_cast<const unsigned short*>(sa + (size_t)c * plane)));
-                else
-                  hv[c] = __float2half_rn(__ldg(reinterpret_cast<const float*>(sa + (size_t)c * plane)));
-              }
+        int off = 0xffff;
+        if (vec_gather) {
+          // rows = the pixels of 32 participating groups; a row whose pixel does not participate stays empty
+          const int gl = tid >> 3, j = tid & 7, gi = ci * 32 + gl;
+          if (gi < n_groups && ((s_gbits[gi] >> j) & 1u)) off = (int)s_glist[gi] * 8 + j;
+          if constexpr (sizeof(T) == 2) {
+            s_tile = two_tiles ? s_tile0 + (size_t)(ci & 1) * 2 * KA * kAmTilePitch : s_tile0;
+            if (!two_tiles && ci > 0) issue_gather(ci, s_tile);
+            asm volatile("cp.async.wait_group 0;\n" ::);
+          } else {
+            // binary32: two 128-bit loads per (group, channel), rounded to binary16 on the way
+            const int ng = min(32, n_groups - ci * 32);
+            for (int i = tid; i < ng * D; i += kAmThreads) {
+              const int gq = i % ng, c = i / ng;
+              const int grp = s_glist[ci * 32 + gq];
+              const int axis = c >= 2 * F ? 1 : 0;
+              __half* dst = s_tile + (size_t)(axis * KA + (c - axis * 2 * F)) * kAmTilePitch + gq * 8;
+              const float4* src = reinterpret_cast<const float4*>(e_img + (size_t)c * plane + span0 + grp * 8);
+              const float4 lo = __ldg(src), hi = __ldg(src + 1);
+              __half2 h[4] = {__floats2half2_rn(lo.x, lo.y), __floats2half2_rn(lo.z, lo.w),
+                              __floats2half2_rn(hi.x, hi.y), __floats2half2_rn(hi.z, hi.w)};
+              *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(h);
             }
+          }
+        } else {
+          // thread j copies pixel j of the tile, all channels (binary32 inputs are rounded to binary16)
+          if (chunk0 + tid < n_active) off = (int)s_list[chunk0 + tid];
+          if (off != 0xffff && am_ok(off < span_len, 1u, status)) {
+            const T* src = e_img + span0 + off;
+            constexpr int FMAX = KA / 2;       // F <= FMAX for this instantiation
 #pragma unroll
-            for (int c = 0; c < 2 * FMAX; ++c)
-              if (c < 2 * F) ta[c * kAmTilePitch] = hv[c];
+            for (int axis = 0; axis < 2; ++axis) {
+              const T* sa = src + (size_t)axis * 2 * F * plane;
+              __half* ta = s_tile + (size_t)axis * KA * kAmTilePitch + tid;
+              // every plane load of this axis is issued before the first value is stored
+              __half hv[2 * FMAX];
+#pragma unroll
+              for (int c = 0; c < 2 * FMAX; ++c) {
+                hv[c] = __ushort_as_half((unsigned short)0);
+                if (c < 2 * F) {
+                  if constexpr (sizeof(T) == 2)
+                    hv[c] = __ushort_as_half(__ldg(reinterpret_cast<const unsigned short*>(sa + (size_t)c * plane)));
+                  else
+                    hv[c] = __float2half_rn(__ldg(reinterpret_cast<const float*>(sa + (size_t)c * plane)));
+                }
+              }
+#pragma unroll
+              for (int c = 0; c < 2 * FMAX; ++c)
+                if (c < 2 * F) ta[c * kAmTilePitch] = hv[c];
+            }
           }
         }
+        s_rowoff[tid] = (uint16_t)off;
         s_nc[tid] = 0;
         s_ck[tid] = -1;
         s_best[tid] = kPackEmpty;
@@ -277,6 +358,9 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
         s_u2[tid] = kPackEmpty;
       }
       __syncthreads();
+      // the other tile buffer was last read before the barrier above: fill it while this tile is swept
+      if (two_tiles && ci + 1 < n_chunks)
+        issue_gather(ci + 1, s_tile0 + (size_t)((ci + 1) & 1) * 2 * KA * kAmTilePitch);
 
       if (dbg_phase == 1) continue;
       // ---- per-warp sweeps: rows m = wid*32 + mt*16 + half*8 + g
@@ -295,7 +379,7 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
           }
       // ||xhat||^2 and ||yhat||^2 of every row from the tensor cores as well: the diagonal of tile x tile^T
       // (the B operand of a row block is that block's own A fragment: {a0, a2} for rows 0-7, {a1, a3} for 8-15)
-      float cs[4], cx[4], thr[4];
+      float cs[4], cx[4], cy[4], thr[4];
       bool live[4];
       {
         float n2[2][4];   // [axis][row r]
@@ -321,7 +405,7 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
           const int m = wid * 32 + (r >> 1) * 16 + (r & 1) * 8 + g;
-          const bool present = m < nrows;
+          const bool present = s_rowoff[m] != 0xffffu;
           const bool finite = (n2[0][r] + n2[1][r]) < inf;
           // binary16 pixels: a non-finite norm is a non-finite pixel.  binary32 pixels: it may also be a value
           // beyond the binary16 range, so the row is scored exactly (and its finiteness checked there).
@@ -337,6 +421,7 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
             delta[axis] = kappa * n1 + 1e-5f * (cfull[axis] + 2.0f * n1 + 2.0f);
           }
           cx[r] = cfull[0] - delta[0];
+          cy[r] = cfull[1] - delta[1];
           cs[r] = (cfull[0] - delta[0]) + (cfull[1] - delta[1]) - 1e-6f * (cfull[0] + cfull[1]);
           if (t4 == 0) {
             s_flag[m] = flag;
@@ -526,23 +611,28 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
           uint32_t bf[2][KS][2];
           load_b(nt, bf);
           const bool ragged = nt * 8 + 8 > kn;
+          // A and B separately (the legacy tensor path is the scarce resource here: two MMAs and an add per
+          // pair are cheaper than a third MMA that would deliver S directly)
           float as[2][4], ax[2][4];
           bool any = false;
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
+            float ay[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              as[mt][i] = cs[mt * 2 + (i >> 1)];
               ax[mt][i] = cx[mt * 2 + (i >> 1)];
+              ay[i] = cy[mt * 2 + (i >> 1)];
             }
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
-              mma_16816(as[mt], af[mt][0][ks], bf[0][ks][0], bf[0][ks][1]);
-              mma_16816(as[mt], af[mt][1][ks], bf[1][ks][0], bf[1][ks][1]);
               mma_16816(ax[mt], af[mt][0][ks], bf[0][ks][0], bf[0][ks][1]);
+              mma_16816(ay, af[mt][1][ks], bf[1][ks][0], bf[1][ks][1]);
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) any = any || (as[mt][i] <= thr[mt * 2 + (i >> 1)]);
+            for (int i = 0; i < 4; ++i) {
+              as[mt][i] = ax[mt][i] + ay[i];
+              any = any || (as[mt][i] <= thr[mt * 2 + (i >> 1)]);
+            }
           }
           if (__any_sync(0xffffffffu, any)) {
             auto pass_mask = [&]() {
@@ -633,8 +723,8 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
           prk[r + 4] = 0; pa[r + 4] = 0.0f; pb[r + 4] = 0.0f;
           if (rk_[r] >= 0) {
             if (((packed >> (8 * r)) & 0xffu) == 1u && !q_over) {
-              const int o = (int)s_list[chunk0 + m];
-              if (am_ok(m < nrows && o < span_len, 3u, status)) s_lab[o] = rk_[r] + 1;
+              const int o = (int)s_rowoff[m];
+              if (am_ok(o < span_len, 3u, status)) s_lab[o] = rk_[r] + 1;
             }
             else pushmask |= 1u << r;
           }
@@ -658,8 +748,8 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
         else return Elem<T>::load1(src + (size_t)(axis * 2 * F + c) * plane);
       };
       auto exact = [&](int m, int k) -> float {
-        if (!am_ok(m >= 0 && m < nrows && k >= 0 && k < K && (int)s_list[chunk0 + m] < span_len, 4u, status)) return inf;
-        const T* src = e_img + span0 + (int)s_list[chunk0 + m];
+        if (!am_ok(m >= 0 && m < kAmMT && k >= 0 && k < K && (int)s_rowoff[m] < span_len, 4u, status)) return inf;
+        const T* src = e_img + span0 + (int)s_rowoff[m];
         const float* pk = pk_img + (size_t)k * D;
         float sx = 0.0f, sy = 0.0f;
         for (int c = 0; c < 2 * F; ++c) {
@@ -710,9 +800,9 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
           const int m = wid * 32 + hl;
           if constexpr (sizeof(T) == 4) {
             // the binary16 copy could not tell an out-of-range value from a non-finite one: look at the originals
-            const T* src = e_img + span0 + (int)s_list[chunk0 + m];
+            const T* src = e_img + span0 + (int)s_rowoff[m];
             float fin = 0.0f;
-            if (am_ok(m < nrows && (int)s_list[chunk0 + m] < span_len, 7u, status))
+            if (am_ok((int)s_rowoff[m] < span_len, 7u, status))
             for (int l = lane; l < 2 * F; l += 32)
               fin = fold_finite(fin, Elem<T>::load1(src + (size_t)(2 * l) * plane),
                                 Elem<T>::load1(src + (size_t)(2 * l + 1) * plane));
@@ -735,9 +825,9 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
         }
       }
       // one lane per row writes the outcome of the rows that went through the queue
-      if (row_l < nrows && am_ok((int)s_list[chunk0 + row_l] < span_len, 6u, status)) {
+      if (s_rowoff[row_l] != 0xffffu && am_ok((int)s_rowoff[row_l] < span_len, 6u, status)) {
         const uint32_t f = s_flag[row_l];
-        const int off = (int)s_list[chunk0 + row_l];
+        const int off = (int)s_rowoff[row_l];
         float d1 = inf, d2 = inf;
         if (f & kRowValid) {
           const unsigned long long bb = s_best[row_l];

@@ -133,12 +133,15 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
                         uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min) {
   // small inputs get short spans so that there are enough CTAs to fill the GPU
   const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
+  // 16-byte gathers of whole 8-pixel groups need aligned planes and the long span
+  const int vec_gather = (span == cpe::kAmSpanMax) && ((uintptr_t)e % 16 == 0) && (HW % 8 == 0);
+  const int two_tiles = (vec_gather && sizeof(T) == 2 && KA == 16) ? 1 : 0;
   // as many peaks resident in shared memory as leave room for two CTAs per SM
   int peak_cap = (p->max_instances + 7) & ~7;
   const int budget = 110 * 1024;
-  const int fixed = cpe::am_smem_layout(KA, 0, span).total;
+  const int fixed = cpe::am_smem_layout(KA, 0, span, two_tiles).total;
   peak_cap = std::max(8, std::min(peak_cap, ((budget - fixed) / ((2 * KA + 8) * 2)) & ~7));
-  const int smem = cpe::am_smem_layout(KA, peak_cap, span).total;
+  const int smem = cpe::am_smem_layout(KA, peak_cap, span, two_tiles).total;
   auto kern = cpe::assign_mma_kernel<T, KA, WANT2>;
   static bool configured = false;   // per instantiation; the attribute is sticky for the process
   if (!configured) {
@@ -152,7 +155,8 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   int need_exact = p->tau < INFINITY ? 1 : 0;
   if (const char* ph = getenv("CPE_DEBUG_PHASE")) need_exact |= (atoi(ph) & 0xf) << 8;   // timing experiments
   kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
-                                            peak_cap, span, vec_mask, labels, best, second, counters, status, votes_to_zero,
+                                            peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status,
+                                            votes_to_zero,
                                             cells, k_min);
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
@@ -242,7 +246,9 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_PEAKS], st));
   {
     const int warps_per_cta = cpe::kPeakThreads / 32;
-    dim3 grid((unsigned)((L.words + warps_per_cta - 1) / warps_per_cta), (unsigned)B);
+    // small maps: one CTA per image does both phases without the cross-CTA hand-over
+    const int ctas = L.words <= 8 * warps_per_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
+    dim3 grid((unsigned)ctas, (unsigned)B);
     cpe::peaks_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
                                                           (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W,
                                                           pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids,

@@ -30,47 +30,48 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   const uint32_t* V = votes + (size_t)b * cells;
   uint32_t* bm = bitmap + (size_t)b * words;
 
-  // ---- phase 1
-  {
-    const int warp = (blockIdx.x * kPeakThreads + tid) >> 5;
-    if (warp < words) {  // whole warps take this branch together
-      const int lin = warp * 32 + lane;
-      bool peak = false;
-      if (lin < cells) {
-        const uint32_t v = __ldg(V + lin);
-        if (v > T_v) {
-          const int cy = lin / bins_w, cx = lin - cy * bins_w;
-          peak = true;
+  // ---- phase 1 (a CTA takes the words blockIdx.x*32 + wid, then strides by the grid: one CTA per image for small maps)
+  for (int warp = blockIdx.x * (kPeakThreads / 32) + wid; warp < words; warp += gridDim.x * (kPeakThreads / 32)) {
+    const int lin = warp * 32 + lane;
+    bool peak = false;
+    if (lin < cells) {
+      const uint32_t v = __ldg(V + lin);
+      if (v > T_v) {
+        const int cy = lin / bins_w, cx = lin - cy * bins_w;
+        peak = true;
 #pragma unroll
-          for (int dy = -1; dy <= 1; ++dy) {
+        for (int dy = -1; dy <= 1; ++dy) {
 #pragma unroll
-            for (int dx = -1; dx <= 1; ++dx) {
-              if (dx == 0 && dy == 0) continue;
-              const int ny = cy + dy, nx = cx + dx;
-              if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
-              const int nlin = ny * bins_w + nx;
-              const uint32_t nv = __ldg(V + nlin);
-              if (nv > v || (nv == v && nlin < lin)) peak = false;
-            }
+          for (int dx = -1; dx <= 1; ++dx) {
+            if (dx == 0 && dy == 0) continue;
+            const int ny = cy + dy, nx = cx + dx;
+            if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+            const int nlin = ny * bins_w + nx;
+            const uint32_t nv = __ldg(V + nlin);
+            if (nv > v || (nv == v && nlin < lin)) peak = false;
           }
         }
       }
-      const uint32_t word = __ballot_sync(0xffffffffu, peak);
-      if (lane == 0) bm[warp] = word;
     }
+    const uint32_t word = __ballot_sync(0xffffffffu, peak);
+    if (lane == 0) bm[warp] = word;
   }
 
-  // ---- which CTA of this image is the last one?
-  __shared__ int s_last;
-  __threadfence();          // this CTA's bitmap words are visible device-wide before its ticket is taken
-  __syncthreads();
-  if (tid == 0) {
-    const uint32_t ticket = atomicAdd(&acc[b * kAccStride + kAccTicket], 1u);
-    s_last = ticket == gridDim.x - 1;
+  // ---- which CTA of this image is the last one?  (with one CTA per image there is nothing to ask)
+  if (gridDim.x > 1) {
+    __shared__ int s_last;
+    __threadfence();          // this CTA's bitmap words are visible device-wide before its ticket is taken
+    __syncthreads();
+    if (tid == 0) {
+      const uint32_t ticket = atomicAdd(&acc[b * kAccStride + kAccTicket], 1u);
+      s_last = ticket == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();          // and the other CTAs' words are visible to this one
+  } else {
+    __syncthreads();
   }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();          // and the other CTAs' words are visible to this one
 
   // ---- phase 2
   int32_t* pc = peak_cell + (size_t)b * K_max;
