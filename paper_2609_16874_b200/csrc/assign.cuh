@@ -30,7 +30,8 @@ __device__ __forceinline__ float score_direct(const float (&e)[D], const float* 
     t = __fsub_rn(e[c + 3], a.w); sx = __fmaf_rn(t, t, sx);
   }
   const float dx = __fsqrt_rn(sx);
-  if (!(dx < bound)) return __int_as_float(0x7f800000);
+  // warp-uniform skip: the y half is only worth its 2F fused multiply-adds if some lane can still use it
+  if (!__any_sync(__activemask(), dx < bound)) return __int_as_float(0x7f800000);
 #pragma unroll
   for (int c = 0; c < D / 2; c += 4) {
     const float4 g = *reinterpret_cast<const float4*>(pk + D / 2 + c);
