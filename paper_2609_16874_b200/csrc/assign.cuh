@@ -11,37 +11,52 @@
 
 namespace cpe {
 
-constexpr int kAssignThreads = 256;
+constexpr int kAssignThreads = 128;
 constexpr int kPeakChunk = 32;  // peaks staged in shared memory per pass
 
-// `bound`: the caller only needs to know d if d < bound.  sqrt(sx) alone already bounds d from below, so when
-// sqrt(sx) >= bound the y half is skipped and +inf is returned (the peak cannot beat `bound`; on equality it
-// would lose the tie to the earlier peak anyway).  Whenever a finite value is returned it is the full score.
+// The x chain and the y chain of one (pixel, peak) pair advance together as the two lanes of packed binary32
+// instructions: e2[c] = (xhat_c, yhat_c), pk2[c] = (P_w[a][c], P_h[b][c]).  Each lane performs exactly the scalar
+// sequence above, so the result has the same bits.
+//
+// `bound2`: the caller only needs d if d < bound, and passes bound^2 (rounded up).  Since sx + sy <= d^2, a pair with
+// sx + sy > bound2 cannot get below the bound: +inf is returned without taking the two IEEE square roots.
 template <int D>
-__device__ __forceinline__ float score_direct(const float (&e)[D], const float* __restrict__ pk, float bound) {
-  float sx = 0.0f, sy = 0.0f;
+__device__ __forceinline__ float score_direct(const float2 (&e2)[D / 2], const float2* __restrict__ pk2, float bound2) {
+  float2 s = make_float2(0.0f, 0.0f);
 #pragma unroll
-  for (int c = 0; c < D / 2; c += 4) {
-    const float4 a = *reinterpret_cast<const float4*>(pk + c);
-    float t;
-    t = __fsub_rn(e[c + 0], a.x); sx = __fmaf_rn(t, t, sx);
-    t = __fsub_rn(e[c + 1], a.y); sx = __fmaf_rn(t, t, sx);
-    t = __fsub_rn(e[c + 2], a.z); sx = __fmaf_rn(t, t, sx);
-    t = __fsub_rn(e[c + 3], a.w); sx = __fmaf_rn(t, t, sx);
+  for (int c = 0; c < D / 2; c += 2) {
+    const float4 q = *reinterpret_cast<const float4*>(pk2 + c);
+    float2 t = sub2_rn(e2[c], make_float2(q.x, q.y));
+    s = fma2_rn(t, t, s);
+    t = sub2_rn(e2[c + 1], make_float2(q.z, q.w));
+    s = fma2_rn(t, t, s);
   }
-  const float dx = __fsqrt_rn(sx);
-  // warp-uniform skip: the y half is only worth its 2F fused multiply-adds if some lane can still use it
-  if (!__any_sync(__activemask(), dx < bound)) return __int_as_float(0x7f800000);
+  if (s.x + s.y > bound2) return __int_as_float(0x7f800000);
+  return __fadd_rn(__fsqrt_rn(s.x), __fsqrt_rn(s.y));
+}
+
+// Four peaks at once: four independent chains keep the FMA pipe busy (one chain alone waits on its own latency).
+// Peaks beyond `kn` must not be passed (the caller pads the shared-memory chunk with copies of a valid peak).
+template <int D>
+__device__ __forceinline__ void score_direct4(const float2 (&e2)[D / 2], const float2* __restrict__ pk2, float bound2,
+                                              float (&d)[4]) {
+  float2 s[4];
 #pragma unroll
-  for (int c = 0; c < D / 2; c += 4) {
-    const float4 g = *reinterpret_cast<const float4*>(pk + D / 2 + c);
-    float t;
-    t = __fsub_rn(e[D / 2 + c + 0], g.x); sy = __fmaf_rn(t, t, sy);
-    t = __fsub_rn(e[D / 2 + c + 1], g.y); sy = __fmaf_rn(t, t, sy);
-    t = __fsub_rn(e[D / 2 + c + 2], g.z); sy = __fmaf_rn(t, t, sy);
-    t = __fsub_rn(e[D / 2 + c + 3], g.w); sy = __fmaf_rn(t, t, sy);
+  for (int j = 0; j < 4; ++j) s[j] = make_float2(0.0f, 0.0f);
+#pragma unroll
+  for (int c = 0; c < D / 2; c += 2) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 q = *reinterpret_cast<const float4*>(pk2 + j * (D / 2) + c);
+      float2 t = sub2_rn(e2[c], make_float2(q.x, q.y));
+      s[j] = fma2_rn(t, t, s[j]);
+      t = sub2_rn(e2[c + 1], make_float2(q.z, q.w));
+      s[j] = fma2_rn(t, t, s[j]);
+    }
   }
-  return __fadd_rn(dx, __fsqrt_rn(sy));
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    d[j] = (s[j].x + s[j].y > bound2) ? __int_as_float(0x7f800000) : __fadd_rn(__fsqrt_rn(s[j].x), __fsqrt_rn(s[j].y));
 }
 
 // Generic-F version of the same arithmetic (any F in [1,16]); e lives in local memory.
@@ -86,15 +101,22 @@ assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW,
 
   bool act = n < HW;
   if (act && fg) act = __ldg(fg + (size_t)b * plane + n) != 0;
-  float e[DT];
+  float e[FT > 0 ? 1 : DT];          // generic path: channel order
+  float2 e2[DT / 2];                 // fixed-F path: (x channel c, y channel c) pairs
   if (act) {
     const T* p = emb + (size_t)b * D * plane + n;
     bool ok = true;
     if constexpr (FT > 0) {
 #pragma unroll
-      for (int c = 0; c < DT; ++c) e[c] = Elem<T>::load1(p + (size_t)c * plane);
+      for (int c = 0; c < DT / 2; ++c) {
+        e2[c].x = Elem<T>::load1(p + (size_t)c * plane);
+        e2[c].y = Elem<T>::load1(p + (size_t)(DT / 2 + c) * plane);
+      }
 #pragma unroll
-      for (int c = 0; c < DT; c += 2) ok = ok && pair_finite(e[c], e[c + 1]);
+      for (int c = 0; c < DT / 2; c += 2) {
+        ok = ok && pair_finite(e2[c].x, e2[c + 1].x);
+        ok = ok && pair_finite(e2[c].y, e2[c + 1].y);
+      }
     } else {
       for (int c = 0; c < D; ++c) e[c] = Elem<T>::load1(p + (size_t)c * plane);
       for (int c = 0; c < D; c += 2) ok = ok && pair_finite(e[c], e[c + 1]);
@@ -104,20 +126,44 @@ assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW,
 
   const float inf = __int_as_float(0x7f800000);
   float d1 = inf, d2 = inf;
+  float bound2 = inf;   // square of the distance a peak has to beat (the runner-up when scores are stored), rounded up
   int k1 = -1;
   for (int k0 = 0; k0 < K; k0 += kPeakChunk) {
     const int kn = min(kPeakChunk, K - k0);
     __syncthreads();
-    for (int i = tid; i < kn * D; i += kAssignThreads) s_pk[i] = pk_img[(size_t)k0 * D + i];
+    if constexpr (FT > 0) {
+      // interleave the peak's two halves: s_pk[kk][2c] = P_w[a][c], s_pk[kk][2c+1] = P_h[b][c]
+      for (int i = tid; i < kn * D; i += kAssignThreads) {
+        const int kk = i / D, j = i - kk * D, c = j >> 1;
+        s_pk[i] = pk_img[(size_t)(k0 + kk) * D + ((j & 1) ? D / 2 + c : c)];
+      }
+    } else {
+      for (int i = tid; i < kn * D; i += kAssignThreads) s_pk[i] = pk_img[(size_t)k0 * D + i];
+    }
     __syncthreads();
     if (act) {
-      for (int kk = 0; kk < kn; ++kk) {
+      int kk = 0;
+      if constexpr (FT > 0) {
+        for (; kk + 4 <= kn; kk += 4) {
+          float d[4];
+          score_direct4<DT>(e2, reinterpret_cast<const float2*>(s_pk + kk * DT), bound2, d);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {     // in ascending k: the lowest k keeps an exact tie
+            if (d[j] < d1) { d2 = d1; d1 = d[j]; k1 = k0 + kk + j; }
+            else if (d[j] < d2) { d2 = d[j]; }
+          }
+          const float bound = best ? d2 : d1;
+          bound2 = bound * bound * (1.0f + 1e-6f);
+        }
+      }
+      for (; kk < kn; ++kk) {
         float d;
-        // only distances below the current runner-up (or best, when no scores are stored) matter
-        if constexpr (FT > 0) d = score_direct<DT>(e, s_pk + kk * DT, best ? d2 : d1);
+        if constexpr (FT > 0) d = score_direct<DT>(e2, reinterpret_cast<const float2*>(s_pk + kk * DT), bound2);
         else d = score_direct_rt(e, s_pk + kk * D, F);
         if (d < d1) { d2 = d1; d1 = d; k1 = k0 + kk; }
         else if (d < d2) { d2 = d; }
+        const float bound = best ? d2 : d1;
+        bound2 = bound * bound * (1.0f + 1e-6f);
       }
     }
   }

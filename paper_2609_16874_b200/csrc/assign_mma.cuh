@@ -181,8 +181,6 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
   __syncthreads();
 
   uint32_t rejected = 0, n_pairs = 0, n_rescored = 0, n_full = 0;
-  const int dbg_phase = (need_exact >> 8) & 0xf;   // timing experiments only: stop a tile after this phase (0 = run all)
-  need_exact &= 0xff;
 
   for (int sp = blockIdx.x; sp < n_spans; sp += gridDim.x) {
     // later spans first: the tail of the voting pass is what is still in L2
@@ -362,7 +360,6 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
       if (two_tiles && ci + 1 < n_chunks)
         issue_gather(ci + 1, s_tile0 + (size_t)((ci + 1) & 1) * 2 * KA * kAmTilePitch);
 
-      if (dbg_phase == 1) continue;
       // ---- per-warp sweeps: rows m = wid*32 + mt*16 + half*8 + g
       // A fragments of both m-tiles and both axes stay in registers for the whole tile
       uint32_t af[2][2][KS][4];
@@ -444,7 +441,6 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
         }
       };
 
-      if (dbg_phase == 2) { if (cs[0] + cx[1] == 12345.0f) s_lab[0] = 1; continue; }
       // sweep 1: the smallest (and, if the runner-up is wanted, second smallest) S_k of every row
       float s1[4], s2[4];
 #pragma unroll
@@ -500,7 +496,6 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
                          : __int_as_float(0x7fc00000);
       }
 
-      if (dbg_phase == 3) { if (thr[0] + thr[3] == 12345.0f) s_lab[0] = 1; continue; }
       // sweep 2: one compare per pair; the few pairs that pass go to the warp's queue
       int q_tail = 0;
       bool q_over = false;
@@ -699,7 +694,6 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
       }
       __syncwarp();
 
-      if (dbg_phase == 4) { if (rk_[0] + rk_[3] + q_tail == 12345) s_lab[0] = 1; continue; }
       // ---- rows with a single surviving pair in the whole quad are decided here; the others go to the queue
       {
         uint32_t packed = extra;

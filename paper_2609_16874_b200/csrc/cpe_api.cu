@@ -152,8 +152,7 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
   dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
   const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
-  int need_exact = p->tau < INFINITY ? 1 : 0;
-  if (const char* ph = getenv("CPE_DEBUG_PHASE")) need_exact |= (atoi(ph) & 0xf) << 8;   // timing experiments
+  const int need_exact = p->tau < INFINITY ? 1 : 0;
   kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
                                             peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status,
                                             votes_to_zero,

@@ -151,6 +151,51 @@ def test_many_peaks_and_fp32_out_of_half_range():
     assert ora["count"][0] == K
 
 
+def test_ragged_batch_scalar_path():
+    # H*W odd (no vector loads anywhere), several images
+    for dtype in ("f16", "f32"):
+        cfg = wl.scaled(wl.CONFIGS["c4"], B=3, H=37, W=53, K=6, bins_w=24, bins_h=20, dtype=dtype, sigma=0.05)
+        fr = wl.make_frame(cfg, 0)
+        check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, T_v=4)
+
+
+def test_degenerate_shapes_and_parameters():
+    rng = np.random.default_rng(3)
+    # one row of pixels, one bin: every participating pixel votes for it and is assigned to it
+    emb = rng.standard_normal((1, 8, 1, 24)).astype(np.float32)
+    fg = np.ones((1, 1, 24), np.uint8)
+    gpu, ora, _ = check_case(emb, fg, 1, 1, T_v=8)
+    assert gpu["count"][0] == 1 and (gpu["labels"] == 1).all()
+    # threshold 0, a single output slot, and K_max equal to the number of peaks
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=64, W=72, K=5, bins_w=24, bins_h=24)
+    fr = wl.make_frame(cfg, 4)
+    gpu, ora, _ = check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, T_v=0)
+    n = int(ora["count"][0])
+    check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, T_v=0, K_max=1)
+    check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, T_v=0, K_max=n)
+    # long thin vote map (1024 x 2 bins)
+    check_case(fr["emb"], fr["fg"], 1024, 2, T_v=2)
+
+
+def test_batch_with_no_few_and_many_peaks_per_image():
+    # one workspace, three images: none / a handful / more than the all-pairs limit of peaks, so that the two
+    # assignment kernels each take some of the images and leave the others alone
+    H, W, F, bw, bh = 96, 128, 4, 64, 48
+    rng = np.random.default_rng(8)
+    emb = np.empty((3, 4 * F, H, W), np.float16)
+    fg = np.zeros((3, H, W), np.uint8)
+    emb[0] = rng.standard_normal((4 * F, H, W)).astype(np.float16)           # image 0: no foreground at all
+    for b, K in ((1, 5), (2, 60)):
+        cells = np.sort(rng.choice(bw // 2 * (bh // 2), K, replace=False))
+        cx, cy = 2 * (cells % (bw // 2)), 2 * (cells // (bw // 2))
+        inst = ((np.arange(H * W) // 40) % K + 1).reshape(H, W).astype(np.int32)
+        cents = np.stack([-1 + 2 * (cx + 1) / (bw + 1), -1 + 2 * (cy + 1) / (bh + 1)], 1)
+        emb[b] = wl.encode(inst, cents, F, 0.03, rng, np.float16)
+        fg[b] = 1
+    gpu, ora, _ = check_case(emb, fg, bw, bh, T_v=8)
+    assert ora["count"].tolist() == [0, 5, 60]
+
+
 def test_host_front_end_matches_device_path():
     cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=96, W=104, K=10, bins_w=24, bins_h=24)
     fr = wl.make_frame(cfg, 0)
