@@ -12,6 +12,7 @@
 
 #include "assign.cuh"
 #include "assign_mma.cuh"
+#include "assign_tc.cuh"
 #include "cpe.h"
 #include "cpe_common.cuh"
 #include "decode_vote.cuh"
@@ -161,6 +162,39 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   return CPE_OK;
 }
 
+// Blackwell tensor-core path (tcgen05, accumulators in tensor memory); needs 16-byte aligned planes.
+template <typename T, int KA, bool WANT2>
+int launch_assign_tc_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                       const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                       uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min) {
+  // small inputs get short spans so that there are enough CTAs to fill the GPU
+  const int span = ((long long)B * HW >= (1 << 20)) ? 2048 : 512;
+  const int two_tiles = (sizeof(T) == 2 && KA == 16) ? 1 : 0;
+  // as many peaks resident in shared memory as leave room for two CTAs per SM
+  int peak_cap = (p->max_instances + cpe::kTcRound - 1) / cpe::kTcRound * cpe::kTcRound;
+  const int budget = 110 * 1024;
+  const int fixed = cpe::tc_smem_layout(KA, 0, span, two_tiles).total;
+  peak_cap = std::max(cpe::kTcRound, std::min(peak_cap, (budget - fixed) / (2 * KA * 2) / cpe::kTcRound * cpe::kTcRound));
+  // never more than two CTAs per SM: each holds half of the SM's tensor memory
+  const int smem = std::max(cpe::tc_smem_layout(KA, peak_cap, span, two_tiles).total, 78 * 1024);
+  auto kern = cpe::assign_tc_kernel<T, KA, WANT2>;
+  static bool configured = false;   // per instantiation; the attribute is sticky for the process
+  if (!configured) {
+    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+    configured = true;
+  }
+  const int n_spans = (HW + span - 1) / span;
+  const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
+  dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
+  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
+  const int need_exact = p->tau < INFINITY ? 1 : 0;
+  kern<<<grid, cpe::kTcThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact, peak_cap,
+                                            span, vec_mask, labels, best, second, counters, status, votes_to_zero, cells,
+                                            k_min);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
 template <typename T>
 int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                   const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
@@ -178,6 +212,23 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   const T* e = static_cast<const T*>(emb);
   const bool want2 = best != nullptr;
   const int k_min = k_limit + 1;
+  // CPE_ASSIGN_PATH=mma keeps the mma.sync kernel, =tc takes the tcgen05 kernel wherever it can run (comparisons);
+  // by default the tcgen05 kernel serves F > 8, where it is the faster one
+  static const char* path = getenv("CPE_ASSIGN_PATH");
+  const bool tc_ok = (uintptr_t)e % 16 == 0 && HW % 8 == 0;
+  const bool use_tc = tc_ok && (path ? strcmp(path, "tc") == 0 : F > 8);
+  if (use_tc) {
+    if (F <= 8) {
+      return want2 ? launch_assign_tc_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                                     status, votes_to_zero, cells, k_min)
+                   : launch_assign_tc_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                      counters, status, votes_to_zero, cells, k_min);
+    }
+    return want2 ? launch_assign_tc_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                                   status, votes_to_zero, cells, k_min)
+                 : launch_assign_tc_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                    counters, status, votes_to_zero, cells, k_min);
+  }
   if (F <= 8) {
     return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
                                                     status, votes_to_zero, cells, k_min)
@@ -630,3 +681,14 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   p.workspace_bytes = CPE_STATIC_SCRATCH_BYTES;
   return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
 }
+
+#ifdef CPE_TC_PROF
+extern "C" int cpe_tc_prof_read(unsigned long long* out16, int reset) {
+  if (cudaMemcpyFromSymbol(out16, cpe::g_tc_prof, 16 * sizeof(unsigned long long)) != cudaSuccess) return -1;
+  if (reset) {
+    unsigned long long z[16] = {0};
+    if (cudaMemcpyToSymbol(cpe::g_tc_prof, z, sizeof(z)) != cudaSuccess) return -1;
+  }
+  return 0;
+}
+#endif
