@@ -107,8 +107,8 @@ __device__ __forceinline__ bool am_ok(bool ok, uint32_t site, uint32_t* status) 
 }
 
 template <typename T, int KA, bool WANT2>
-__global__ void __launch_bounds__(kAmThreads, 2)
-assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
+__device__ __forceinline__ void
+assign_mma_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
                   const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
                   int peak_cap, int span, int vec_mask, int vec_gather, int32_t* __restrict__ labels, float* __restrict__ best,
                   float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
@@ -860,6 +860,16 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
     if (ws) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_RESCORED], ws);
     if (wf) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_FULL_SCORED], wf);
   }
+}
+
+template <typename T, int KA, bool WANT2>
+__global__ void __launch_bounds__(kAmThreads, 2)
+assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
+                  const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
+                  int peak_cap, int span, int vec_mask, int vec_gather, int32_t* __restrict__ labels, float* __restrict__ best,
+                  float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
+                  uint32_t* __restrict__ votes, int cells, int k_min) {
+  assign_mma_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status_all, votes, cells, k_min);
 }
 
 }  // namespace cpe

@@ -8,25 +8,36 @@
 //     L := 2 S - |Delta| = max(A,B) + 3 min(A,B)   and   S <= L <= d^2 <= 2 S.
 // S and Delta are each one dot product over all 4F channels away from a per-pixel constant (Delta takes the y half
 // with the opposite sign, which the instruction descriptor's negate bit supplies).  The tensor cores deliver, for a
-// tile of 128 pixels x 64 peaks, S_k and Delta_k into tensor memory, the accumulators having been pre-loaded with
-// the per-pixel constants lowered by every error of the approximation (binary16 rounding of the palette and, for
-// binary32 inputs, of the pixel; accumulation), and each thread, owning ONE pixel row, reads its row back with
-// tcgen05.ld:
+// tile of 128 pixels x 64 peaks, the two dot products into tensor memory; a thread that owns ONE pixel row reads
+// the row back with tcgen05.ld and adds the row's constants, lowered by every error of the approximation
+// (binary16 rounding of the palette and, for binary32 inputs, of the pixel; accumulation):
 //   pass 1   the smallest S_k (the second smallest when the runner-up is wanted): d_best^2 <= 2 (S_min + slack) =: thr,
 //            so a peak with L_k > thr cannot be the arg-min.                             1/2 instruction per pair
-//   pass 2   L_k <= thr as a bit mask per row.                                           3 instructions per pair
-//   A row with one bit is decided (no scores wanted, tau = +inf).  A row with several keeps them in registers and
-//   its thread re-scores them in binary32 in the one fixed operation order that defines the result; a row with more
-//   than kTcCand scores every peak.
+//   pass 2   L_k <= thr as a bit mask per row, 4 instructions per pair.  A peak that passes gets bounds
+//            dlo <= d_k <= dhi from its S and Delta; the smallest dhi bounds the best distance, and the row's
+//            candidates are the peaks with dlo below it.
+//   A row with one candidate is decided (no scores wanted, tau = +inf).  The others are queued, per warp, and
+//   worked off when the queue fills up, and at the end by all warps: one lane per (pixel, candidate) pair scores it
+//   in binary32 in the one fixed operation order that defines the result, then one lane per pixel picks the winner.
+//   A row with more than kTcCand candidates scores every peak, a warp per row.
 //
-// Work decomposition: a CTA walks spans of consecutive pixels; it compacts the span's participating 8-pixel groups
-// and gathers 32 groups (256 rows) at a time with 16-byte asynchronous copies into a shared-memory tile that already
-// is the MMA's A operand (pixel-major core matrices, no swizzle; the planar [channel][pixel] input needs no
-// transpose).  The eight threads that fetch a group's channels also reduce the squared norms of its eight pixels
-// among themselves, each ending up with the norms of the row it owns: one barrier per MMA round is all the
-// synchronisation a tile needs.  The peak operand (K-major, rows -2 ex | -2 ey in binary16) is resident in shared
-// memory.  One thread issues the MMAs of a round (2 row blocks x {S, Delta} x 4F/16 k-steps); everybody waits on an
-// mbarrier with a bounded spin.  Two CTAs per SM, 256 tensor-memory columns each.
+// The CTA is a pipeline of two roles that meet only at mbarriers:
+//   producers (4 warps)   take spans of 1024 pixels from a ticket counter: mask pass, compaction of the participating
+//                         8-pixel groups into a ring; per tile of 16 groups (128 rows): 16-byte asynchronous copies
+//                         straight into the MMA's A operand layout (pixel-major core matrices, no swizzle; the planar
+//                         [channel][pixel] input needs no transpose), two tiles ahead; the 8 lanes that fetch a
+//                         group's channels reduce the squared norms of its 8 pixels among themselves, each ending up
+//                         with the norms of the row it describes; row data (pixel index, constants, slack, flags)
+//                         into shared memory.  They never touch tensor memory.
+//   consumers (4 warps)   wait for a stage, read their rows, release the stage, decide or queue, write labels (8 lanes
+//                         = the 8 pixels of a group: full 32-byte sectors).  The last warp to release a stage issues
+//                         the MMAs of the round after next into it (one lane: {S, Delta} x 4F/16 k-steps of M=128,
+//                         N=64, committed to the stage's mbarrier and, with the tile's last round, to the tile
+//                         buffer's).
+// Two tensor-memory stages of 128 columns, four tile buffers (two for F > 8); two CTAs per SM.  Every wait is
+// bounded; a wait that runs out raises a flag that every other wait polls, the status word records it, and the
+// kernel winds down.  (A CTA of a kernel that uses tensor memory keeps the SM to itself until it has given up its
+// right to allocate: hence the relinquish right after the allocation.)
 #pragma once
 
 #include "assign_mma.cuh"
@@ -34,42 +45,53 @@
 
 namespace cpe {
 
-#ifdef CPE_TC_PROF
-__device__ unsigned long long g_tc_prof[16];
-#define TC_PROF(i) do { if (tid == 0) { const long long t_ = clock64(); atomicAdd(&g_tc_prof[i], (unsigned long long)(t_ - prof_t)); prof_t = t_; } } while (0)
-#else
-#define TC_PROF(i) do { } while (0)
-#endif
-
-constexpr int kTcThreads = 256;
-constexpr int kTcRows = 256;        // rows (pixels) per tile: two MMA row blocks of 128
-constexpr int kTcRound = 64;        // peaks per MMA round: S and Delta of both row blocks fill 256 tensor-memory columns
-constexpr int kTcCols = 256;        // tensor-memory columns allocated per CTA
-constexpr int kTcCand = 6;          // candidates a row keeps; more than that and it scores every peak
-constexpr int kTcQueue = 3072;      // queue slots (8 bytes): per undecided row a header and one slot per candidate
-constexpr int kTcFlushAt = kTcQueue - kTcRows * (kTcCand + 1);   // above this a tile's pushes might not fit: score first
-constexpr int kTcHardQueue = 512;   // rows that score every peak
-constexpr int kTcHardFlushAt = kTcHardQueue - kTcRows;
+constexpr int kTcThreads = 256;       // warps 0-3 consume (and issue the MMAs), warps 4-7 produce
+constexpr int kTcRows = 128;          // rows (pixels) per tile: one MMA row block
+constexpr int kTcGroups = kTcRows / 8;
+constexpr int kTcRound = 64;          // peaks per MMA round: S and Delta fill one 128-column stage
+constexpr int kTcCols = 256;          // tensor-memory columns allocated per CTA: two stages
+constexpr int kTcMaxTiles = 4;        // tile buffers: 4 for F <= 8 (copies run two tiles ahead), 2 above (none ahead)
+constexpr int kTcSpan = 1024;         // pixels per producer step: one 8-pixel group per producer thread
+constexpr int kTcRing = 512;          // group ring entries (a span adds at most 128, a tile takes 16)
+constexpr int kTcCand = 8;            // candidates a row keeps (in shared memory); more than that and it scores every peak
+constexpr int kTcQueue = 768;         // queue slots (8 bytes) per consumer warp: a header and one slot per candidate
+constexpr int kTcFlushAt = kTcQueue - 32 * (kTcCand + 1);   // above this a tile's pushes might not fit: score first
+constexpr int kTcHardQueue = 64;      // rows that score every peak, per consumer warp
+constexpr int kTcHardFlushAt = kTcHardQueue - 32;
 constexpr uint32_t kTcHeader = 0x80000000u;
-constexpr int kTcWaitLimit = 1 << 20;
+constexpr int kTcWaitLimit = 1 << 22;
+
+// row flags handed from the producers to the consumers
+constexpr uint32_t kRfGroup = 1u;     // the row belongs to a real group of the tile (its label is written)
+constexpr uint32_t kRfPresent = 2u;   // ... and holds a participating pixel
+constexpr uint32_t kRfLive = 4u;      // ... that is finite: the filter applies
+constexpr uint32_t kRfHard = 8u;      // binary32 pixel beyond the binary16 range: score every peak
+constexpr uint32_t kRfEnd = 16u;      // no more tiles
 
 struct TcSmem {
-  int tile, tile2, peaks, lab, queue, hardq, glist, gbits, misc, total;
+  int tiles, peaks, queue, hardq, cand, clo, ring, ringbits, rpix, rslack, rcs, rcd, rflags, misc, total;
 };
 
 // peak_cap must be a multiple of kTcRound
-__host__ __device__ inline TcSmem tc_smem_layout(int KA, int peak_cap, int span, int two_tiles) {
+__host__ __device__ constexpr int tc_tiles(int KA) { return KA == 16 ? 4 : 2; }
+
+__host__ __device__ inline TcSmem tc_smem_layout(int KA, int peak_cap) {
   TcSmem s;
   int off = 0;
-  s.tile = off;   off += 2 * KA * kTcRows * 2;
-  s.tile2 = off;  off += two_tiles ? 2 * KA * kTcRows * 2 : 0;
-  s.peaks = off;  off += peak_cap * 2 * KA * 2;
-  s.lab = off;    off += span * 4;
-  s.queue = off;  off += kTcQueue * 8;
-  s.hardq = off;  off += kTcHardQueue * 4;
-  s.glist = off;  off += 256 * 2;
-  s.gbits = off;  off += 256;
-  s.misc = off;   off += 128;   // scan scratch (9 ints), queue counters, tensor-memory base, mbarrier
+  s.tiles = off;    off += tc_tiles(KA) * 2 * KA * kTcRows * 2;
+  s.peaks = off;    off += peak_cap * 2 * KA * 2;
+  s.queue = off;    off += 4 * kTcQueue * 8;
+  s.hardq = off;    off += 4 * kTcHardQueue * 4;
+  s.cand = off;     off += kTcCand * kTcRows * 2;
+  s.clo = off;      off += kTcCand * kTcRows * 4;
+  s.ring = off;     off += kTcRing * 4;
+  s.ringbits = off; off += kTcRing;
+  s.rpix = off;     off += tc_tiles(KA) * kTcRows * 4;
+  s.rslack = off;   off += tc_tiles(KA) * kTcRows * 4;
+  s.rcs = off;      off += tc_tiles(KA) * kTcRows * 4;
+  s.rcd = off;      off += tc_tiles(KA) * kTcRows * 4;
+  s.rflags = off;   off += tc_tiles(KA) * kTcRows * 4;
+  s.misc = off;     off += 256;   // producer scan scratch, abort flag, tensor-memory base, mbarriers
   s.total = off;
   return s;
 }
@@ -91,10 +113,12 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr, uint32_t lbo_bytes, 
 constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 15) | ((uint32_t)(kTcRound >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t kTcNegB = 1u << 14;
 
-__device__ __forceinline__ void tc_mma(uint32_t taddr, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+// D (tensor memory) = A B (+ D if accumulate)
+__device__ __forceinline__ void tc_mma(uint32_t taddr, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
   asm volatile(
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(taddr), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(1u)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(taddr), "l"(adesc), "l"(bdesc), "r"(idesc),
+      "r"(accumulate ? 1u : 0u)
       : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint32_t mbar) {
@@ -104,14 +128,30 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Bounded wait for the given phase of an mbarrier; false if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
-  uint32_t done = 0;
-  for (int it = 0; it < kTcWaitLimit && !done; ++it) {
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(mbar) : "memory");
+}
+// Bounded wait for the phase of the given parity; gives up early once the CTA's abort flag is up.  False: gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, const volatile int* abort_flag) {
+  for (int it = 0; it < kTcWaitLimit; ++it) {
+    uint32_t done;
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
                  : "=r"(done) : "r"(mbar), "r"(parity) : "memory");
+    if (done) return true;
+    if ((it & 15) == 15 && *abort_flag) return false;
   }
-  return done != 0;
+  return false;
+}
+// Barrier among the 128 producer threads that also ORs a flag (barrier resource 1)
+__device__ __forceinline__ bool producers_sync_or(bool flag) {
+  uint32_t r;
+  asm volatile(
+      "{\n.reg .pred p, q;\nsetp.ne.b32 p, %1, 0;\nbarrier.cta.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}\n"
+      : "=r"(r) : "r"(flag ? 1u : 0u) : "memory");
+  return r != 0;
 }
 
 // 32 consecutive columns of this thread's tensor-memory lane from each of two addresses; the wait is part of the same
@@ -155,25 +195,11 @@ __device__ __forceinline__ void tc_ld32(uint32_t ta, float (&va)[32]) {
 #pragma unroll
   for (int j = 0; j < 32; ++j) va[j] = __uint_as_float(r[j]);
 }
-// the same value into 32 consecutive columns of this thread's lane
-__device__ __forceinline__ void tc_st32_fill(uint32_t taddr, float value) {
-  const uint32_t c = __float_as_uint(value);
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr), "r"(c)
-      : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
 __device__ __forceinline__ float min3f(float a, float b, float c) {
   float r;
   asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-
-// Offset, in halves, of element (row m, k-slot s) in a tile of kTcRows rows stored as pixel-major core matrices:
-// a core matrix holds 8 k-slots x 8 rows, 16 bytes (8 rows) per k-slot; cores are contiguous along the rows.
-__device__ __forceinline__ int tc_tile_off(int m, int s) { return (s >> 3) * (kTcRows * 8) + (m >> 3) * 64 + (s & 7) * 8 + (m & 7); }
 
 // Sum over the 8 lanes of an aligned lane group of 8 values each, lane j of the group ending up with the total
 // of value j (7 exchanges).
@@ -193,7 +219,7 @@ __device__ __forceinline__ float reduce_scatter8(const float (&a)[8], int j) {
   return keep + __shfl_xor_sync(0xffffffffu, send, 1);
 }
 
-// What the scoring step needs to know about the image and the CTA's shared memory.
+// What the scoring step needs to know about the image.
 template <typename T>
 struct TcScore {
   const T* e_img;
@@ -201,13 +227,9 @@ struct TcScore {
   size_t plane;
   int F, K;
   float tau;
-  int32_t* s_lab;
   int32_t* lab_img;
   float* best_img;
   float* second_img;
-  unsigned long long* s_queue;
-  uint32_t* s_hardq;
-  uint32_t* s_qn;      // [0] queue slots in use, [1] hard rows listed
   uint32_t* status;
 };
 
@@ -243,41 +265,35 @@ __device__ __forceinline__ float tc_exact(const TcScore<T>& sc, uint32_t pix, in
   return __fadd_rn(__fsqrt_rn(s[0]), __fsqrt_rn(s[1]));
 }
 
-// A pixel of the span whose labels are still staged in shared memory gets its label there; an earlier span's
-// label map has been stored already, so the label goes to the map itself.
 template <typename T>
-__device__ __forceinline__ void tc_write_outcome(const TcScore<T>& sc, long long span0, int span_len, uint32_t pix, bool ok,
-                                                 float d1, float d2, int k1, uint32_t& rejected) {
+__device__ __forceinline__ void tc_write_outcome(const TcScore<T>& sc, uint32_t pix, bool ok, float d1, float d2, int k1,
+                                                 uint32_t& rejected) {
   const float inf = __int_as_float(0x7f800000);
+  int label = 0;
   if (ok && k1 >= 0) {
-    if (d1 < sc.tau) {
-      const long long rel = (long long)pix - span0;
-      if (rel >= 0 && rel < span_len) sc.s_lab[rel] = k1 + 1;
-      else sc.lab_img[pix] = k1 + 1;
-    } else {
-      ++rejected;
-    }
+    if (d1 < sc.tau) label = k1 + 1; else ++rejected;
   }
+  sc.lab_img[pix] = label;
   if (sc.best_img) {
     sc.best_img[pix] = ok ? d1 : inf;
     sc.second_img[pix] = ok ? d2 : inf;
   }
 }
 
-// Scores everything queued so far, all threads busy: one thread per (pixel, candidate) pair, then one thread per
-// pixel picks the winner among its pairs; a warp per pixel that scores every peak.  Called by all threads of the CTA
-// right after a barrier; nobody pushes while it runs.  A function of its own: one copy, its own registers.
+// Works off one consumer warp's queues, all lanes busy: one lane per (pixel, candidate) pair, then one lane per
+// pixel picks the winner among its pairs; the whole warp for a pixel that scores every peak.  Called by all 32
+// lanes of a warp; with n_parts > 1 several warps share the queue (part = which share) and the steps are separated
+// by CTA barriers, so every thread of the CTA has to make the call (n = nh = 0 for a warp without a share).
+// A function of its own: one copy, its own registers.
 template <typename T, int KA>
-__device__ __noinline__ void tc_flush(const TcScore<T>& sc, long long span0, int span_len, uint32_t& rejected,
-                                      uint32_t& n_full) {
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+__device__ __noinline__ void tc_flush_warp(const TcScore<T>& sc, unsigned long long* Q, int n, const uint32_t* H, int nh,
+                                           int part, int n_parts, uint32_t& rejected, uint32_t& n_full) {
+  const int lane = (threadIdx.x & 31) + 32 * part, stride = 32 * n_parts;
   const float inf = __int_as_float(0x7f800000);
-  const int n = (int)min(*reinterpret_cast<volatile uint32_t*>(sc.s_qn), (uint32_t)kTcQueue);
-  const int nh = (int)min(*reinterpret_cast<volatile uint32_t*>(sc.s_qn + 1), (uint32_t)kTcHardQueue);
   const int K = sc.K, F = sc.F;
-  unsigned long long* Q = sc.s_queue;
+  if (n_parts > 1) __syncthreads(); else __syncwarp();
   // pairs: (pixel << 32 | k)  ->  (score << 32 | k)
-  for (int e = tid; e < n; e += kTcThreads) {
+  for (int e = lane; e < n; e += stride) {
     const unsigned long long v = Q[e];
     const uint32_t lo = (uint32_t)v, pix = (uint32_t)(v >> 32);
     if (lo & kTcHeader) continue;
@@ -285,15 +301,35 @@ __device__ __noinline__ void tc_flush(const TcScore<T>& sc, long long span0, int
     if (am_ok((int)lo < K, 5u, sc.status)) d = tc_exact<T, KA>(sc, pix, (int)lo);
     Q[e] = ((unsigned long long)__float_as_uint(d) << 32) | lo;
   }
-  // rows that score every peak (pixels beyond the binary16 range, or too many candidates): a warp per row
-  for (int h = wid; h < nh; h += kTcThreads / 32) {
-    const uint32_t pix = sc.s_hardq[h];
+  if (n_parts > 1) __syncthreads(); else __syncwarp();
+  // headers: (pixel << 32 | header bit | count); the row's pairs follow in ascending k, so that the lowest k keeps a tie
+  for (int e = lane; e < n; e += stride) {
+    const unsigned long long v = Q[e];
+    const uint32_t lo = (uint32_t)v, pix = (uint32_t)(v >> 32);
+    if (!(lo & kTcHeader)) continue;
+    const int cnt = (int)(lo & 0xffu);
+    if (!am_ok(cnt <= kTcCand && e + cnt < kTcQueue, 4u, sc.status)) continue;
+    float d1 = inf, d2 = inf;
+    int k1 = -1;
+    for (int i = 1; i <= cnt; ++i) {
+      const unsigned long long w = Q[e + i];
+      const float d = __uint_as_float((uint32_t)(w >> 32));
+      const int k = (int)(uint32_t)w;
+      if (d < d1) { d2 = d1; d1 = d; k1 = k; }
+      else if (d < d2) { d2 = d; }
+    }
+    tc_write_outcome(sc, pix, true, d1, d2, k1, rejected);
+  }
+  // rows that score every peak (pixels beyond the binary16 range, or too many candidates)
+  const int wl = threadIdx.x & 31;   // lane within the warp
+  for (int h = part; h < nh; h += n_parts) {
+    const uint32_t pix = H[h];
     bool ok = true;
     if constexpr (sizeof(T) == 4) {
       // the binary16 copy could not tell an out-of-range value from a non-finite one: look at the originals
       const T* src = sc.e_img + pix;
       float fin = 0.0f;
-      for (int l = lane; l < 2 * F; l += 32)
+      for (int l = wl; l < 2 * F; l += 32)
         fin = fold_finite(fin, Elem<T>::load1(src + (size_t)(2 * l) * sc.plane), Elem<T>::load1(src + (size_t)(2 * l + 1) * sc.plane));
       ok = !__any_sync(0xffffffffu, fin != fin);
     }
@@ -301,7 +337,7 @@ __device__ __noinline__ void tc_flush(const TcScore<T>& sc, long long span0, int
     int k1 = -1;
     if (ok) {
 #pragma unroll 1
-      for (int k = lane; k < K; k += 32) {
+      for (int k = wl; k < K; k += 32) {
         const float d = tc_exact<T, KA>(sc, pix, k);
         if (d < d1) { d2 = d1; d1 = d; k1 = k; }
         else if (d < d2) { d2 = d; }
@@ -320,63 +356,54 @@ __device__ __noinline__ void tc_flush(const TcScore<T>& sc, long long span0, int
       k1 = pack_k(bestp);
       d2 = r2;
     }
-    if (lane == 0) {
+    if (wl == 0) {
       if (ok) ++n_full;
-      tc_write_outcome(sc, span0, span_len, pix, ok, d1, d2, k1, rejected);
+      tc_write_outcome(sc, pix, ok, d1, d2, k1, rejected);
     }
   }
-  __syncthreads();
-  if (tid == 0) {
-    sc.s_qn[0] = 0;      // everybody has read the counts; nobody pushes before this function's last barrier
-    sc.s_qn[1] = 0;
-  }
-  // headers: (pixel << 32 | header bit | count); the row's pairs follow in ascending k, so that the lowest k keeps a tie
-  for (int e = tid; e < n; e += kTcThreads) {
-    const unsigned long long v = Q[e];
-    const uint32_t lo = (uint32_t)v, pix = (uint32_t)(v >> 32);
-    if (!(lo & kTcHeader)) continue;
-    const int cnt = (int)(lo & 0xffu);
-    if (!am_ok(cnt <= kTcCand && e + cnt < kTcQueue, 4u, sc.status)) continue;
-    float d1 = inf, d2 = inf;
-    int k1 = -1;
-    for (int i = 1; i <= cnt; ++i) {
-      const unsigned long long w = Q[e + i];
-      const float d = __uint_as_float((uint32_t)(w >> 32));
-      const int k = (int)(uint32_t)w;
-      if (d < d1) { d2 = d1; d1 = d; k1 = k; }
-      else if (d < d2) { d2 = d; }
-    }
-    tc_write_outcome(sc, span0, span_len, pix, true, d1, d2, k1, rejected);
-  }
-  __syncthreads();
+  __syncwarp();
 }
 
-// Requires 16-byte aligned planes: emb 16-byte aligned and HW a multiple of 8 (the caller falls back to the
-// mma.sync kernel otherwise).  KA = 16 serves F <= 8, KA = 32 serves F <= 16.
+// Requires 16-byte aligned planes: emb 16-byte aligned and HW a multiple of 8 (the caller takes the mma.sync kernel
+// otherwise).  KA = 16 serves F <= 8, KA = 32 serves F <= 16.  Images with fewer than k_min or more than
+// min(k_max, peak_cap) peaks are not touched.
 template <typename T, int KA, bool WANT2>
-__global__ void __launch_bounds__(kTcThreads, 2)
-assign_tc_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
+__device__ __forceinline__ void
+assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
                  const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
-                 int peak_cap, int span, int vec_mask, int32_t* __restrict__ labels, float* __restrict__ best,
+                 int peak_cap, int vec_mask, int32_t* __restrict__ labels, float* __restrict__ best,
                  float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
-                 uint32_t* __restrict__ votes, int cells, int k_min) {
+                 uint32_t* __restrict__ votes, int cells, int k_min, int k_max, uint32_t* __restrict__ acc) {
   constexpr int KS = KA / 16;                       // k-steps per axis
+  constexpr int kTiles = tc_tiles(KA);              // tile buffers
+  constexpr int kAhead = kTiles - 2;                // tiles whose copies are in flight while one is being completed
   constexpr int kTileHalves = 2 * KA * kTcRows;
-  constexpr uint32_t kTileLbo = kTcRows * 16;       // bytes between core matrices along K in the tile
+  constexpr uint32_t kTileLbo = kTcRows * 16;       // bytes between core matrices along K in a tile
   extern __shared__ __align__(1024) unsigned char tc_smem[];
-  constexpr int two_tiles = (sizeof(T) == 2 && KA == 16) ? 1 : 0;   // prefetch the next tile while this one is swept
-  const TcSmem L = tc_smem_layout(KA, peak_cap, span, two_tiles);
-  int32_t* s_lab = reinterpret_cast<int32_t*>(tc_smem + L.lab);
-  __half* s_tile0 = reinterpret_cast<__half*>(tc_smem + L.tile);
+  const TcSmem L = tc_smem_layout(KA, peak_cap);
+  __half* s_tiles = reinterpret_cast<__half*>(tc_smem + L.tiles);
   __half* s_pk = reinterpret_cast<__half*>(tc_smem + L.peaks);
-  uint16_t* s_glist = reinterpret_cast<uint16_t*>(tc_smem + L.glist);     // participating 8-pixel groups of the span
-  uint8_t* s_gbits = reinterpret_cast<uint8_t*>(tc_smem + L.gbits);       // which of a group's 8 pixels participate
   unsigned long long* s_queue = reinterpret_cast<unsigned long long*>(tc_smem + L.queue);
   uint32_t* s_hardq = reinterpret_cast<uint32_t*>(tc_smem + L.hardq);
-  int* s_scan = reinterpret_cast<int*>(tc_smem + L.misc);                 // [0..8] warp offsets and total
-  uint32_t* s_qn = reinterpret_cast<uint32_t*>(s_scan + 10);              // [0] queue slots in use, [1] hard rows listed
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_scan + 12);
-  uint64_t* s_mbar = reinterpret_cast<uint64_t*>(tc_smem + L.misc + 64);
+  uint16_t* s_cand = reinterpret_cast<uint16_t*>(tc_smem + L.cand);       // [slot][row]: the peaks that passed, per row
+  float* s_clo = reinterpret_cast<float*>(tc_smem + L.clo);               // [slot][row]: their lower bounds of the distance
+  uint32_t* s_ring = reinterpret_cast<uint32_t*>(tc_smem + L.ring);       // participating 8-pixel groups, in pixel order
+  uint8_t* s_ringbits = reinterpret_cast<uint8_t*>(tc_smem + L.ringbits); // which of a group's 8 pixels participate
+  uint32_t* s_rpix = reinterpret_cast<uint32_t*>(tc_smem + L.rpix);       // per tile buffer and row: pixel index
+  float* s_rslack = reinterpret_cast<float*>(tc_smem + L.rslack);         // ... the row's error bound dS
+  float* s_rcs = reinterpret_cast<float*>(tc_smem + L.rcs);               // ... S_lo = cS + the S accumulator
+  float* s_rcd = reinterpret_cast<float*>(tc_smem + L.rcd);               // ... Delta = cD + the Delta accumulator
+  uint32_t* s_rflags = reinterpret_cast<uint32_t*>(tc_smem + L.rflags);   // ... kRf* flags
+  int* s_scan = reinterpret_cast<int*>(tc_smem + L.misc);                 // [0..3] producer warps' group counts
+  volatile int* s_abort = s_scan + 8;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_scan + 9);
+  int* s_qfill = s_scan + 10;                                             // [0..7] the consumer warps' queue fills at the end
+  uint32_t* s_relcnt = reinterpret_cast<uint32_t*>(s_scan + 18);          // [2] releases of a stage so far
+  volatile uint32_t* s_endtile = reinterpret_cast<volatile uint32_t*>(s_scan + 20);   // index of the end marker's tile, once known
+  const uint32_t mbar0 = (uint32_t)__cvta_generic_to_shared(tc_smem + L.misc + 96);
+  // mbarriers: a stage's MMAs are done [2], it has been read [2]; a tile buffer's pixels and row data are in place [4],
+  // the buffer has been read by its last MMA [4], its row data have been read by the consumers [4]
+  const uint32_t mb_done = mbar0, mb_free = mbar0 + 16, mb_meta = mbar0 + 32, mb_tile = mbar0 + 64, mb_rows = mbar0 + 96;
 
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -389,231 +416,171 @@ assign_tc_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
   const uint8_t* fg_img = fg ? fg + (size_t)b * plane : nullptr;
   const float* pk_img = peak_emb + (size_t)b * K_max * D;
   const int K = count_ptr[b];
-  if (K < k_min) return;     // few peaks: this image is done by the plain all-pairs kernel launched next to this one
+  if (K < k_min || K > k_max || K > peak_cap) return;
   const float inf = __int_as_float(0x7f800000);
   const float qnan = __int_as_float(0x7fc00000);
-  const int n_spans = (HW + span - 1) / span;
-  const int n_pchunks = K > 0 ? (K + peak_cap - 1) / peak_cap : 0;
   int32_t* lab_img = labels + (size_t)b * plane;
   float* best_img = best ? best + (size_t)b * plane : nullptr;
   float* second_img = second ? second + (size_t)b * plane : nullptr;
-  const int n_grp_span = span >> 3;                 // 8-pixel groups per span (<= 256): thread t owns group t
-  const uint32_t mbar = (uint32_t)__cvta_generic_to_shared(s_mbar);
   const uint32_t pk_lbo = (uint32_t)peak_cap * 16u; // bytes between core matrices along K in the peak operand
-  const bool score_all = WANT2 || need_exact;       // scores wanted: every passing pair is re-scored
-  const bool one_round = n_pchunks == 1 && K <= kTcRound;   // pass 2 finds pass 1's accumulators still in tensor memory
-  // a row's 8 pixels = the 8 lanes gl*8 .. gl*8+7; lane cq fetches channels cq, cq+8, ... of group gl and owns row tid
-  const int gl = tid >> 3, cq = tid & 7;
+  const bool score_all = WANT2 || need_exact;       // scores wanted: every row is re-scored
+  const int R1 = (K + kTcRound - 1) / kTcRound;     // rounds of 64 peaks
+  const bool combined = R1 == 1;                    // one round serves both passes
+  const int n_rounds = combined ? 1 : 2 * R1;       // per tile: pass 1 rounds (S only), then pass 2 rounds (S and Delta)
 
-  // ---- one-time set-up: tensor memory, barrier, zeroed tiles (padding k-slots must stay zero), peak operand
+  // ---- one-time set-up: tensor memory, barriers, zeroed tiles (padding k-slots must stay zero), peak operand
   if (wid == 0) {
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(s_tmem);
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst), "r"(kTcCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar) : "memory");
-    s_qn[0] = 0;
-    s_qn[1] = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(mb_done + 8 * i, 1);    // the MMA commit
+      mbar_init(mb_free + 8 * i, 4);    // one arrival per consumer warp
+    }
+    for (int i = 0; i < kTcMaxTiles; ++i) {
+      mbar_init(mb_meta + 8 * i, 4);    // one arrival per producer warp
+      mbar_init(mb_tile + 8 * i, 1);    // the MMA commit
+      mbar_init(mb_rows + 8 * i, 4);    // one arrival per consumer warp
+    }
+    *s_abort = 0;
+    for (int i = 0; i < 8; ++i) s_qfill[i] = 0;
+    s_relcnt[0] = 0;
+    s_relcnt[1] = 0;
+    *s_endtile = 0xffffffffu;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i < (1 + two_tiles) * kTileHalves / 2; i += kTcThreads) reinterpret_cast<uint32_t*>(s_tile0)[i] = 0u;
-
+  for (int i = tid; i < kTiles * kTileHalves / 2; i += kTcThreads) reinterpret_cast<uint32_t*>(s_tiles)[i] = 0u;
   // peak operand, K-major core matrices: row k = [-2 ex (2F), 0.., -2 ey (2F), 0..] in binary16 (the factor -2 is
   // exact); rows beyond the last peak are NaN, so that their columns never win a minimum nor pass a comparison
-  auto load_peaks = [&](int pc) {
-    const int k0 = pc * peak_cap;
-    const int kn = min(peak_cap, K - k0);
-    const int kn_r = (kn + kTcRound - 1) / kTcRound * kTcRound;
+  {
+    const int kn_r = R1 * kTcRound;
     for (int i = tid; i < kn_r * 2 * KA; i += kTcThreads) {
       const int k = i / (2 * KA), s = i - k * 2 * KA;
       const int axis = s / KA, cc = s - axis * KA;
       float v = 0.0f;
-      if (k >= kn) v = qnan;
-      else if (cc < 2 * F) v = -2.0f * pk_img[(size_t)(k0 + k) * D + axis * 2 * F + cc];
+      if (k >= K) v = qnan;
+      else if (cc < 2 * F) v = -2.0f * pk_img[(size_t)k * D + axis * 2 * F + cc];
       s_pk[(s >> 3) * (peak_cap * 8) + k * 8 + (s & 7)] = __float2half_rn(v);
     }
-    fence_async_smem();
-  };
-  if (n_pchunks == 1) load_peaks(0);
+  }
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  // this thread's row of the tile: row block mt = wid / 4 uses tensor-memory columns [128 mt, 128 mt + 128):
-  // S in the first 64, Delta in the last 64; a warp reaches the 32 lanes 32 (wid % 4) ...
-  const uint32_t t_row = tmem + ((uint32_t)((wid & 3) * 32) << 16) + (uint32_t)((wid >> 2) * 128);
-  uint32_t phase = 0;
-  bool failed = false, timed_out = false;
-
-  // MMAs of one round: peaks [n0, n0 + 64) of the resident chunk against both row blocks of the tile
-  auto issue_round = [&](const __half* tile, int n0, bool with_delta) {
-    const uint32_t a0 = (uint32_t)__cvta_generic_to_shared(tile);
-    const uint32_t b0 = (uint32_t)__cvta_generic_to_shared(s_pk) + (uint32_t)n0 * 16u;
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int acc = 0; acc < 2; ++acc) {
-        if (acc == 1 && !with_delta) continue;
-#pragma unroll
-        for (int ks = 0; ks < 2 * KS; ++ks) {
-          const uint64_t da = tc_desc(a0 + (uint32_t)ks * 2u * kTileLbo + (uint32_t)mt * 2048u, kTileLbo, 128u);
-          const uint64_t db = tc_desc(b0 + (uint32_t)ks * 2u * pk_lbo, pk_lbo, 128u);
-          const uint32_t id = (acc == 1 && ks >= KS) ? (kTcIdesc | kTcNegB) : kTcIdesc;
-          tc_mma(tmem + (uint32_t)(mt * 128 + acc * 64), da, db, id);
-        }
-      }
-    tc_commit(mbar);
-  };
 
   uint32_t rejected = 0, n_pairs = 0, n_rescored = 0, n_full = 0;
   TcScore<T> sc;
   sc.e_img = e_img; sc.pk_img = pk_img; sc.plane = plane; sc.F = F; sc.K = K; sc.tau = tau;
-  sc.s_lab = s_lab; sc.lab_img = lab_img; sc.best_img = best_img; sc.second_img = second_img;
-  sc.s_queue = s_queue; sc.s_hardq = s_hardq; sc.s_qn = s_qn; sc.status = status;
-#ifdef CPE_TC_PROF
-  long long prof_t = clock64();
-#endif
+  sc.lab_img = lab_img; sc.best_img = best_img; sc.second_img = second_img; sc.status = status;
 
-  for (int sp = blockIdx.x; sp < n_spans && !failed; sp += gridDim.x) {
-    // later spans first: the tail of the voting pass is what is still in L2
-    const long long span0 = (long long)(n_spans - 1 - sp) * span;
-    const int span_len = (int)min((long long)span, (long long)HW - span0);
+  if (wid >= 4) {
+    // =============================================================================================== producers
+    const int ptid = tid - 128, pw = ptid >> 5;
+    const int gl = ptid >> 3, cq = ptid & 7;        // lane cq fetches channels cq, cq+8, ... of group gl, owns row ptid
+    const int n_spans = (HW + kTcSpan - 1) / kTcSpan;
+    const bool lab16 = ((uintptr_t)lab_img & 15u) == 0;
+    const bool sc16 = best_img && ((uintptr_t)best_img & 15u) == 0 && ((uintptr_t)second_img & 15u) == 0;
+    uint32_t t = 0, tdone = 0;                      // tiles issued, tiles completed
+    uint32_t ring_head = 0, ring_tail = 0;          // groups taken, groups appended
+    bool bad = false;                               // some producer's wait has run out: the same in all producers
+    bool my_bad = false;                            // this thread's wait has run out (not yet agreed on)
+    int pend_ng[3] = {0, 0, 0};                     // groups of the tiles whose copies are in flight, oldest first
+    uint32_t pend_head[3] = {0, 0, 0};
+    int n_pend = 0;
 
-    // ---- mask pass and compaction of the span's participating 8-pixel groups; background pixels get their outputs here
-    {
-      const long long p0 = span0 + (long long)tid * 8;
-      const bool mine = tid < n_grp_span && p0 < HW;     // HW is a multiple of 8: the whole group is inside
-      uint32_t bits = 0;
-      if (mine) {
-        if (!fg_img) {
-          bits = 0xffu;
-        } else if (vec_mask) {
-          const uint2 w = __ldg(reinterpret_cast<const uint2*>(fg_img + p0));
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            bits |= (((w.x >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
-            bits |= (((w.y >> (8 * j)) & 0xffu) ? 1u : 0u) << (4 + j);
-          }
-        } else {
-          for (int j = 0; j < 8; ++j)
-            if (__ldg(fg_img + p0 + j)) bits |= 1u << j;
-        }
-        if (best_img) {
-          for (int j = 0; j < 8; ++j)
-            if (K == 0 || !((bits >> j) & 1u)) {
-              best_img[p0 + j] = inf;
-              second_img[p0 + j] = inf;
-            }
-        }
-      }
-      for (int i = tid; i < span / 4; i += kTcThreads) reinterpret_cast<int4*>(s_lab)[i] = make_int4(0, 0, 0, 0);
-      const uint32_t gm = __ballot_sync(0xffffffffu, bits != 0);
-      if (lane == 0) s_scan[wid] = __popc(gm);
-      __syncthreads();
-      if (tid == 0) {
-        int run = 0;
-#pragma unroll
-        for (int w = 0; w < kTcThreads / 32; ++w) {
-          const int v = s_scan[w];
-          s_scan[w] = run;
-          run += v;
-        }
-        s_scan[kTcThreads / 32] = run;
-      }
-      __syncthreads();
-      if (bits) {
-        const int gi = s_scan[wid] + __popc(gm & ((1u << lane) - 1u));
-        s_glist[gi] = (uint16_t)tid;
-        s_gbits[gi] = (uint8_t)bits;
-      }
-      __syncthreads();
-    }
-    const int n_groups = s_scan[kTcThreads / 32];
-    const int n_chunks = K > 0 ? (n_groups + 31) / 32 : 0;
-    TC_PROF(0);
-
-    // One tile = 32 groups x 4F channels, 16 bytes (8 pixels of one channel) per copy, written where the MMA reads
-    // them: k-slot s of group gl at core matrix (gl, s / 8), row s % 8.  This thread: group gl, channels cq, cq+8, ...
     auto slot_of = [&](int c) { return c >= 2 * F ? KA + (c - 2 * F) : c; };
     auto unit_ptr = [&](__half* tile, int c) {
       const int s = slot_of(c);
       return tile + (s >> 3) * (kTcRows * 8) + gl * 64 + (s & 7) * 8;
     };
-    auto issue_gather = [&](int ci, __half* dst_tile) {
+    // copies of tile t (ng groups from ring position head) into buffer t % kTiles
+    auto issue = [&](int ng, uint32_t head) {
+      const int us = (int)(t % kTiles);
+      if (!my_bad && !mbar_wait(mb_tile + 8 * us, ((t / kTiles) & 1u) ^ 1u, s_abort)) {   // its previous tile has been read
+        my_bad = true;
+        *s_abort = 1;
+      }
       if constexpr (sizeof(T) == 2) {
-        const int gi = ci * 32 + gl;
-        if (gi < n_groups) {
-          const T* src0 = e_img + span0 + (int)s_glist[gi] * 8;
+        if (!my_bad && gl < ng) {
+          const T* src0 = e_img + (size_t)s_ring[(head + gl) & (kTcRing - 1)] * 8;
+          __half* tile = s_tiles + (size_t)us * kTileHalves;
           for (int c = cq; c < D; c += 8) {
-            const uint32_t d32 = (uint32_t)__cvta_generic_to_shared(unit_ptr(dst_tile, c));
+            const uint32_t d32 = (uint32_t)__cvta_generic_to_shared(unit_ptr(tile, c));
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d32), "l"(src0 + (size_t)c * plane));
           }
         }
         asm volatile("cp.async.commit_group;\n" ::);
       }
     };
-    if (two_tiles && n_chunks > 0) issue_gather(0, s_tile0);
-
-    for (int ci = 0; ci < n_chunks && !failed; ++ci) {
-      __half* s_tile = two_tiles ? s_tile0 + (size_t)(ci & 1) * kTileHalves : s_tile0;
-      const int gi = ci * 32 + gl;
-      // ---- gather (or its completion) and the squared norms of the group's 8 pixels over this thread's channels
+    // everything else for tile u: norms, constants, rounds.  `newer` = copy groups issued after this tile's.
+    auto complete = [&](uint32_t u, int ng, uint32_t head, int newer) {
+      const int us = (int)(u % kTiles);
+      __half* tile = s_tiles + (size_t)us * kTileHalves;
       float ax[8], ay[8];
 #pragma unroll
       for (int r = 0; r < 8; ++r) ax[r] = ay[r] = 0.0f;
       auto add_squares = [&](const uint4& q, int c) {
         const __half2* h = reinterpret_cast<const __half2*>(&q);
-        float t[8];
+        float f[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float2 f = __half22float2(h[i]);
-          t[2 * i] = f.x * f.x;
-          t[2 * i + 1] = f.y * f.y;
+          const float2 v = __half22float2(h[i]);
+          f[2 * i] = v.x;
+          f[2 * i + 1] = v.y;
         }
         if (c < 2 * F) {
 #pragma unroll
-          for (int r = 0; r < 8; ++r) ax[r] += t[r];
+          for (int r = 0; r < 8; ++r) ax[r] = fmaf(f[r], f[r], ax[r]);
         } else {
 #pragma unroll
-          for (int r = 0; r < 8; ++r) ay[r] += t[r];
+          for (int r = 0; r < 8; ++r) ay[r] = fmaf(f[r], f[r], ay[r]);
         }
       };
+      uint32_t grp = 0, bits = 0;
+      if (gl < ng) {
+        grp = s_ring[(head + gl) & (kTcRing - 1)];
+        bits = s_ringbits[(head + gl) & (kTcRing - 1)];
+      }
       if constexpr (sizeof(T) == 2) {
-        if (!two_tiles) issue_gather(ci, s_tile);
-        asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-        if (gi < n_groups)
-          for (int c = cq; c < D; c += 8) add_squares(*reinterpret_cast<const uint4*>(unit_ptr(s_tile, c)), c);
+        if (newer >= 2) asm volatile("cp.async.wait_group 2;\n" ::: "memory");
+        else if (newer == 1) asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+        if (gl < ng)
+          for (int c = cq; c < D; c += 8) add_squares(*reinterpret_cast<const uint4*>(unit_ptr(tile, c)), c);
       } else {
         // binary32: two 128-bit loads per unit, rounded to binary16 on the way
-        if (gi < n_groups) {
-          const T* src0 = e_img + span0 + (int)s_glist[gi] * 8;
+        if (gl < ng) {
+          const T* src0 = e_img + (size_t)grp * 8;
           for (int c = cq; c < D; c += 8) {
             const float4* src = reinterpret_cast<const float4*>(src0 + (size_t)c * plane);
             const float4 lo = __ldg(src), hi = __ldg(src + 1);
             __half2 h[4] = {__floats2half2_rn(lo.x, lo.y), __floats2half2_rn(lo.z, lo.w),
                             __floats2half2_rn(hi.x, hi.y), __floats2half2_rn(hi.z, hi.w)};
             const uint4 q = *reinterpret_cast<const uint4*>(h);
-            *reinterpret_cast<uint4*>(unit_ptr(s_tile, c)) = q;
+            *reinterpret_cast<uint4*>(unit_ptr(tile, c)) = q;
             add_squares(q, c);
           }
         }
       }
       fence_async_smem();
       const float nx = reduce_scatter8(ax, cq), ny = reduce_scatter8(ay, cq);
-      TC_PROF(1);
 
-      // ---- this thread's row (pixel cq of group gl): error bounds, accumulator constants
-      int off = 0xffff;
-      if (gi < n_groups && ((s_gbits[gi] >> cq) & 1u)) off = (int)s_glist[gi] * 8 + cq;
-      const bool present = off != 0xffff && am_ok(off < span_len, 1u, status);
+      // this thread's row (pixel cq of group gl): flags, error bounds, accumulator constants
+      const bool in_group = gl < ng;
+      const bool present = in_group && ((bits >> cq) & 1u);
       const bool finite = (nx + ny) < inf;
       // binary16 pixels: a non-finite norm is a non-finite pixel.  binary32 pixels: it may also be a value beyond
       // the binary16 range, so the row is scored exactly (and its finiteness checked there).
-      bool valid = present && (finite || sizeof(T) == 4);
-      bool hard = present && !finite && sizeof(T) == 4;
       const bool live = present && finite;
-      float cS, cD, dS;      // accumulator constants; S_lo <= S <= S_lo + 2 dS and |Delta - Delta_c| <= dS
+      uint32_t flags = 0;
+      if (in_group) flags |= kRfGroup;
+      if (present) flags |= kRfPresent;
+      if (live) flags |= kRfLive;
+      if (present && !finite && sizeof(T) == 4) flags |= kRfHard;
+      float cS, cD, dS;      // S_lo <= S <= S_lo + 2 dS and |Delta - Delta_c| <= dS
       {
         const float kappa = (sizeof(T) == 4 ? 3.0f : 1.0f) * 4.93e-4f;   // 2^-11 * 1.01 (x3: pixel rounding too)
         const float sq2f = sqrtf(2.0f * (float)F);
@@ -627,171 +594,423 @@ assign_tc_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
         cS = (cfx + cfy) - dS;
         cD = nnx - nny;
       }
-      TC_PROF(2);
+      // row data for the consumers (who must be through with the buffer's previous tile's); with the arrival the tile
+      // is handed to the MMA warp as well
+      if (!my_bad && !mbar_wait(mb_rows + 8 * us, ((u / kTiles) & 1u) ^ 1u, s_abort)) {
+        my_bad = true;
+        *s_abort = 1;
+      }
+      s_rpix[us * kTcRows + ptid] = grp * 8u + (uint32_t)cq;
+      s_rslack[us * kTcRows + ptid] = dS;
+      s_rcs[us * kTcRows + ptid] = cS;
+      s_rcd[us * kTcRows + ptid] = cD;
+      s_rflags[us * kTcRows + ptid] = flags;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(mb_meta + 8 * us);
+    };
+    // a new tile's copies go out, then the oldest tile in flight is completed once kAhead newer ones are on their way
+    auto emit = [&](int ng) {
+      const uint32_t head = ring_head;
+      issue(ng, head);
+      ring_head += (uint32_t)ng;
+      pend_ng[n_pend] = ng;
+      pend_head[n_pend] = head;
+      ++n_pend;
+      ++t;
+      if (n_pend > kAhead) {
+        complete(tdone, pend_ng[0], pend_head[0], n_pend - 1);
+        ++tdone;
+        pend_ng[0] = pend_ng[1]; pend_ng[1] = pend_ng[2];
+        pend_head[0] = pend_head[1]; pend_head[1] = pend_head[2];
+        --n_pend;
+      }
+    };
 
-      // One round: constants into tensor memory, barrier, MMAs, wait.  Returns false, for every thread, once any
-      // thread's wait has run out (the barrier itself carries the flag).
-      bool first_round = true;
-      auto run_round = [&](int n0, bool with_delta) -> bool {
-        tc_st32_fill(t_row, cS);
-        tc_st32_fill(t_row + 32, cS);
-        if (with_delta) {
-          tc_st32_fill(t_row + 64, cD);
-          tc_st32_fill(t_row + 96, cD);
+    // mask of this thread's group in a span, loaded one span ahead
+    auto load_mask = [&](int sp) -> uint32_t {
+      const long long p0 = (long long)(n_spans - 1 - sp) * kTcSpan + (long long)ptid * 8;
+      uint32_t bits = 0;
+      if (sp >= 0 && sp < n_spans && p0 < HW) {        // HW is a multiple of 8: the whole group is inside
+        if (!fg_img) {
+          bits = 0xffu;
+        } else if (vec_mask) {
+          const uint2 w = __ldg(reinterpret_cast<const uint2*>(fg_img + p0));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            bits |= (((w.x >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+            bits |= (((w.y >> (8 * j)) & 0xffu) ? 1u : 0u) << (4 + j);
+          }
+        } else {
+          for (int j = 0; j < 8; ++j)
+            if (__ldg(fg_img + p0 + j)) bits |= 1u << j;
         }
-        tc_wait_st();
-        tc_fence_before();
-        // the barrier also tells whether any wait has run out, and whether the queues have to be worked off before
-        // this tile pushes (the last thread to arrive sees every push of the previous tile)
-        const bool full = *reinterpret_cast<volatile uint32_t*>(s_qn) > (uint32_t)kTcFlushAt ||
-                          *reinterpret_cast<volatile uint32_t*>(s_qn + 1) > (uint32_t)kTcHardFlushAt;
-        bool flush = false;
-        if (__syncthreads_or((timed_out || full) ? 1 : 0)) {
-          if (__syncthreads_or(timed_out ? 1 : 0)) return false;
-          flush = true;
+      }
+      return bits;
+    };
+    // Spans are handed out by a ticket counter (one per image, zero at launch): later spans first, because the tail
+    // of the voting pass is what is still in L2, and dynamically, because the participating pixels are spread unevenly.
+    uint32_t* ticket = acc + b * kAccStride + kAccSpan;
+    if (ptid == 0) s_scan[6] = (int)atomicAdd(ticket, 1u);
+    bad = producers_sync_or(my_bad);
+    int cur = s_scan[6];
+    uint32_t next_bits = load_mask(cur);
+    while (cur < n_spans && !bad) {
+      const long long span0 = (long long)(n_spans - 1 - cur) * kTcSpan;
+      const long long p0 = span0 + (long long)ptid * 8;
+      const uint32_t bits = next_bits;
+      if (ptid == 0) s_scan[7] = (int)atomicAdd(ticket, 1u);    // the span after this one
+      if (p0 < HW && bits == 0) {
+        // a group without a participating pixel: its outputs are written here
+        if (lab16) {
+          reinterpret_cast<int4*>(lab_img + p0)[0] = make_int4(0, 0, 0, 0);
+          reinterpret_cast<int4*>(lab_img + p0)[1] = make_int4(0, 0, 0, 0);
+        } else {
+          for (int j = 0; j < 8; ++j) lab_img[p0 + j] = 0;
         }
-        if (tid == 0) {
-          tc_fence_after();
-          issue_round(s_tile, n0, with_delta);
+        if (best_img) {
+          if (sc16) {
+            const float4 v = make_float4(inf, inf, inf, inf);
+            reinterpret_cast<float4*>(best_img + p0)[0] = v;
+            reinterpret_cast<float4*>(best_img + p0)[1] = v;
+            reinterpret_cast<float4*>(second_img + p0)[0] = v;
+            reinterpret_cast<float4*>(second_img + p0)[1] = v;
+          } else {
+            for (int j = 0; j < 8; ++j) {
+              best_img[p0 + j] = inf;
+              second_img[p0 + j] = inf;
+            }
+          }
         }
-        // every thread is past the previous tile: its buffer can take the tile after this one
-        if (first_round && two_tiles && ci + 1 < n_chunks) issue_gather(ci + 1, s_tile0 + (size_t)((ci + 1) & 1) * kTileHalves);
-        first_round = false;
-        if (flush) tc_flush<T, KA>(sc, span0, span_len, rejected, n_full);   // while the tensor cores work
-        if (!mbar_wait(mbar, phase)) {
-          timed_out = true;
-          am_ok(false, 8u, status);
+      }
+      // append the participating groups to the ring, in pixel order
+      const uint32_t gm = __ballot_sync(0xffffffffu, bits != 0);
+      if (lane == 0) s_scan[pw] = __popc(gm);
+      bad = producers_sync_or(my_bad);
+      if (bad) break;
+      const int nxt = s_scan[7];
+      next_bits = load_mask(nxt);                      // in flight while this span's tiles are put together
+      int before = 0, total = 0;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const int v = s_scan[w];
+        if (w < pw) before += v;
+        total += v;
+      }
+      if (bits) {
+        const uint32_t pos = ring_tail + (uint32_t)before + (uint32_t)__popc(gm & ((1u << lane) - 1u));
+        s_ring[pos & (kTcRing - 1)] = (uint32_t)(p0 >> 3);
+        s_ringbits[pos & (kTcRing - 1)] = (uint8_t)bits;
+      }
+      bad = producers_sync_or(my_bad);  // ring entries written, scan scratch free again
+      if (bad) break;
+      ring_tail += (uint32_t)total;
+      while (ring_tail - ring_head >= (uint32_t)kTcGroups) emit(kTcGroups);
+      cur = nxt;
+    }
+    if (!bad && ring_tail != ring_head) emit((int)(ring_tail - ring_head));
+    while (!bad && n_pend > 0) {
+      complete(tdone, pend_ng[0], pend_head[0], n_pend - 1);
+      ++tdone;
+      pend_ng[0] = pend_ng[1]; pend_ng[1] = pend_ng[2];
+      pend_head[0] = pend_head[1]; pend_head[1] = pend_head[2];
+      --n_pend;
+    }
+    if (!bad) {
+      // end marker in the row data of the next tile buffer, once the buffer's previous tile has been worked off
+      const int us = (int)(t % kTiles);
+      if (!mbar_wait(mb_tile + 8 * us, ((t / kTiles) & 1u) ^ 1u, s_abort) ||
+          !mbar_wait(mb_rows + 8 * us, ((t / kTiles) & 1u) ^ 1u, s_abort)) {
+        my_bad = true;
+        *s_abort = 1;
+      }
+      s_rflags[us * kTcRows + ptid] = kRfEnd;
+      if (ptid == 0) *s_endtile = t;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(mb_meta + 8 * us);
+    }
+    if (bad || my_bad) {
+      *s_abort = 1;
+      am_ok(false, 8u, status);
+    }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
+  } else {
+    // =============================================================================================== consumers
+    const uint32_t t_lane = tmem + ((uint32_t)(wid * 32) << 16);
+    unsigned long long* Qw = s_queue + (size_t)wid * kTcQueue;
+    uint32_t* Hw = s_hardq + (size_t)wid * kTcHardQueue;
+    int qn = 0, nh = 0;                             // the warp's queue fill (the same in all lanes)
+    uint32_t t = 0, rc = 0;                         // tiles taken, rounds taken
+    bool bad = false;                               // a wait of this warp has run out
+    // waits as a warp: either every lane saw the phase complete, or the warp gives up
+    auto wait_all = [&](uint32_t mbar, uint32_t parity) {
+      const bool ok = mbar_wait(mbar, parity, s_abort);
+      return __all_sync(0xffffffffu, ok) != 0;
+    };
+    // MMAs of round q (counted over all tiles) into stage q & 1; called by one lane.  The tile's operand has to be in
+    // place (its end marker stops the issue) and the stage has to have been read by all four consumer warps.
+    const uint64_t da0 = tc_desc((uint32_t)__cvta_generic_to_shared(s_tiles), kTileLbo, 128u);
+    const uint64_t db0 = tc_desc((uint32_t)__cvta_generic_to_shared(s_pk), pk_lbo, 128u);
+    auto issue_round = [&](uint32_t q) -> bool {
+      const uint32_t tq = q / (uint32_t)n_rounds;
+      const int r = (int)(q - tq * (uint32_t)n_rounds);
+      const int us = (int)(tq % kTiles);
+      const uint32_t as = q & 1u;
+      // wait for the tile's operand -- or for the news that the tiles ended before this one
+      {
+        bool ready = false;
+        for (int it = 0; it < kTcWaitLimit && !ready; ++it) {
+          uint32_t done;
+          asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                       : "=r"(done) : "r"(mb_meta + 8 * us), "r"((tq / kTiles) & 1u) : "memory");
+          if (done) ready = true;
+          else if (*s_endtile < tq) return true;
+          else if ((it & 15) == 15 && *s_abort) return false;
         }
-        phase ^= 1u;
-        tc_fence_after();
-        return true;
-      };
+        if (!ready) return false;
+      }
+      if (*reinterpret_cast<volatile uint32_t*>(s_rflags + us * kTcRows) & kRfEnd) return true;
+      if (!mbar_wait(mb_free + 8 * as, ((q >> 1) & 1u) ^ 1u, s_abort)) return false;
+      tc_fence_after();
+      const bool with_delta = combined || r >= R1;
+      const uint64_t da = da0 + (uint64_t)(((uint32_t)us * (kTileHalves * 2)) >> 4);
+      const uint64_t db = db0 + (uint64_t)(((uint32_t)((r % R1) * kTcRound) * 16u) >> 4);
+#pragma unroll
+      for (int acc = 0; acc < 2; ++acc) {
+        if (acc == 1 && !with_delta) continue;
+#pragma unroll
+        for (int ks = 0; ks < 2 * KS; ++ks) {
+          const uint32_t id = (acc == 1 && ks >= KS) ? (kTcIdesc | kTcNegB) : kTcIdesc;
+          tc_mma(tmem + as * 128u + (uint32_t)(acc * 64), da + (uint64_t)((ks * 2u * kTileLbo) >> 4),
+                 db + (uint64_t)((ks * 2u * pk_lbo) >> 4), id, ks > 0);
+        }
+      }
+      tc_commit(mb_done + 8 * as);
+      if (r == n_rounds - 1) tc_commit(mb_tile + 8 * us);
+      return true;
+    };
+    // This warp is through with round q's stage.  The last of the four warps to say so issues round q + 2 into it.
+    auto release_stage = [&](uint32_t q) {
+      const uint32_t as = q & 1u;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(mb_free + 8 * as);
+        const uint32_t old = atomicAdd(&s_relcnt[as], 1u);
+        if ((old & 3u) == 3u && !issue_round(q + 2)) {
+          *s_abort = 1;
+          am_ok(false, 11u, status);
+        }
+      }
+      __syncwarp();
+    };
+    // the first two rounds have nobody to release their stages
+    if (tid == 0) {
+      if (!issue_round(0) || !issue_round(1)) {
+        *s_abort = 1;
+        am_ok(false, 11u, status);
+      }
+    }
+    __syncwarp();
+
+    while (true) {
+      const int us = (int)(t % kTiles);
+      if (!wait_all(mb_meta + 8 * us, (t / kTiles) & 1u)) { bad = true; break; }
+      const uint32_t flags = s_rflags[us * kTcRows + tid];
+      if (flags & kRfEnd) break;                    // every row of the marker carries it
+      const uint32_t pix = s_rpix[us * kTcRows + tid];
+      const float dS = s_rslack[us * kTcRows + tid];
+      const float cS = s_rcs[us * kTcRows + tid], cD = s_rcd[us * kTcRows + tid];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(mb_rows + 8 * us);       // the buffer's row data may be overwritten
+      const bool live = (flags & kRfLive) != 0;
 
       // ---- pass 1: the smallest (and, if the runner-up is wanted, second smallest) S_k of the row
       float s1 = inf, s2 = inf;
-      for (int pc = 0; pc < n_pchunks && !failed; ++pc) {
-        if (n_pchunks > 1) { __syncthreads(); load_peaks(pc); __syncthreads(); }
-        const int kn = min(peak_cap, K - pc * peak_cap);
-        for (int n0 = 0; n0 < kn && !failed; n0 += kTcRound) {
-          if (!run_round(n0, one_round)) { failed = true; break; }
-          for (int c0 = 0; c0 < kTcRound && n0 + c0 < kn; c0 += 32) {
-            float vS[32];
-            tc_ld32(t_row + c0, vS);
-            if constexpr (WANT2) {
+      uint32_t as = 0;
+      for (int r = 0; r < R1; ++r) {
+        as = rc & 1u;
+        if (!wait_all(mb_done + 8 * as, (rc >> 1) & 1u)) { bad = true; break; }
+        tc_fence_after();
+        const int kn = K - r * kTcRound;
+        for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
+          float vS[32];
+          tc_ld32(t_lane + as * 128u + (uint32_t)c0, vS);
+          if constexpr (WANT2) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float v = (vS[j] == vS[j]) ? vS[j] : inf;   // columns beyond the last peak are NaN
-                const float lo = fminf(s1, v), hi = fmaxf(s1, v);
-                s1 = lo;
-                s2 = fminf(s2, hi);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j += 2) s1 = min3f(s1, vS[j], vS[j + 1]);
+            for (int j = 0; j < 32; ++j) {
+              const float v = (vS[j] == vS[j]) ? vS[j] : inf;   // columns beyond the last peak are NaN
+              const float lo = fminf(s1, v), hi = fmaxf(s1, v);
+              s1 = lo;
+              s2 = fminf(s2, hi);
             }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) s1 = min3f(s1, vS[j], vS[j + 1]);
           }
         }
+        if (!combined) {
+          release_stage(rc);
+          ++rc;
+        }
       }
-      if (failed) break;
-      TC_PROF(3);
+      if (bad) break;
       // d_best^2 <= 2 S_true(arg-min) <= 2 (S_lo + 2 dS).  A peak can only win if L_true <= d_best^2, and what pass 2
       // computes, 2 S_lo - |Delta_c|, is at most L_true + dS: the test is 2 S_lo - |Delta_c| <= 2 (S_min + 2 dS) + dS.
       // Rows without a usable pixel get a NaN threshold: no comparison with it is ever true.
-      const float sref = WANT2 ? s2 : s1;
-      const float thr = live ? (2.0f * (sref + 2.0f * dS) * (1.0f + 1e-5f) + 1e-6f) + dS : qnan;
+      // The accumulators hold the dot products alone: S_lo = cS + S_acc, Delta_c = cD + Delta_acc.  The row constant
+      // 2 cS is moved to the other side of the comparison (rounded up).
+      const float sref = (WANT2 ? s2 : s1) + cS;
+      const float thr_full = (2.0f * (sref + 2.0f * dS) * (1.0f + 1e-5f) + 1e-6f) + dS;
+      const float thr = live ? (thr_full - 2.0f * cS) + 1e-5f * (fabsf(thr_full) + 2.0f * cS) : qnan;
 
-      // ---- pass 2: L_k <= thr as a bit mask; the peaks that pass are the row's candidates
-      int cnt = 0, ck0 = -1, ck1 = -1, ck2 = -1, ck3 = -1, ck4 = -1, ck5 = -1;
-      for (int pc = 0; pc < n_pchunks && !failed; ++pc) {
-        if (n_pchunks > 1) { __syncthreads(); load_peaks(pc); __syncthreads(); }
-        const int k0 = pc * peak_cap;
-        const int kn = min(peak_cap, K - k0);
-        for (int n0 = 0; n0 < kn && !failed; n0 += kTcRound) {
-          if (!one_round && !run_round(n0, true)) { failed = true; break; }
-          for (int c0 = 0; c0 < kTcRound && n0 + c0 < kn; c0 += 32) {
-            float vS[32], vD[32];
-            tc_ld32x2(t_row + c0, t_row + 64 + c0, vS, vD);
-            uint32_t mk = 0;
+      // ---- pass 2: L_k <= thr as a bit mask.  A peak that passes gets bounds dlo <= d <= dhi from its S and Delta
+      // (A = (S + Delta) / 2, B = (S - Delta) / 2); the smallest dhi, U, bounds the best distance, and the candidates
+      // are the peaks with dlo <= U.  (The runner-up wanted: the second smallest dhi.)
+      int cnt = 0;                       // candidates appended so far
+      bool lost = false;                 // some candidate has no bounds: keep them all
+      float U1 = inf, U2 = inf;
+      auto append = [&](int k, float dlo) {
+        if (cnt < kTcCand) {
+          s_cand[cnt * kTcRows + tid] = (uint16_t)k;
+          s_clo[cnt * kTcRows + tid] = dlo;
+        }
+        ++cnt;
+      };
+      for (int r = 0; r < R1; ++r) {
+        if (!combined) {
+          as = rc & 1u;
+          if (!wait_all(mb_done + 8 * as, (rc >> 1) & 1u)) { bad = true; break; }
+          tc_fence_after();
+        }
+        const int kn = K - r * kTcRound;
+        for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
+          float vS[32], vD[32];
+          tc_ld32x2(t_lane + as * 128u + (uint32_t)c0, t_lane + as * 128u + 64u + (uint32_t)c0, vS, vD);
+          uint32_t mk = 0, mk2 = 0;     // two chains: the OR into one mask would serialise the loop
+          float xs = 0.0f, xd = 0.0f;   // S and Delta of the last column that passed
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (fmaf(2.0f, vS[j], -fabsf(vD[j])) <= thr) mk |= 1u << j;
-            const int rem = kn - (n0 + c0);
-            if (rem < 32) mk &= (1u << rem) - 1u;
-            if (mk) {
-              const int kbase = k0 + n0 + c0;
-              n_pairs += (uint32_t)__popc(mk);
+          for (int j = 0; j < 32; j += 2) {
+            const float d0 = vD[j] + cD, d1 = vD[j + 1] + cD;
+            if (fmaf(2.0f, vS[j], -fabsf(d0)) <= thr) { mk |= 1u << j; xs = vS[j]; xd = d0; }
+            if (fmaf(2.0f, vS[j + 1], -fabsf(d1)) <= thr) { mk2 |= 1u << (j + 1); xs = vS[j + 1]; xd = d1; }
+          }
+          mk |= mk2;
+          const int rem = kn - c0;
+          if (rem < 32) mk &= (1u << rem) - 1u;
+          if (mk) {
+            const int kbase = r * kTcRound + c0;
+            n_pairs += (uint32_t)__popc(mk);
+            if ((mk & (mk - 1)) == 0) {
+              // the only one of these 32 columns: its S and Delta are at hand
+              const float Slo = cS + xs;
+              const float e = dS + 4e-6f * (fabsf(Slo) + fabsf(xd));           // |S - S_lo - e| <= e, |Delta - xd| <= e
+              const float a_lo = 0.5f * (Slo + xd - e), b_lo = 0.5f * (Slo - xd - e);
+              const float dlo = (__fsqrt_rn(fmaxf(a_lo, 0.0f)) + __fsqrt_rn(fmaxf(b_lo, 0.0f))) * (1.0f - 2e-6f);
+              const float dhi = (__fsqrt_rn(fmaxf(a_lo + 2.0f * e, 0.0f)) + __fsqrt_rn(fmaxf(b_lo + 2.0f * e, 0.0f))) * (1.0f + 2e-6f);
+              if (dhi < U1) { U2 = U1; U1 = dhi; }
+              else if (dhi < U2) { U2 = dhi; }
+              const float Uref = WANT2 ? U2 : U1;
+              if (dlo <= Uref * (1.0f + 4e-5f) + 1e-6f) append(kbase + __ffs(mk) - 1, dlo);
+            } else {
+              // several in one block of columns: kept without bounds
+              lost = true;
               while (mk) {
-                const int k = kbase + __ffs(mk) - 1;
+                append(kbase + __ffs(mk) - 1, 0.0f);
                 mk &= mk - 1;
-                if (cnt == 0) ck0 = k;
-                else if (cnt == 1) ck1 = k;
-                else if (cnt == 2) ck2 = k;
-                else if (cnt == 3) ck3 = k;
-                else if (cnt == 4) ck4 = k;
-                else if (cnt == 5) ck5 = k;
-                ++cnt;
               }
             }
           }
         }
+        release_stage(rc);
+        ++rc;
       }
-      if (failed) break;
+      if (bad) break;
+      // what is left of the list once U is final (the order, ascending k, is kept)
+      if (cnt <= kTcCand) {
+        const float Uref = WANT2 ? U2 : U1;
+        const float Um = Uref * (1.0f + 4e-5f) + 1e-6f;
+        int kept = 0;
+        for (int i = 0; i < cnt; ++i) {
+          const float dlo = s_clo[i * kTcRows + tid];
+          const uint16_t k = s_cand[i * kTcRows + tid];
+          if (lost || dlo <= Um) {
+            s_cand[kept * kTcRows + tid] = k;
+            ++kept;
+          }
+        }
+        cnt = kept;
+      }
+      if (bad) break;
       if (live) am_ok(cnt > 0, 9u, status);                 // the arg-min always passes
-      TC_PROF(4);
 
       // ---- the row's outcome: decided here, or queued for the scoring step
-      if (valid && cnt > kTcCand) hard = true;
-      if (present) {
-        const uint32_t pix = (uint32_t)(span0 + off);
-        int want_score = 0;                                 // (kept as separate statements)
-        if (live && score_all) want_score = 1;
-        if (live && cnt > 1) want_score = 1;
-        if (hard) {
-          const uint32_t hp = atomicAdd(s_qn + 1, 1u);
-          if (am_ok(hp < (uint32_t)kTcHardQueue, 2u, status)) s_hardq[hp] = pix;
-        } else if (want_score) {
-          const uint32_t pos = atomicAdd(s_qn, (uint32_t)(1 + cnt));
-          if (am_ok(pos + (uint32_t)cnt < (uint32_t)kTcQueue, 3u, status)) {
-            const unsigned long long hi = (unsigned long long)pix << 32;
-            s_queue[pos] = hi | kTcHeader | (uint32_t)cnt;
-            s_queue[pos + 1] = hi | (uint32_t)ck0;
-            if (cnt > 1) s_queue[pos + 2] = hi | (uint32_t)ck1;
-            if (cnt > 2) s_queue[pos + 3] = hi | (uint32_t)ck2;
-            if (cnt > 3) s_queue[pos + 4] = hi | (uint32_t)ck3;
-            if (cnt > 4) s_queue[pos + 5] = hi | (uint32_t)ck4;
-            if (cnt > 5) s_queue[pos + 6] = hi | (uint32_t)ck5;
-            if (cnt > 1) ++n_rescored;
-          }
-        } else if (valid && cnt == 1) {
-          s_lab[off] = ck0 + 1;                            // decided by the filter alone (tau = +inf, no scores)
-        } else if (best_img) {
-          best_img[pix] = inf;                             // a pixel that takes no part (non-finite)
+      int hard = (flags & kRfHard) ? 1 : 0;
+      if (live && cnt > kTcCand) hard = 1;
+      int want = 0;                                         // (kept as separate statements)
+      if (live && score_all) want = 1;
+      if (live && cnt > 1) want = 1;
+      if (hard) want = 0;
+      if (flags & kRfGroup) {
+        // 8 lanes = the 8 pixels of a group: a full 32-byte sector.  Queued rows get their label when they are scored.
+        int label = 0;
+        if (live && !want && !hard && cnt == 1) label = (int)s_cand[tid] + 1;   // decided by the filter alone (tau = +inf, no scores)
+        lab_img[pix] = label;
+        if (best_img && !want && !hard) {
+          best_img[pix] = inf;                              // a pixel that takes no part
           second_img[pix] = inf;
         }
       }
-      TC_PROF(5);
+      {
+        // queue slots: the few lanes that queue take them with an atomic on the warp's counter (the order of the
+        // rows within the queue does not matter)
+        const int need = want ? 1 + cnt : 0;
+        if (want) {
+          const int pos = atomicAdd(&s_qfill[wid], need);
+          if (am_ok(pos >= 0 && pos + cnt < kTcQueue, 3u, status)) {
+            const unsigned long long hi = (unsigned long long)pix << 32;
+            Qw[pos] = hi | kTcHeader | (uint32_t)cnt;
+            for (int i = 0; i < cnt; ++i) Qw[pos + 1 + i] = hi | (uint32_t)s_cand[i * kTcRows + tid];
+            if (cnt > 1) ++n_rescored;
+          }
+        }
+        __syncwarp();
+        qn = *reinterpret_cast<volatile int*>(&s_qfill[wid]);
+        const uint32_t hm = __ballot_sync(0xffffffffu, hard != 0);
+        if (hard) {
+          const int hp = nh + __popc(hm & ((1u << lane) - 1u));
+          if (am_ok(hp < kTcHardQueue, 2u, status)) Hw[hp] = pix;
+        }
+        nh += __popc(hm);
+        if (qn > kTcFlushAt || nh > kTcHardFlushAt) {
+          tc_flush_warp<T, KA>(sc, Qw, min(qn, kTcQueue), Hw, min(nh, kTcHardQueue), 0, 1, rejected, n_full);
+          qn = 0;
+          nh = 0;
+          if (lane == 0) s_qfill[wid] = 0;
+          __syncwarp();
+        }
+      }
+      ++t;
     }
-    if (failed) break;
-    __syncthreads();
-    TC_PROF(6);
-    // ---- label map of the span: every pixel written, 128-bit stores when the span is aligned
-    if ((span_len & 3) == 0 && ((uintptr_t)(lab_img + span0) & 15u) == 0) {
-      for (int i = tid; i < span_len / 4; i += kTcThreads)
-        reinterpret_cast<int4*>(lab_img + span0)[i] = reinterpret_cast<const int4*>(s_lab)[i];
-    } else {
-      for (int i = tid; i < span_len; i += kTcThreads) lab_img[span0 + i] = s_lab[i];
+    if (bad) {
+      *s_abort = 1;
+      am_ok(false, 10u, status);
     }
-    __syncthreads();
-    TC_PROF(7);
+    __syncwarp();
+    if (lane == 0) {
+      s_qfill[wid] = min(qn, kTcQueue);
+      s_qfill[4 + wid] = min(nh, kTcHardQueue);
+    }
   }
 
-  // ---- what is still queued (every span's label map has been stored)
-  __syncthreads();
-  if (!failed) tc_flush<T, KA>(sc, -1, 0, rejected, n_full);
-
-  // ---- tear-down: no copy in flight, tensor memory returned
-  asm volatile("cp.async.wait_all;\n" ::: "memory");
+  // ---- every role is through: what is still queued is scored by all warps, two per queue
   tc_fence_before();
+  __syncthreads();
+  if (!*s_abort) {
+    const int q = wid & 3, part = wid >> 2;
+    tc_flush_warp<T, KA>(sc, s_queue + (size_t)q * kTcQueue, s_qfill[q], s_hardq + (size_t)q * kTcHardQueue, s_qfill[4 + q],
+                         part, 2, rejected, n_full);
+  }
+  // ---- tear-down: tensor memory returned
   __syncthreads();
   if (wid == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcCols) : "memory");
 
@@ -804,6 +1023,31 @@ assign_tc_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     if (wp) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_FILTER_PAIRS], wp);
     if (ws) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_RESCORED], ws);
     if (wf) atomicAdd(&counters[b * CPE_CNT_N + CPE_CNT_FULL_SCORED], wf);
+  }
+}
+
+// One launch for every image that the all-pairs kernel leaves alone: the tcgen05 pipeline where the peaks fit one
+// round (there it is the faster one), the mma.sync kernel for more peaks.  The number of peaks is only known on the
+// device, so the choice is made here, per image.
+template <typename T, int KA, bool WANT2>
+__global__ void __launch_bounds__(kTcThreads, 2)
+assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int K_max,
+                     const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
+                     int tc_peak_cap, int tc_k_max, int tc_vec_mask, int mma_peak_cap, int mma_span, int mma_vec_mask,
+                     int mma_vec_gather, int32_t* __restrict__ labels, float* __restrict__ best, float* __restrict__ second,
+                     uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all, uint32_t* __restrict__ votes, int cells,
+                     int k_min, uint32_t* __restrict__ acc) {
+  static_assert(kTcThreads == kAmThreads, "both bodies run with the same block size");
+  if (count_ptr[blockIdx.y] <= tc_k_max)
+    assign_tc_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, tc_peak_cap, tc_vec_mask, labels,
+                                 best, second, counters, status_all, votes, cells, k_min, tc_k_max, acc);
+  else {
+    // This kernel is one that uses tensor memory: a CTA that takes the other path gives up its right to allocate at
+    // once, or the SM would not take a second CTA while this one runs.
+    if (threadIdx.x < 32) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    assign_mma_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, mma_peak_cap, mma_span,
+                                  mma_vec_mask, mma_vec_gather, labels, best, second, counters, status_all, votes, cells,
+                                  tc_k_max + 1);
   }
 }
 

@@ -162,35 +162,45 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   return CPE_OK;
 }
 
-// Blackwell tensor-core path (tcgen05, accumulators in tensor memory); needs 16-byte aligned planes.
+// The filtered assignment for 16-byte aligned planes: one launch, the tcgen05 pipeline for the images whose peaks
+// fit one of its rounds, the mma.sync body for the others (the choice is made on the device, per image).
 template <typename T, int KA, bool WANT2>
-int launch_assign_tc_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                       const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                       uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min) {
-  // small inputs get short spans so that there are enough CTAs to fill the GPU
-  const int span = ((long long)B * HW >= (1 << 20)) ? 2048 : 512;
-  const int two_tiles = (sizeof(T) == 2 && KA == 16) ? 1 : 0;
-  // as many peaks resident in shared memory as leave room for two CTAs per SM
-  int peak_cap = (p->max_instances + cpe::kTcRound - 1) / cpe::kTcRound * cpe::kTcRound;
-  const int budget = 110 * 1024;
-  const int fixed = cpe::tc_smem_layout(KA, 0, span, two_tiles).total;
-  peak_cap = std::max(cpe::kTcRound, std::min(peak_cap, (budget - fixed) / (2 * KA * 2) / cpe::kTcRound * cpe::kTcRound));
-  // never more than two CTAs per SM: each holds half of the SM's tensor memory
-  const int smem = std::max(cpe::tc_smem_layout(KA, peak_cap, span, two_tiles).total, 78 * 1024);
-  auto kern = cpe::assign_tc_kernel<T, KA, WANT2>;
+int launch_assign_filter_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                           const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
+                           uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min, uint32_t* acc) {
+  // tcgen05 body: as many peaks resident in shared memory as leave room for two CTAs per SM (each CTA holds half of
+  // the SM's tensor memory, so there must never be more than two)
+  const int budget = 104 * 1024;
+  int tc_cap = (p->max_instances + cpe::kTcRound - 1) / cpe::kTcRound * cpe::kTcRound;
+  const int tc_fixed = cpe::tc_smem_layout(KA, 0).total;
+  tc_cap = std::max(cpe::kTcRound, std::min(tc_cap, (budget - tc_fixed) / (2 * KA * 2) / cpe::kTcRound * cpe::kTcRound));
+  // beyond one round the mma.sync body is the faster one (CPE_ASSIGN_PATH=tc lifts the limit: tests, comparisons)
+  static const char* path = getenv("CPE_ASSIGN_PATH");
+  const int tc_k_max = (path && strcmp(path, "tc") == 0) ? tc_cap : std::min(tc_cap, cpe::kTcRound);
+  const int tc_smem = cpe::tc_smem_layout(KA, tc_cap).total;
+  // mma.sync body
+  const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
+  const int vec_gather = span == cpe::kAmSpanMax ? 1 : 0;
+  const int two_tiles = (vec_gather && sizeof(T) == 2 && KA == 16) ? 1 : 0;
+  int mma_cap = (p->max_instances + 7) & ~7;
+  const int mma_fixed = cpe::am_smem_layout(KA, 0, span, two_tiles).total;
+  mma_cap = std::max(8, std::min(mma_cap, ((110 * 1024 - mma_fixed) / ((2 * KA + 8) * 2)) & ~7));
+  const int mma_smem = cpe::am_smem_layout(KA, mma_cap, span, two_tiles).total;
+  const int smem = std::max(std::max(tc_smem, mma_smem), 78 * 1024);
+  auto kern = cpe::assign_filter_kernel<T, KA, WANT2>;
   static bool configured = false;   // per instantiation; the attribute is sticky for the process
   if (!configured) {
     CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
     configured = true;
   }
-  const int n_spans = (HW + span - 1) / span;
+  const int n_spans = (HW + cpe::kTcSpan - 1) / cpe::kTcSpan;
   const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
   dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
   const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
   const int need_exact = p->tau < INFINITY ? 1 : 0;
-  kern<<<grid, cpe::kTcThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact, peak_cap,
-                                            span, vec_mask, labels, best, second, counters, status, votes_to_zero, cells,
-                                            k_min);
+  kern<<<grid, cpe::kTcThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact, tc_cap, tc_k_max,
+                                            vec_mask, mma_cap, span, vec_mask, vec_gather, labels, best, second, counters,
+                                            status, votes_to_zero, cells, k_min, acc);
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -198,7 +208,7 @@ int launch_assign_tc_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, in
 template <typename T>
 int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                   const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                  uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells) {
+                  uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, uint32_t* acc) {
   if (p->flags & CPE_FLAG_EXACT_ASSIGN)
     return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
                                   votes_to_zero, cells, 0x7fffffff);
@@ -212,22 +222,19 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   const T* e = static_cast<const T*>(emb);
   const bool want2 = best != nullptr;
   const int k_min = k_limit + 1;
-  // CPE_ASSIGN_PATH=mma keeps the mma.sync kernel, =tc takes the tcgen05 kernel wherever it can run (comparisons);
-  // by default the tcgen05 kernel serves F > 8, where it is the faster one
+  // CPE_ASSIGN_PATH=mma in the environment keeps the mma.sync kernel everywhere (comparisons)
   static const char* path = getenv("CPE_ASSIGN_PATH");
-  const bool tc_ok = (uintptr_t)e % 16 == 0 && HW % 8 == 0;
-  const bool use_tc = tc_ok && (path ? strcmp(path, "tc") == 0 : F > 8);
-  if (use_tc) {
-    if (F <= 8) {
-      return want2 ? launch_assign_tc_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
-                                                     status, votes_to_zero, cells, k_min)
-                   : launch_assign_tc_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                      counters, status, votes_to_zero, cells, k_min);
-    }
-    return want2 ? launch_assign_tc_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
-                                                   status, votes_to_zero, cells, k_min)
-                 : launch_assign_tc_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                    counters, status, votes_to_zero, cells, k_min);
+  const bool aligned = (uintptr_t)e % 16 == 0 && HW % 8 == 0;
+  if (aligned && !(path && strcmp(path, "mma") == 0)) {
+    if (F <= 8)
+      return want2 ? launch_assign_filter_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                         counters, status, votes_to_zero, cells, k_min, acc)
+                   : launch_assign_filter_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                          counters, status, votes_to_zero, cells, k_min, acc);
+    return want2 ? launch_assign_filter_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                       counters, status, votes_to_zero, cells, k_min, acc)
+                 : launch_assign_filter_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
+                                                        counters, status, votes_to_zero, cells, k_min, acc);
   }
   if (F <= 8) {
     return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
@@ -311,9 +318,9 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_ASSIGN], st));
   uint32_t* votes_to_zero = keep_votes ? nullptr : votes;
   rc = p->dtype == CPE_F32 ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second,
-                                                  counters, status, votes_to_zero, L.cells)
+                                                  counters, status, votes_to_zero, L.cells, acc)
                            : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best,
-                                                   second, counters, status, votes_to_zero, L.cells);
+                                                   second, counters, status, votes_to_zero, L.cells, acc);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "assign"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
@@ -681,14 +688,3 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   p.workspace_bytes = CPE_STATIC_SCRATCH_BYTES;
   return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
 }
-
-#ifdef CPE_TC_PROF
-extern "C" int cpe_tc_prof_read(unsigned long long* out16, int reset) {
-  if (cudaMemcpyFromSymbol(out16, cpe::g_tc_prof, 16 * sizeof(unsigned long long)) != cudaSuccess) return -1;
-  if (reset) {
-    unsigned long long z[16] = {0};
-    if (cudaMemcpyToSymbol(cpe::g_tc_prof, z, sizeof(z)) != cudaSuccess) return -1;
-  }
-  return 0;
-}
-#endif

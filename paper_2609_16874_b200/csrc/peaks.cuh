@@ -124,6 +124,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     acc[b * kAccStride + kAccVoting] = 0u;
     acc[b * kAccStride + kAccNonfinite] = 0u;
     acc[b * kAccStride + kAccTicket] = 0u;
+    acc[b * kAccStride + kAccSpan] = 0u;
     uint32_t* cnt = counters + b * CPE_CNT_N;
     cnt[CPE_CNT_VOTING] = voting;
     cnt[CPE_CNT_NONFINITE] = nonfinite;
