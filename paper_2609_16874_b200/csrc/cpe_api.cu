@@ -95,12 +95,27 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
   return CPE_OK;
 }
 
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 template <typename T>
 int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                         const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
                         uint32_t* counters, uint32_t* votes_to_zero, int cells, int k_limit) {
   const T* e = static_cast<const T*>(emb);
-  dim3 grid((unsigned)(((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads), (unsigned)B);
+  // eight CTAs of 128 threads per SM, shared among the images, walk the pixel blocks
+  const long long n_blocks = ((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads;
+  const long long per_image = std::max(1, (8 * sm_count() + B - 1) / B);
+  dim3 grid((unsigned)std::min(n_blocks, per_image), (unsigned)B);
 #define CPE_LAUNCH_ASSIGN(FT_)                                                                                  \
   cpe::assign_kernel<T, FT_><<<grid, cpe::kAssignThreads, 0, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, \
                                                                   p->tau, labels, best, second, counters, votes_to_zero, cells, \
@@ -116,17 +131,6 @@ int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int
   return CPE_OK;
 }
 
-int sm_count() {
-  static int cached[64] = {0};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (!cached[dev]) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
 
 template <typename T, int KA, bool WANT2>
 int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
