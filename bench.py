@@ -43,10 +43,10 @@ FALLBACK_HBM_GBS = 6650.0
 # (smsp__inst_executed.sum), which is what an instruction-bound kernel is measured against.
 NCU = {
     # (workload, stage): {"traffic": bytes, "warp_inst": count, "kernel": name}
-    ("c2", "assign"): {"traffic": 22036480, "warp_inst": 14519639, "kernel": "assign_kernel<float,8>"},
-    ("c2", "decode_vote"): {"traffic": 22059264, "warp_inst": 4131965, "kernel": "decode_vote_vec_kernel<float,8>"},
-    ("c3", "assign"): {"traffic": 88034304, "warp_inst": 69783301, "kernel": "assign_mma_kernel<__half,16,false>"},
-    ("c3", "decode_vote"): {"traffic": 86884608, "warp_inst": 26566909, "kernel": "decode_vote_vec_kernel<__half,8>"},
+    ("c2", "assign"): {"traffic": 22046464, "warp_inst": 10145531, "kernel": "assign_kernel<float,8>"},
+    ("c2", "decode_vote"): {"traffic": 22059520, "warp_inst": 4131965, "kernel": "decode_vote_vec_kernel<float,8>"},
+    ("c3", "assign"): {"traffic": 95789568, "warp_inst": 46424257, "kernel": "assign_filter_kernel<__half,16,false>"},
+    ("c3", "decode_vote"): {"traffic": 89585408, "warp_inst": 26567474, "kernel": "decode_vote_vec_kernel<__half,8>"},
 }
 # Ceiling for instruction-bound kernels: 148 SMs x 4 schedulers x 1 warp instruction per clock x 1.965 GHz.
 ALU_PEAK_GWARPINST = 148 * 4 * 1.965
@@ -368,7 +368,7 @@ def run_ours(args, cfg):
             "workload": cfg.describe(), "name": cfg.name, "frames_per_rank": n_frames,
             "l2": ("inputs rotate over %d frames, %.0f MB > L2" % (n_frames, n_frames * cfg.emb_bytes / 1e6)
                    if flush is None else "a 252 MB buffer is rewritten between steps, outside the timed events"),
-            "launch": "one CUDA graph replay per step (%d kernels + 1 memset node)" % kernel_nodes,
+            "launch": "one CUDA graph replay per step (%d kernel nodes, no memset)" % kernel_nodes,
             "timing": "sum of per-step CUDA-event times on the launching stream; span of the region %.3f ms" % span_ms,
             "parallelism": "independent frames per rank, no collective",
             "instances_found_last_step": count_last.tolist(),
