@@ -71,6 +71,8 @@ def _load():
         lib.cpe_oracle_assign_image.restype = c_int
         lib.cpe_oracle_decode.argtypes = ([vp, vp] + [c_int] * 9 + [c_dbl, c_int] + [vp] * 9)
         lib.cpe_oracle_decode.restype = c_int
+        lib.cpe_oracle_soft_votes.argtypes = [vp, c_int, vp] + [c_int] * 6 + [vp, c_int, vp]
+        lib.cpe_oracle_soft_votes.restype = c_int
         _lib = lib
     return _lib
 
@@ -225,3 +227,24 @@ def decode(emb: np.ndarray, fg, bins_w: int, bins_h: int, T_v: int = 8, tau=np.i
         raise RuntimeError(f"cpe_oracle_decode failed: {rc}")
     return {"labels": labels, "centroids": centroids, "count": count, "votes": V, "peak_cell": pc,
             "peak_votes": pv, "best": best, "second": second, "counters": counters}
+
+
+def soft_votes(emb: np.ndarray, fg, bins_w: int, bins_h: int, sample_cells=None) -> np.ndarray:
+    """The soft-vote histogram of Eq. 6 in binary64: ``[B, bins_h, bins_w]``, or ``[B, n]`` for the ``n`` linear cells
+    ``b * bins_w + a`` listed in ``sample_cells``."""
+    emb = np.ascontiguousarray(emb)
+    B, D, H, W = emb.shape
+    F = D // 4
+    fgc = None if fg is None else np.ascontiguousarray(fg, np.uint8)
+    if sample_cells is None:
+        cells, n = None, 0
+        out = np.empty((B, bins_h, bins_w), np.float64)
+    else:
+        cells = np.ascontiguousarray(sample_cells, np.int32)
+        n = int(cells.size)
+        out = np.empty((B, n), np.float64)
+    rc = _load().cpe_oracle_soft_votes(_ptr(emb), _dtype_code(emb), _ptr(fgc), B, H, W, F, bins_w, bins_h, _ptr(cells), n,
+                                       _ptr(out))
+    if rc:
+        raise RuntimeError(f"cpe_oracle_soft_votes failed: {rc}")
+    return out

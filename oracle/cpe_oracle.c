@@ -14,6 +14,8 @@
  *   - local maxima: strict maximum in the 8-connected neighbourhood
  *     above a threshold                                                 Sec. 3.2, "Local Maxima Search"
  *   - assignment m = argmin_k d(a_k, b_k), kept iff d < tau             Eq. 7, Eq. 8
+ *   - soft-vote histogram H(a,b) = sum_ij exp(-d_ij(a,b))               Eq. 5, Eq. 6 (cpe_oracle_soft_votes; a second
+ *     vote mode next to the hard vote, the plain definition in binary64)
  *   - the HARD vote (one integer vote per pixel into the nearest Eq. 9 bin of a per-pixel
  *     centroid estimate) replaces the soft vote of Eq. 5-6.  The paper does not define a
  *     per-pixel estimate; the one used here is coarse-to-fine phase unwrapping of the
@@ -351,6 +353,59 @@ int cpe_oracle_assign_image(const void* emb_img, int dtype, const uint8_t* fg_im
 }
 
 /* ------------------------------------------------------------- the whole chain ---- */
+
+/* ------------------------------------------- Eq. 4-6: the soft-vote histogram (binary64) ---- */
+
+/*
+ * The paper's coarse voting histogram, written out as printed: every participating pixel (i, j) adds the weight
+ *     w_ij(a, b) = exp(-(||xhat(i,j) - P_w[a]|| + ||yhat(i,j) - P_h[b]||))          Eq. 4, Eq. 5
+ * to bin (a, b):  H(a, b) = sum over the participating pixels of w_ij(a, b).          Eq. 6
+ * (Eq. 10-11 factorise the same sum as E_x^T E_y; this is the unfactorised definition.)  Euclidean norms, not
+ * squared.  A pixel takes part iff its mask byte is non-zero (all pixels if fg is NULL) and all its channels are
+ * finite -- the same participating set as the hard vote.  Palette rows are the binary32 tables of Eq. 9.
+ * out: [B][bins_h][bins_w] doubles, or, with n_sample > 0, [B][n_sample] for the linear cells b*bins_w + a listed
+ * in sample_cells (so that a few bins of a large problem can be checked).
+ */
+int cpe_oracle_soft_votes(const void* emb, int dtype, const uint8_t* fg, int B, int H, int W, int F, int bins_w,
+                          int bins_h, const int32_t* sample_cells, int n_sample, double* out) {
+  if (!emb || !out || B < 1 || H < 1 || W < 1 || F < 1 || bins_w < 1 || bins_h < 1) return -1;
+  float* Pw = (float*)malloc(sizeof(float) * (size_t)bins_w * 2 * F);
+  float* Ph = (float*)malloc(sizeof(float) * (size_t)bins_h * 2 * F);
+  if (!Pw || !Ph) { free(Pw); free(Ph); return -2; }
+  cpe_oracle_palette(bins_w, F, Pw);
+  cpe_oracle_palette(bins_h, F, Ph);
+  const size_t HW = (size_t)H * W;
+  const int n_cells = n_sample > 0 ? n_sample : bins_w * bins_h;
+  for (int b = 0; b < B; ++b) {
+    const size_t base = (size_t)b * 4 * F * HW;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(g_threads)
+    for (int ci = 0; ci < n_cells; ++ci) {
+      const int lin = n_sample > 0 ? sample_cells[ci] : ci;
+      const int a = lin % bins_w, bb = lin / bins_w;
+      double sum = 0.0;
+      for (size_t p = 0; p < HW; ++p) {
+        if (fg && !fg[(size_t)b * HW + p]) continue;
+        int finite = 1;
+        for (int l = 0; l < 2 * F && finite; ++l)
+          finite = pair_is_finite(load_elem(emb, dtype, base + (size_t)(2 * l) * HW + p),
+                                  load_elem(emb, dtype, base + (size_t)(2 * l + 1) * HW + p));
+        if (!finite) continue;
+        double sx = 0.0, sy = 0.0;
+        for (int c = 0; c < 2 * F; ++c) {
+          const double tx = (double)load_elem(emb, dtype, base + (size_t)c * HW + p) - (double)Pw[(size_t)a * 2 * F + c];
+          const double ty = (double)load_elem(emb, dtype, base + (size_t)(2 * F + c) * HW + p) - (double)Ph[(size_t)bb * 2 * F + c];
+          sx += tx * tx;
+          sy += ty * ty;
+        }
+        sum += exp(-(sqrt(sx) + sqrt(sy)));
+      }
+      out[(size_t)b * n_cells + ci] = sum;
+    }
+  }
+  free(Pw);
+  free(Ph);
+  return 0;
+}
 
 /*
  * Same argument order as the library's decode entry point, host pointers, plus the intermediates.

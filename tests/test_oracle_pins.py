@@ -515,3 +515,75 @@ def test_hard_vote_peak_equals_soft_vote_argmax_on_alias_free_grid():
     direct = np.exp(-(dy[:, None, :] + dx[None, :, :])).sum(2)           # Eq. 6
     np.testing.assert_allclose(Hsoft, direct, rtol=1e-12)
     assert int(np.argmax(Hsoft)) == int(res["peak_cell"][0, 0])
+
+
+# ---------------------------------------------------------------- soft-vote histogram (Eq. 4-6)
+
+def _gamma(p, F):
+    """Eq. 2 in binary64: (sin, cos) of pi 2^l p, l = 0..F-1, interleaved."""
+    out = np.empty(2 * F)
+    for l in range(F):
+        out[2 * l] = np.sin(np.pi * 2.0 ** l * p)
+        out[2 * l + 1] = np.cos(np.pi * 2.0 ** l * p)
+    return out
+
+
+def test_soft_votes_of_one_clean_pixel_follow_the_chord_length_formula():
+    """One pixel that encodes (px, py) exactly: ||gamma(p) - gamma(q)||^2 = sum_l (2 - 2 cos(pi 2^l (p - q))), so every
+    bin's weight has a closed form that never forms a difference of embeddings (Eq. 2, Eq. 4, Eq. 5)."""
+    F, bw, bh = 5, 13, 9
+    px, py = 0.3127, -0.6421
+    emb = np.zeros((1, 4 * F, 1, 1), np.float64)
+    emb[0, :2 * F, 0, 0] = _gamma(px, F)
+    emb[0, 2 * F:, 0, 0] = _gamma(py, F)
+    H = oracle.soft_votes(emb.astype(np.float32), None, bw, bh)[0]
+    def chord(p, q):
+        return np.sqrt(sum(2.0 - 2.0 * np.cos(np.pi * 2.0 ** l * (p - q)) for l in range(F)))
+    for b in range(bh):
+        for a in range(bw):
+            qa, qb = -1 + 2 * (a + 1) / (bw + 1), -1 + 2 * (b + 1) / (bh + 1)
+            want = np.exp(-(chord(px, qa) + chord(py, qb)))
+            assert abs(H[b, a] - want) <= 2e-6 * want + 1e-12, (a, b, H[b, a], want)   # binary32 inputs and palette
+
+
+def test_soft_votes_match_a_numpy_restatement_and_factorise():
+    """Tiny random input: the histogram equals the sum over pixels of the outer product of the two weight vectors
+    (Eq. 10-11), computed here with numpy norms and einsum from the oracle-independent Eq. 9 positions."""
+    rng = np.random.default_rng(7)
+    F, bw, bh, B, Hh, Ww = 3, 6, 5, 2, 4, 7
+    emb = rng.standard_normal((B, 4 * F, Hh, Ww)).astype(np.float32)
+    fg = (rng.random((B, Hh, Ww)) < 0.7).astype(np.uint8)
+    Pw = np.stack([_gamma(-1 + 2 * (i + 1) / (bw + 1), F) for i in range(bw)]).astype(np.float32).astype(np.float64)
+    Ph = np.stack([_gamma(-1 + 2 * (i + 1) / (bh + 1), F) for i in range(bh)]).astype(np.float32).astype(np.float64)
+    got = oracle.soft_votes(emb, fg, bw, bh)
+    for b in range(B):
+        x = emb[b, :2 * F].reshape(2 * F, -1).T.astype(np.float64)
+        y = emb[b, 2 * F:].reshape(2 * F, -1).T.astype(np.float64)
+        keep = fg[b].ravel() != 0
+        Ex = np.exp(-np.linalg.norm(x[keep, None, :] - Pw[None], axis=2))
+        Ey = np.exp(-np.linalg.norm(y[keep, None, :] - Ph[None], axis=2))
+        want = np.einsum("pb,pa->ba", Ey, Ex)
+        assert np.allclose(got[b], want, rtol=1e-12, atol=0)
+        assert np.isclose(got[b].sum(), (Ex.sum(1) * Ey.sum(1)).sum(), rtol=1e-12)   # separability of the total
+
+
+def test_soft_votes_skip_masked_and_nonfinite_pixels_and_sampled_cells_agree():
+    rng = np.random.default_rng(11)
+    F, bw, bh = 2, 5, 4
+    emb = rng.standard_normal((1, 4 * F, 3, 8)).astype(np.float32)
+    fg = np.ones((1, 3, 8), np.uint8)
+    full = oracle.soft_votes(emb, fg, bw, bh)
+    # masking a pixel removes exactly its own contribution
+    fg2 = fg.copy(); fg2[0, 1, 3] = 0
+    one = np.zeros_like(emb[:, :, :1, :1]); one[...] = emb[:, :, 1:2, 3:4]
+    assert np.allclose(full - oracle.soft_votes(emb, fg2, bw, bh), oracle.soft_votes(one, None, bw, bh), rtol=1e-9, atol=1e-15)
+    # a pixel with a non-finite channel does not take part
+    bad = emb.copy(); bad[0, 5, 1, 3] = np.inf
+    assert np.allclose(oracle.soft_votes(bad, fg, bw, bh), oracle.soft_votes(emb, fg2, bw, bh), rtol=1e-12, atol=0)
+    # fg = None means every pixel
+    assert np.array_equal(oracle.soft_votes(emb, None, bw, bh), full)
+    cells = np.array([0, 7, bw * bh - 1, 11], np.int32)
+    assert np.array_equal(oracle.soft_votes(emb, fg, bw, bh, sample_cells=cells)[0], full[0].ravel()[cells])
+    # binary16 inputs are widened exactly
+    h = emb.astype(np.float16)
+    assert np.array_equal(oracle.soft_votes(h, fg, bw, bh), oracle.soft_votes(h.astype(np.float32), fg, bw, bh))
