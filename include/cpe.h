@@ -251,6 +251,22 @@ void cpe_host_ctx_destroy(cpe_host_ctx* ctx);
 int cpe_decode_static(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
                       const cpe_params* params, int32_t* out_labels, float* out_centroids, int32_t* out_count);
 
+/*
+ * Second vote mode: the paper's soft-vote histogram (Eq. 4, Eq. 5, Eq. 6),
+ *     H(a, b) = sum over the participating pixels (i, j) of exp(-(||xhat(i,j) - P_w[a]|| + ||yhat(i,j) - P_h[b]||)),
+ * computed in the factorised form H = E_x^T E_y of Eq. 10-11, with E_x and E_y formed tile by tile on the SM and
+ * never stored (the paper materialises both and calls a library GEMM).  Same inputs, layout, participating set
+ * (mask byte non-zero, all channels finite) and palettes (set up by cpe_init_workspace in params->workspace) as
+ * cpe_decode.  out_hist: device memory, float [B][bins_h][bins_w], written completely (zeroed first, then
+ * accumulated: the reduction over pixel tiles uses binary32 atomics, so the last bits depend on the schedule).
+ * Accuracy: |H - H_exact| <= 2e-3 H per bin (binary16 rounding of the two weights that meet in the second
+ * contraction).  Enqueues on the stream, capturable, no host synchronisation.
+ * Errors: as cpe_decode; CPE_ERR_ALIGN also if emb is not 16-byte aligned or H*W is not a multiple of 8 (this
+ * entry point has the vectorised path only).
+ */
+int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                   const cpe_params* params, float* out_hist);
+
 #ifdef __cplusplus
 }
 #endif

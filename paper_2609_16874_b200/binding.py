@@ -38,7 +38,7 @@ EXPORTS = (
     "cpe_workspace_size", "cpe_init_workspace", "cpe_decode", "cpe_get_intermediate", "cpe_strerror",
     "cpe_last_cuda_error", "cpe_graph_create", "cpe_graph_launch", "cpe_graph_destroy", "cpe_graph_kernel_nodes",
     "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
-    "cpe_decode_static",
+    "cpe_decode_static", "cpe_soft_votes",
 )
 
 
@@ -121,6 +121,8 @@ def load() -> ctypes.CDLL:
     lib.cpe_host_ctx_destroy.restype = None
     lib.cpe_decode_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, pp, vp, vp, vp]
     lib.cpe_decode_static.restype = ci
+    lib.cpe_soft_votes.argtypes = [vp, vp, vp, ci, ci, ci, ci, pp, vp]
+    lib.cpe_soft_votes.restype = ci
     _lib = lib
     return lib
 
@@ -158,6 +160,11 @@ def cpe_decode_static(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_
     """``cpe_decode`` on the library's built-in scratch array: no workspace, no allocation (see ``cpe.h``)."""
     return int(load().cpe_decode_static(stream, emb, fg_mask or None, B, H, W, F, ctypes.byref(params), out_labels,
                                         out_centroids, out_count))
+
+
+def cpe_soft_votes(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_hist) -> int:
+    """The soft-vote histogram of Eq. 6, ``float [B, bins_h, bins_w]`` (see ``cpe.h``)."""
+    return int(load().cpe_soft_votes(stream, emb, fg_mask or None, B, H, W, F, ctypes.byref(params), out_hist))
 
 
 def cpe_get_intermediate(params: cpe_params, which, B, H, W, F):
@@ -262,6 +269,16 @@ class Decoder:
         s = stream if stream is not None else self.torch.cuda.current_stream(self.device)
         _check(cpe_decode(s.cuda_stream, *self._args(emb, fg)), "cpe_decode")
         return self.labels, self.centroids, self.count
+
+    def soft_votes(self, emb, fg=None, out=None, stream=None):
+        """Enqueue the soft-vote histogram of Eq. 6 of these tensors; returns ``float32 [B, bins_h, bins_w]``."""
+        torch = self.torch
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        if out is None:
+            out = torch.empty((self.B, self.params.bins_h, self.params.bins_w), dtype=torch.float32, device=self.device)
+        _check(cpe_soft_votes(s.cuda_stream, emb.data_ptr(), 0 if fg is None else fg.data_ptr(), self.B, self.H, self.W,
+                              self.F, self.params, out.data_ptr()), "cpe_soft_votes")
+        return out
 
     def capture(self, emb, fg=None, stream=None):
         """Capture one decode of these tensors into a CUDA graph; returns a handle for :meth:`replay`."""

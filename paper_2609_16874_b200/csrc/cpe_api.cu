@@ -17,6 +17,7 @@
 #include "cpe_common.cuh"
 #include "decode_vote.cuh"
 #include "peaks.cuh"
+#include "soft_vote.cuh"
 
 namespace {
 
@@ -691,4 +692,53 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   p.workspace = slot.ptr;
   p.workspace_bytes = CPE_STATIC_SCRATCH_BYTES;
   return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
+}
+
+namespace {
+template <typename T, int KA>
+int launch_soft_votes_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
+                        const float* pal_w, const float* pal_h, float* hist, uint32_t* status) {
+  const int smem = cpe::sv_smem_layout(KA).total;
+  auto kern = cpe::soft_vote_kernel<T, KA>;
+  static bool configured = false;   // per instantiation; the attribute is sticky for the process
+  if (!configured) {
+    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    configured = true;
+  }
+  // one CTA per SM (it holds all of the SM's tensor memory): the SMs are shared among the images and the
+  // 128 x 128 blocks of bins, the CTAs of one block split the pixels
+  const int n_blocks = ((p->bins_w + cpe::kSvBins - 1) / cpe::kSvBins) * ((p->bins_h + cpe::kSvBins - 1) / cpe::kSvBins);
+  const int n_spans = (HW + cpe::kTcSpan - 1) / cpe::kTcSpan;
+  const int split = std::max(1, std::min(n_spans, sm_count() / std::max(1, n_blocks * B)));
+  dim3 grid((unsigned)split, (unsigned)n_blocks, (unsigned)B);
+  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
+  kern<<<grid, cpe::kSvThreads, smem, st>>>(e, fg, HW, F, p->bins_w, p->bins_h, pal_w, pal_h, vec_mask, hist, status);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+}  // namespace
+
+extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
+                   const cpe_params* params, float* out_hist) {
+  if (!emb || !out_hist) return CPE_ERR_NULL;
+  cpe::Layout L;
+  int rc = check_workspace(B, H, W, F, params, &L);
+  if (rc) return rc;
+  const long long HW = (long long)H * W;
+  if ((uintptr_t)emb % 16 || HW % 8 || (uintptr_t)out_hist % 4) return CPE_ERR_ALIGN;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(params->workspace);
+  const float* pal_w = reinterpret_cast<const float*>(ws + L.pal_w);
+  const float* pal_h = reinterpret_cast<const float*>(ws + L.pal_h);
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.status);
+  CPE_CUDA(cudaMemsetAsync(out_hist, 0, sizeof(float) * (size_t)B * params->bins_w * params->bins_h, st));
+  if (params->dtype == CPE_F32)
+    return F <= 8 ? launch_soft_votes_t<float, 16>(st, static_cast<const float*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
+                                                   pal_h, out_hist, status)
+                  : launch_soft_votes_t<float, 32>(st, static_cast<const float*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
+                                                   pal_h, out_hist, status);
+  return F <= 8 ? launch_soft_votes_t<__half, 16>(st, static_cast<const __half*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
+                                                  pal_h, out_hist, status)
+                : launch_soft_votes_t<__half, 32>(st, static_cast<const __half*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
+                                                  pal_h, out_hist, status);
 }

@@ -1,0 +1,91 @@
+"""Soft-vote histogram (Eq. 4-6): CUDA path vs the binary64 oracle, through the C ABI.  All tests need a B200."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_16874_b200 import binding as cb
+from paper_2609_16874_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+# Per bin: binary16 rounding of E_x and of E_y (2^-11 each) before the second contraction, binary32 accumulation and
+# atomics (~1e-6), first contraction good to ~1e-6 in the squared distance (operands split into two binary16 parts).
+REL = 2e-3
+
+
+def run_soft(emb, fg, bins_w, bins_h):
+    import torch
+    B, D, H, W = emb.shape
+    F = D // 4
+    dtype = "f32" if emb.dtype == np.float32 else "f16"
+    dec = cb.Decoder(B, H, W, F, dtype, bins_w, bins_h)
+    d_emb = torch.from_numpy(emb).cuda()
+    d_fg = None if fg is None else torch.from_numpy(np.ascontiguousarray(fg, np.uint8)).cuda()
+    out = dec.soft_votes(d_emb, d_fg)
+    out2 = dec.soft_votes(d_emb, d_fg)          # a second call starts from zero again
+    torch.cuda.synchronize()
+    status = int(np.bitwise_or.reduce(dec.intermediate(cb.CPE_INT_STATUS).cpu().numpy()))
+    h, h2 = out.cpu().numpy(), out2.cpu().numpy()
+    dec.close()
+    assert not (status & cb.CPE_STATUS_INTERNAL), hex(status)
+    assert np.allclose(h, h2, rtol=1e-5, atol=0)
+    return h
+
+
+def check(emb, fg, bins_w, bins_h, cells=None):
+    got = run_soft(emb, fg, bins_w, bins_h)
+    if cells is None:
+        want = oracle.soft_votes(emb, fg, bins_w, bins_h)
+        g = got.astype(np.float64)
+    else:
+        want = oracle.soft_votes(emb, fg, bins_w, bins_h, sample_cells=cells)
+        g = got.reshape(got.shape[0], -1)[:, cells].astype(np.float64)
+    err = np.abs(g - want)
+    assert (err <= REL * want + 1e-30).all(), (float((err / np.maximum(want, 1e-300)).max()), float(want.max()))
+    return got, want
+
+
+@pytest.mark.parametrize("name,over", [
+    ("c1", dict()),                                                    # 128x128, F=4, fp32, 32x32 bins: one block
+    ("c2", dict(H=192, W=256, K=12)),                                  # F=8 fp32, 64x64
+    ("c3", dict(H=64, W=128, K=6, bins_w=144, bins_h=132)),            # fp16; bins beyond one 128-block on both axes
+    ("c5", dict(H=96, W=128, K=12, bins_w=48, bins_h=40)),             # F=16 fp16 (two k-steps per axis)
+])
+def test_soft_votes_match_the_definition(name, over):
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 0)
+    got, want = check(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)
+    assert want.max() > 0.5      # the histogram has real peaks: the check is not about noise floors only
+
+
+def test_soft_votes_without_mask_batch_and_odd_harmonics():
+    rng = np.random.default_rng(3)
+    for F, dtype in ((3, np.float32), (5, np.float16)):
+        emb = (0.6 * rng.standard_normal((2, 4 * F, 40, 48))).astype(dtype)
+        check(emb, None, 21, 37)
+        fg = (rng.random((2, 40, 48)) < 0.3).astype(np.uint8)
+        fg[1] = 0                                                      # an image without participating pixels
+        got, want = check(emb, fg, 21, 37)
+        assert (got[1] == 0).all()
+
+
+def test_soft_votes_skip_nonfinite_and_out_of_range_pixels():
+    rng = np.random.default_rng(5)
+    F = 4
+    emb = rng.standard_normal((1, 4 * F, 32, 64)).astype(np.float32)
+    emb[0, 3, 5, 7] = np.inf
+    emb[0, 9, 6, 1] = np.nan
+    emb[0, 2, 8, 9] = 1.0e6          # finite, far beyond binary16: its weights are exp(-1e6) = 0
+    check(emb, None, 16, 16)
+    h = emb.astype(np.float16)
+    h[0, 1, 2, 3] = np.float16(np.inf)
+    check(h, None, 16, 16)
+
+
+def test_soft_votes_full_size_c2_on_sampled_bins():
+    cfg = wl.CONFIGS["c2"]
+    fr = wl.make_frame(cfg, 0)
+    rng = np.random.default_rng(9)
+    cells = np.unique(np.concatenate([rng.integers(0, cfg.bins_w * cfg.bins_h, 24),
+                                      np.argsort(oracle.votes(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)["votes"].ravel())[-8:]]))
+    check(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cells=cells.astype(np.int32))
