@@ -393,6 +393,10 @@ def run_ours(args, cfg):
             except Exception as exc:   # a parity-test workload must not take the headline line down with it
                 others[name] = {"error": repr(exc)}
         line["other_configs"] = others
+        try:
+            line["soft_votes"] = measure_soft_votes(cfg, max(20, min(K, 100)), max(3, min(Wm, 10)), dev)
+        except Exception as exc:
+            line["soft_votes"] = {"error": repr(exc)}
     print(json.dumps(line))
     dist_util.shutdown()
 
@@ -436,6 +440,48 @@ def measure_other(cfg, steps, warmup, dev):
             "frac_of_algorithmic_bytes_roofline": alg / (peak_gbs * 1e9) / (p50 * 1e-3)}
 
 
+# Ceiling of the special-function units: 148 SMs x 16 results per clock x 1.965 GHz.
+SFU_PEAK_GOPS = 148 * 16 * 1.965
+
+
+def measure_soft_votes(cfg, steps, warmup, dev):
+    """The second vote mode (`cpe_soft_votes`, Eq. 6) on the same workload: device time per call over rotating
+    frames.  Its floor is the special-function units: every (participating pixel, bin of either axis) pair costs
+    one square root and one exponential."""
+    import torch
+    from paper_2609_16874_b200 import binding as cb
+    n_frames = frames_needed(cfg)
+    frames = [wl.make_frame(cfg, f) for f in range(n_frames)]
+    d_emb = [torch.from_numpy(f["emb"]).to(dev) for f in frames]
+    d_fg = [torch.from_numpy(f["fg"]).to(dev) for f in frames]
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        out = dec.soft_votes(d_emb[0], d_fg[0], stream=stream)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(warmup + steps):
+            j = i - warmup
+            if j >= 0:
+                ev[j][0].record(stream)
+            dec.soft_votes(d_emb[i % n_frames], d_fg[i % n_frames], out=out, stream=stream)
+            if j >= 0:
+                ev[j][1].record(stream)
+        stream.synchronize()
+    ms = np.array([a.elapsed_time(b) for a, b in ev])
+    dec.close()
+    part = float(np.mean([f["fg"].sum() for f in frames]))
+    n_ab, n_bb = -(-cfg.bins_w // 128), -(-cfg.bins_h // 128)
+    pairs = part * (cfg.bins_w + cfg.bins_h)                       # the method's own count
+    r32 = lambda n: min(128, -(-n // 32) * 32)
+    issued = part * sum(r32(cfg.bins_w - 128 * i) + r32(cfg.bins_h - 128 * j) for i in range(n_ab) for j in range(n_bb))   # what the blocks evaluate
+    p50 = float(np.percentile(ms, 50))
+    return {"entry_point": "cpe_soft_votes", "p50_ms": p50, "value": cfg.pixels / (p50 * 1e-3) / 1e6, "unit": UNIT,
+            "bound": "sfu", "pixel_bin_pairs": pairs, "sfu_ops_algorithmic": 2 * pairs, "sfu_ops_issued": 2 * issued,
+            "achieved_gops": 2 * pairs / (p50 * 1e-3) / 1e9, "peak_gops": SFU_PEAK_GOPS,
+            "frac": 2 * pairs / (p50 * 1e-3) / 1e9 / SFU_PEAK_GOPS,
+            "note": "memset + one kernel per call; two tcgen05 contractions per 128-pixel tile, weights kept on the SM"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -447,9 +493,17 @@ def main():
     ap.add_argument("--only-default", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--quick", action="store_true",
                     help="profiling runs: no clock pre-heat, no host-buffer leg, no CPU baseline (few launches)")
+    ap.add_argument("--soft-votes", action="store_true",
+                    help="profiling runs: only the second vote mode (cpe_soft_votes) on the chosen workload")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
     cfg = wl.CONFIGS[args.config]
+    if args.soft_votes:
+        import torch
+        dev = torch.device("cuda", 0)
+        torch.cuda.set_device(dev)
+        print(json.dumps({"soft_votes": measure_soft_votes(cfg, args.steps, args.warmup, dev), "name": cfg.name}))
+        return
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

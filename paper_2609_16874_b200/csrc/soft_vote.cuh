@@ -112,6 +112,9 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < kSvTiles * 2 * kPartHalves / 2; i += kSvThreads) reinterpret_cast<uint32_t*>(s_tiles)[i] = 0u;
+  for (int i = tid; i < kTcRows * kSvBins; i += kSvThreads) {      // E_x and E_y are contiguous
+    reinterpret_cast<uint32_t*>(s_ex)[i] = 0u;
+  }
   // -2 P rows of this block, split into binary16 high and low parts; K-major core matrices: (bin n, slot s) at
   // (s / 8) * (128 * 8) + n * 8 + s % 8.  Bins beyond the map are zero rows (their H entries are never stored).
   for (int i = tid; i < 2 * kSvBins * KA; i += kSvThreads) {
@@ -281,14 +284,20 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     uint32_t t = 0;
     bool bad = false;
     const float log2e = 1.4426950408889634f;
+    const int na = min(kSvBins, bins_w - a0), nb = min(kSvBins, bins_h - b0);   // bins of this block that exist
 
-    // exp(-sqrt(max(c + D, 0))) for 8 consecutive bins, rounded to binary16
+    // exp(-sqrt(max(c + D, 0))) for 8 consecutive bins, rounded to binary16.  The special-function unit's
+    // approximations (sqrt, 2^x: about 2^-22 relative each) are far inside the binary16 rounding that follows.
     auto weights8 = [&](const float* v, float c, bool live) -> uint4 {
-      __half h[8];
+      __half2 h[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float d = sqrtf(fmaxf(c + v[i], 0.0f));
-        h[i] = __float2half_rn(live ? exp2f(-d * log2e) : 0.0f);
+      for (int i = 0; i < 4; ++i) {
+        float d0, d1, e0, e1;
+        asm("sqrt.approx.f32 %0, %1;" : "=f"(d0) : "f"(fmaxf(c + v[2 * i], 0.0f)));
+        asm("sqrt.approx.f32 %0, %1;" : "=f"(d1) : "f"(fmaxf(c + v[2 * i + 1], 0.0f)));
+        asm("ex2.approx.f32 %0, %1;" : "=f"(e0) : "f"(-d0 * log2e));
+        asm("ex2.approx.f32 %0, %1;" : "=f"(e1) : "f"(-d1 * log2e));
+        h[i] = __floats2half2_rn(live ? e0 : 0.0f, live ? e1 : 0.0f);
       }
       return *reinterpret_cast<const uint4*>(h);
     };
@@ -339,13 +348,19 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       {
         unsigned char* ex_row = reinterpret_cast<unsigned char*>(s_ex) + (tid >> 3) * kELbo + (tid & 7) * 16;
         unsigned char* ey_row = reinterpret_cast<unsigned char*>(s_ey) + (tid >> 3) * kELbo + (tid & 7) * 16;
-        for (int c0 = 0; c0 < kSvBins; c0 += 32) {
+        // only the bins that exist (in steps of 32): the rest of the E tiles stays zero
+        for (int c0 = 0; c0 < max(na, nb); c0 += 32) {
           float vx[32], vy[32];
           tc_ld32x2(t_lane + (uint32_t)c0, t_lane + 128u + (uint32_t)c0, vx, vy);
+          if (c0 < na) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            *reinterpret_cast<uint4*>(ex_row + ((c0 >> 3) + g) * 128) = weights8(vx + 8 * g, cx, live);
-            *reinterpret_cast<uint4*>(ey_row + ((c0 >> 3) + g) * 128) = weights8(vy + 8 * g, cy, live);
+            for (int g = 0; g < 4; ++g)
+              *reinterpret_cast<uint4*>(ex_row + ((c0 >> 3) + g) * 128) = weights8(vx + 8 * g, cx, live);
+          }
+          if (c0 < nb) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+              *reinterpret_cast<uint4*>(ey_row + ((c0 >> 3) + g) * 128) = weights8(vy + 8 * g, cy, live);
           }
         }
       }
