@@ -73,6 +73,8 @@ def _load():
         lib.cpe_oracle_decode.restype = c_int
         lib.cpe_oracle_soft_votes.argtypes = [vp, c_int, vp] + [c_int] * 6 + [vp, c_int, vp]
         lib.cpe_oracle_soft_votes.restype = c_int
+        lib.cpe_oracle_instance_masks.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp]
+        lib.cpe_oracle_instance_masks.restype = c_int
         _lib = lib
     return _lib
 
@@ -248,3 +250,16 @@ def soft_votes(emb: np.ndarray, fg, bins_w: int, bins_h: int, sample_cells=None)
     if rc:
         raise RuntimeError(f"cpe_oracle_soft_votes failed: {rc}")
     return out
+
+
+def instance_masks(labels: np.ndarray, n_planes: int, want_planes: bool = True):
+    """One-hot mask planes ``uint8 [B, n_planes, H, W]`` (or None) and pixel counters ``uint32 [B, n_planes]`` of a
+    label map (0 = none, m + 1 = mask m)."""
+    labels = np.ascontiguousarray(labels, np.int32)
+    B, H, W = labels.shape
+    planes = np.empty((B, n_planes, H, W), np.uint8) if want_planes else None
+    pixels = np.empty((B, n_planes), np.uint32)
+    rc = _load().cpe_oracle_instance_masks(_ptr(labels), B, H, W, n_planes, _ptr(planes), _ptr(pixels))
+    if rc:
+        raise RuntimeError(f"cpe_oracle_instance_masks failed: {rc}")
+    return planes, pixels

@@ -354,6 +354,31 @@ int cpe_oracle_assign_image(const void* emb_img, int dtype, const uint8_t* fg_im
 
 /* ------------------------------------------------------------- the whole chain ---- */
 
+/* ------------------------------------------------ Sec. 3.2 "Mask aggregation": per-instance outputs ---- */
+
+/*
+ * The paper's output form of the assignment: one binary mask per candidate centroid and a counter of the pixels
+ * that went to it (Eq. 8; Sec. 3.2: "output masks ... and a counter").  From a label map (0 = none, m + 1 = mask m):
+ * planes[b][m][i][j] = 1 iff labels[b][i][j] == m + 1, pixels[b][m] = number of such pixels, for m < n_planes.
+ * Either output may be NULL.
+ */
+int cpe_oracle_instance_masks(const int32_t* labels, int B, int H, int W, int n_planes, uint8_t* planes,
+                              uint32_t* pixels) {
+  if (!labels || B < 1 || H < 1 || W < 1 || n_planes < 1) return -1;
+  const size_t HW = (size_t)H * W;
+  for (int b = 0; b < B; ++b)
+    for (int m = 0; m < n_planes; ++m) {
+      uint32_t cnt = 0;
+      for (size_t p = 0; p < HW; ++p) {
+        const int hit = labels[(size_t)b * HW + p] == m + 1;
+        if (planes) planes[((size_t)b * n_planes + m) * HW + p] = (uint8_t)hit;
+        cnt += (uint32_t)hit;
+      }
+      if (pixels) pixels[(size_t)b * n_planes + m] = cnt;
+    }
+  return 0;
+}
+
 /* ------------------------------------------- Eq. 4-6: the soft-vote histogram (binary64) ---- */
 
 /*

@@ -587,3 +587,21 @@ def test_soft_votes_skip_masked_and_nonfinite_pixels_and_sampled_cells_agree():
     # binary16 inputs are widened exactly
     h = emb.astype(np.float16)
     assert np.array_equal(oracle.soft_votes(h, fg, bw, bh), oracle.soft_votes(h.astype(np.float32), fg, bw, bh))
+
+
+# ---------------------------------------------------------------- per-instance outputs (Sec. 3.2, Eq. 8)
+
+def test_instance_masks_partition_the_labelled_pixels_and_count_them():
+    """Planes are disjoint, their union is the set of labelled pixels, counters equal numpy's bincount, labels beyond
+    the planes asked for are left out, and the label map is recovered from the planes."""
+    rng = np.random.default_rng(21)
+    labels = rng.integers(0, 8, (2, 9, 13)).astype(np.int32)
+    planes, pixels = oracle.instance_masks(labels, 5)
+    assert planes.dtype == np.uint8 and set(np.unique(planes)) <= {0, 1}
+    assert np.array_equal(planes.sum(1), ((labels >= 1) & (labels <= 5)).astype(np.uint64))
+    for b in range(2):
+        assert np.array_equal(pixels[b], np.bincount(labels[b].ravel(), minlength=9)[1:6])
+    back = (planes * np.arange(1, 6, dtype=np.int32)[None, :, None, None]).sum(1)
+    assert np.array_equal(back, np.where(labels <= 5, labels, 0))
+    assert oracle.instance_masks(labels, 7, want_planes=False)[0] is None
+    assert np.array_equal(oracle.instance_masks(labels, 7, want_planes=False)[1][:, :5], pixels)
