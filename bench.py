@@ -397,6 +397,10 @@ def run_ours(args, cfg):
             line["soft_votes"] = measure_soft_votes(cfg, max(20, min(K, 100)), max(3, min(Wm, 10)), dev)
         except Exception as exc:
             line["soft_votes"] = {"error": repr(exc)}
+        try:
+            line["instance_masks"] = {n: measure_instance_masks(wl.CONFIGS[n], 20, 3, dev) for n in (cfg.name, "c5")}
+        except Exception as exc:
+            line["instance_masks"] = {"error": repr(exc)}
     print(json.dumps(line))
     dist_util.shutdown()
 
@@ -480,6 +484,40 @@ def measure_soft_votes(cfg, steps, warmup, dev):
             "achieved_gops": 2 * pairs / (p50 * 1e-3) / 1e9, "peak_gops": SFU_PEAK_GOPS,
             "frac": 2 * pairs / (p50 * 1e-3) / 1e9 / SFU_PEAK_GOPS,
             "note": "memset + one kernel per call; two tcgen05 contractions per 128-pixel tile, weights kept on the SM"}
+
+
+def measure_instance_masks(cfg, steps, warmup, dev):
+    """`cpe_instance_masks` (the paper's one-hot planes and pixel counters) after one decode of the workload: a
+    store-bound pass, 4 bytes read and n_planes bytes written per pixel; planes = the number of instances found."""
+    import torch
+    from paper_2609_16874_b200 import binding as cb
+    fr = wl.make_frame(cfg, 0)
+    d_emb, d_fg = torch.from_numpy(fr["emb"]).to(dev), torch.from_numpy(fr["fg"]).to(dev)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev)
+    dec.decode(d_emb, d_fg)
+    torch.cuda.synchronize()
+    n_planes = max(1, int(dec.count.max().item()))
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(warmup + steps):
+            j = i - warmup
+            if j >= 0:
+                ev[j][0].record(stream)
+            planes, pixels = dec.instance_masks(n_planes, stream=stream)
+            if j >= 0:
+                ev[j][1].record(stream)
+            del planes, pixels
+        stream.synchronize()
+    ms = np.array([a.elapsed_time(b) for a, b in ev])
+    dec.close()
+    peak_gbs, _ = measured_peaks()
+    p50 = float(np.percentile(ms, 50))
+    nbytes = cfg.pixels * (4 + n_planes)
+    return {"entry_point": "cpe_instance_masks", "n_planes": n_planes, "p50_ms": p50, "bound": "hbm",
+            "algorithmic_bytes": nbytes, "achieved": nbytes / (p50 * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
+            "frac": nbytes / (p50 * 1e-3) / 1e9 / peak_gbs,
+            "note": "includes torch's allocation of the output planes on the stream and the counters' memset"}
 
 
 def main():

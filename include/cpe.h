@@ -267,6 +267,21 @@ int cpe_decode_static(cpe_stream_t stream, const void* emb, const uint8_t* fg_ma
 int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
                    const cpe_params* params, float* out_hist);
 
+/*
+ * The paper's output form of the assignment (Sec. 3.2 "Mask aggregation", Eq. 8): one binary mask per candidate
+ * centroid and a counter of the pixels that went to it, expanded from a label map as cpe_decode writes it
+ * (0 = no mask, m + 1 = mask m).  For m < n_planes:
+ *   out_planes [B][n_planes][H][W] uint8:  1 where labels == m + 1, else 0   (NULL: not wanted)
+ *   out_pixels [B][n_planes] uint32:       the number of such pixels         (NULL: not wanted)
+ * labels, out_planes, out_pixels: device memory owned by the caller; labels int32 [B][H][W].  n_planes in
+ * [1, 8191] (usually the decode's max_instances or the largest count); labels above n_planes are ignored.  Both
+ * outputs are written completely.  Enqueues on the stream (a memset of the counters and one kernel), capturable.
+ * Errors: CPE_ERR_NULL (labels, or both outputs NULL), CPE_ERR_SIZE, CPE_ERR_ALIGN (labels / out_pixels not 4-byte
+ * aligned), CPE_ERR_CUDA.
+ */
+int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, int B, int H, int W, int n_planes,
+                       uint8_t* out_planes, uint32_t* out_pixels);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,7 +38,7 @@ EXPORTS = (
     "cpe_workspace_size", "cpe_init_workspace", "cpe_decode", "cpe_get_intermediate", "cpe_strerror",
     "cpe_last_cuda_error", "cpe_graph_create", "cpe_graph_launch", "cpe_graph_destroy", "cpe_graph_kernel_nodes",
     "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
-    "cpe_decode_static", "cpe_soft_votes",
+    "cpe_decode_static", "cpe_soft_votes", "cpe_instance_masks",
 )
 
 
@@ -123,6 +123,8 @@ def load() -> ctypes.CDLL:
     lib.cpe_decode_static.restype = ci
     lib.cpe_soft_votes.argtypes = [vp, vp, vp, ci, ci, ci, ci, pp, vp]
     lib.cpe_soft_votes.restype = ci
+    lib.cpe_instance_masks.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.cpe_instance_masks.restype = ci
     _lib = lib
     return lib
 
@@ -165,6 +167,11 @@ def cpe_decode_static(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_
 def cpe_soft_votes(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_hist) -> int:
     """The soft-vote histogram of Eq. 6, ``float [B, bins_h, bins_w]`` (see ``cpe.h``)."""
     return int(load().cpe_soft_votes(stream, emb, fg_mask or None, B, H, W, F, ctypes.byref(params), out_hist))
+
+
+def cpe_instance_masks(stream, labels, B, H, W, n_planes, out_planes, out_pixels) -> int:
+    """One-hot mask planes and per-instance pixel counters of a label map (see ``cpe.h``)."""
+    return int(load().cpe_instance_masks(stream, labels, B, H, W, n_planes, out_planes or None, out_pixels or None))
 
 
 def cpe_get_intermediate(params: cpe_params, which, B, H, W, F):
@@ -279,6 +286,17 @@ class Decoder:
         _check(cpe_soft_votes(s.cuda_stream, emb.data_ptr(), 0 if fg is None else fg.data_ptr(), self.B, self.H, self.W,
                               self.F, self.params, out.data_ptr()), "cpe_soft_votes")
         return out
+
+    def instance_masks(self, n_planes, want_planes=True, stream=None):
+        """One-hot planes ``uint8 [B, n_planes, H, W]`` (or None) and counters ``int32 [B, n_planes]`` of ``labels``."""
+        torch = self.torch
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        planes = (torch.empty((self.B, n_planes, self.H, self.W), dtype=torch.uint8, device=self.device)
+                  if want_planes else None)
+        pixels = torch.empty((self.B, n_planes), dtype=torch.int32, device=self.device)
+        _check(cpe_instance_masks(s.cuda_stream, self.labels.data_ptr(), self.B, self.H, self.W, n_planes,
+                                  0 if planes is None else planes.data_ptr(), pixels.data_ptr()), "cpe_instance_masks")
+        return planes, pixels
 
     def capture(self, emb, fg=None, stream=None):
         """Capture one decode of these tensors into a CUDA graph; returns a handle for :meth:`replay`."""

@@ -16,6 +16,7 @@
 #include "cpe.h"
 #include "cpe_common.cuh"
 #include "decode_vote.cuh"
+#include "instance_masks.cuh"
 #include "peaks.cuh"
 #include "soft_vote.cuh"
 
@@ -741,4 +742,24 @@ extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_
                                                   pal_h, out_hist, status)
                 : launch_soft_votes_t<__half, 32>(st, static_cast<const __half*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
                                                   pal_h, out_hist, status);
+}
+
+extern "C" int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, int B, int H, int W, int n_planes,
+                                  uint8_t* out_planes, uint32_t* out_pixels) {
+  if (!labels || (!out_planes && !out_pixels)) return CPE_ERR_NULL;
+  if (B < 1 || H < 1 || W < 1 || n_planes < 1 || n_planes > 8191 || (long long)H * W > 0x7fffffffLL) return CPE_ERR_SIZE;
+  if ((uintptr_t)labels % 4 || (uintptr_t)out_pixels % 4) return CPE_ERR_ALIGN;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int HW = H * W;
+  if (out_pixels) CPE_CUDA(cudaMemsetAsync(out_pixels, 0, sizeof(uint32_t) * (size_t)B * n_planes, st));
+  // 128-bit accesses need aligned rows of every image and plane
+  const int vec = ((uintptr_t)labels % 16 == 0) && (HW % 16 == 0) && (!out_planes || (uintptr_t)out_planes % 16 == 0);
+  const long long n_chunks = ((long long)HW + cpe::kImPixels - 1) / cpe::kImPixels;
+  const long long ctas = (n_chunks + cpe::kImThreads - 1) / cpe::kImThreads;
+  const long long per_image = std::max(1, (8 * sm_count() + B - 1) / B);
+  dim3 grid((unsigned)std::min(ctas, per_image), (unsigned)B);
+  const size_t smem = out_pixels ? sizeof(uint32_t) * (size_t)(n_planes + 1) : 0;
+  cpe::instance_masks_kernel<<<grid, cpe::kImThreads, smem, st>>>(labels, HW, n_planes, vec, out_planes, out_pixels);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
 }
