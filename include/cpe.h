@@ -282,6 +282,17 @@ int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask,
 int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, int B, int H, int W, int n_planes,
                        uint8_t* out_planes, uint32_t* out_pixels);
 
+/*
+ * Layout variant.  The paper writes the network prediction as H_O x W_O x 4L (Sec. 3.1, Eq. 3); cpe_decode reads
+ * planes.  cpe_channels_last_to_planar copies emb_nhwc [B][H][W][4F] into emb_planar [B][4F][H][W] (same element
+ * type, dtype = CPE_F32 or CPE_F16; both device memory owned by the caller, not overlapping), one read and one
+ * write of the embedding, so that a producer of the paper's layout can feed the decoder.  Enqueues one kernel on
+ * the stream; capturable.  Errors: CPE_ERR_NULL, CPE_ERR_SIZE (B, H, W < 1, F outside [1,16]), CPE_ERR_DTYPE,
+ * CPE_ERR_ALIGN (pointers not aligned to the element size), CPE_ERR_CUDA.
+ */
+int cpe_channels_last_to_planar(cpe_stream_t stream, const void* emb_nhwc, void* emb_planar, int B, int H, int W, int F,
+                                int dtype);
+
 #ifdef __cplusplus
 }
 #endif

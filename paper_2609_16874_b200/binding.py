@@ -38,7 +38,7 @@ EXPORTS = (
     "cpe_workspace_size", "cpe_init_workspace", "cpe_decode", "cpe_get_intermediate", "cpe_strerror",
     "cpe_last_cuda_error", "cpe_graph_create", "cpe_graph_launch", "cpe_graph_destroy", "cpe_graph_kernel_nodes",
     "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
-    "cpe_decode_static", "cpe_soft_votes", "cpe_instance_masks",
+    "cpe_decode_static", "cpe_soft_votes", "cpe_instance_masks", "cpe_channels_last_to_planar",
 )
 
 
@@ -125,6 +125,8 @@ def load() -> ctypes.CDLL:
     lib.cpe_soft_votes.restype = ci
     lib.cpe_instance_masks.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     lib.cpe_instance_masks.restype = ci
+    lib.cpe_channels_last_to_planar.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci]
+    lib.cpe_channels_last_to_planar.restype = ci
     _lib = lib
     return lib
 
@@ -172,6 +174,11 @@ def cpe_soft_votes(stream, emb, fg_mask, B, H, W, F, params: cpe_params, out_his
 def cpe_instance_masks(stream, labels, B, H, W, n_planes, out_planes, out_pixels) -> int:
     """One-hot mask planes and per-instance pixel counters of a label map (see ``cpe.h``)."""
     return int(load().cpe_instance_masks(stream, labels, B, H, W, n_planes, out_planes or None, out_pixels or None))
+
+
+def cpe_channels_last_to_planar(stream, emb_nhwc, emb_planar, B, H, W, F, dtype) -> int:
+    """``[B, H, W, 4F]`` to the planar ``[B, 4F, H, W]`` that ``cpe_decode`` reads (see ``cpe.h``)."""
+    return int(load().cpe_channels_last_to_planar(stream, emb_nhwc, emb_planar, B, H, W, F, dtype))
 
 
 def cpe_get_intermediate(params: cpe_params, which, B, H, W, F):

@@ -17,6 +17,7 @@
 #include "cpe_common.cuh"
 #include "decode_vote.cuh"
 #include "instance_masks.cuh"
+#include "layout.cuh"
 #include "peaks.cuh"
 #include "soft_vote.cuh"
 
@@ -760,6 +761,31 @@ extern "C" int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, in
   dim3 grid((unsigned)std::min(ctas, per_image), (unsigned)B);
   const size_t smem = out_pixels ? sizeof(uint32_t) * (size_t)(n_planes + 1) : 0;
   cpe::instance_masks_kernel<<<grid, cpe::kImThreads, smem, st>>>(labels, HW, n_planes, vec, out_planes, out_pixels);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
+extern "C" int cpe_channels_last_to_planar(cpe_stream_t stream, const void* emb_nhwc, void* emb_planar, int B, int H,
+                                           int W, int F, int dtype) {
+  if (!emb_nhwc || !emb_planar) return CPE_ERR_NULL;
+  if (B < 1 || H < 1 || W < 1 || F < 1 || F > 16 || (long long)H * W > 0x7fffffffLL) return CPE_ERR_SIZE;
+  if (dtype != CPE_F32 && dtype != CPE_F16) return CPE_ERR_DTYPE;
+  const size_t esz = dtype == CPE_F32 ? 4 : 2;
+  if ((uintptr_t)emb_nhwc % esz || (uintptr_t)emb_planar % esz) return CPE_ERR_ALIGN;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int HW = H * W, D = 4 * F;
+  dim3 grid((unsigned)((HW + cpe::kLyPixels - 1) / cpe::kLyPixels), (unsigned)B);
+  const size_t smem = (size_t)cpe::kLyPixels * (D + 1) * esz;
+  // 128-bit accesses: every tile of the source starts on a 16-byte boundary iff 128 * D * esz does (always) and the
+  // base does; a plane piece does iff the base, the plane pitch H * W and the tile start are multiples of 16 bytes
+  const int vec_in = (uintptr_t)emb_nhwc % 16 == 0 && ((size_t)HW * D * esz) % 16 == 0;
+  const int vec_out = (uintptr_t)emb_planar % 16 == 0 && ((size_t)HW * esz) % 16 == 0;
+  if (dtype == CPE_F32)
+    cpe::channels_last_to_planar_kernel<float><<<grid, cpe::kLyThreads, smem, st>>>(
+        static_cast<const float*>(emb_nhwc), static_cast<float*>(emb_planar), HW, D, vec_in, vec_out);
+  else
+    cpe::channels_last_to_planar_kernel<__half><<<grid, cpe::kLyThreads, smem, st>>>(
+        static_cast<const __half*>(emb_nhwc), static_cast<__half*>(emb_planar), HW, D, vec_in, vec_out);
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
