@@ -67,8 +67,12 @@ def _load():
         lib.cpe_oracle_centroid_px.argtypes = [c_int] * 6 + [vp]
         lib.cpe_oracle_centroid_px.restype = None
         lib.cpe_oracle_assign_image.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, vp, c_int, vp, c_int,
-                                                c_dbl, vp, ctypes.c_int64, vp, vp, vp, vp]
+                                                c_dbl, vp, ctypes.c_int64, vp, vp, vp, vp, vp]
         lib.cpe_oracle_assign_image.restype = c_int
+        lib.cpe_oracle_vote_sums.argtypes = [vp, vp, c_int, c_int, c_int, c_int, vp]
+        lib.cpe_oracle_vote_sums.restype = c_int
+        lib.cpe_oracle_refined_peaks.argtypes = [vp, vp, c_int, c_int, vp] + [c_int] * 4 + [vp, vp, vp]
+        lib.cpe_oracle_refined_peaks.restype = c_int
         lib.cpe_oracle_decode.argtypes = ([vp, vp] + [c_int] * 9 + [c_dbl, c_int] + [vp] * 9)
         lib.cpe_oracle_decode.restype = c_int
         lib.cpe_oracle_soft_votes.argtypes = [vp, c_int, vp] + [c_int] * 6 + [vp, c_int, vp]
@@ -179,8 +183,10 @@ def centroid_px(cx: int, cy: int, bins_w: int, bins_h: int, H: int, W: int):
 
 
 def assign_image(emb_img: np.ndarray, fg_img, bins_w: int, bins_h: int, peak_cell: np.ndarray, tau=np.inf,
-                 idx=None):
-    """Eq. 7-8 for one image ``[4F, H, W]``; ``idx`` restricts the work to sampled flat pixel indices."""
+                 idx=None, peak_emb=None):
+    """Eq. 7-8 for one image ``[4F, H, W]``; ``idx`` restricts the work to sampled flat pixel indices.
+
+    ``peak_emb`` ``[count, 4F]`` float32 replaces the palette rows of the peaks' bins as the candidates."""
     emb_img = np.ascontiguousarray(emb_img)
     D, H, W = emb_img.shape
     F = D // 4
@@ -198,9 +204,12 @@ def assign_image(emb_img: np.ndarray, fg_img, bins_w: int, bins_h: int, peak_cel
     best = np.empty(shape, np.float64)
     second = np.empty(shape, np.float64)
     rej = np.zeros(1, np.int64)
+    if peak_emb is not None:
+        peak_emb = np.ascontiguousarray(peak_emb, np.float32)
+        assert peak_emb.shape == (pc.shape[0], D)
     rc = _load().cpe_oracle_assign_image(_ptr(emb_img), _dtype_code(emb_img), _ptr(fgc), H, W, F, _ptr(Pw), _ptr(Ph),
                                          bins_w, _ptr(pc), pc.shape[0], float(tau), _ptr(idx), n, _ptr(labels),
-                                         _ptr(best), _ptr(second), _ptr(rej))
+                                         _ptr(best), _ptr(second), _ptr(rej), _ptr(peak_emb))
     if rc:
         raise RuntimeError(f"cpe_oracle_assign_image failed: {rc}")
     return {"labels": labels, "best": best, "second": second, "tau_rejected": int(rej[0])}
@@ -229,6 +238,68 @@ def decode(emb: np.ndarray, fg, bins_w: int, bins_h: int, T_v: int = 8, tau=np.i
         raise RuntimeError(f"cpe_oracle_decode failed: {rc}")
     return {"labels": labels, "centroids": centroids, "count": count, "votes": V, "peak_cell": pc,
             "peak_votes": pv, "best": best, "second": second, "counters": counters}
+
+
+def vote_sums(est: np.ndarray, cell: np.ndarray, bins_w: int, bins_h: int) -> np.ndarray:
+    """Fixed-point (2^-24) sums of the estimates per cell, ``[B, bins_h, bins_w, 2]`` int64."""
+    est = np.ascontiguousarray(est, np.float32)
+    cell = np.ascontiguousarray(cell, np.int32)
+    B, H, W = cell.shape
+    sums = np.empty((B, bins_h, bins_w, 2), np.int64)
+    rc = _load().cpe_oracle_vote_sums(_ptr(est), _ptr(cell), B, H, W, bins_w * bins_h, _ptr(sums))
+    if rc:
+        raise RuntimeError(f"cpe_oracle_vote_sums failed: {rc}")
+    return sums
+
+
+def refined_peaks(V: np.ndarray, sums: np.ndarray, peak_cell: np.ndarray, F: int, H: int, W: int):
+    """Refined candidates of ONE image: gamma(mean estimate of the peak's 3x3 window) and the mean in pixels."""
+    V = np.ascontiguousarray(V, np.uint32)
+    sums = np.ascontiguousarray(sums, np.int64)
+    pc = np.ascontiguousarray(peak_cell, np.int32)
+    bh, bw = V.shape
+    K = pc.shape[0]
+    pe = np.empty((K, 4 * F), np.float32)
+    cen = np.empty((K, 2), np.float32)
+    mean = np.empty((K, 2), np.float64)
+    rc = _load().cpe_oracle_refined_peaks(_ptr(V), _ptr(sums), bw, bh, _ptr(pc), K, F, H, W, _ptr(pe), _ptr(cen),
+                                          _ptr(mean))
+    if rc:
+        raise RuntimeError(f"cpe_oracle_refined_peaks failed: {rc}")
+    return {"peak_emb": pe, "centroids": cen, "mean": mean}
+
+
+def decode_refined(emb: np.ndarray, fg, bins_w: int, bins_h: int, T_v: int = 8, tau=np.inf, K_max: int = 1024,
+                   levels: int = 0):
+    """The chain with sub-cell refined candidates: votes and sums, peaks, gamma(mean), assignment."""
+    emb = np.ascontiguousarray(emb)
+    B, D, H, W = emb.shape
+    F = D // 4
+    v = votes(emb, fg, bins_w, bins_h, levels, want_est=True, want_cell=True)
+    sums = vote_sums(v["est"], v["cell"], bins_w, bins_h)
+    labels = np.empty((B, H, W), np.int32)
+    best = np.empty((B, H, W), np.float64)
+    second = np.empty((B, H, W), np.float64)
+    centroids = np.full((B, K_max, 2), np.nan, np.float32)
+    peak_emb = np.zeros((B, K_max, D), np.float32)
+    pc_all = np.full((B, K_max), -1, np.int32)
+    count = np.zeros(B, np.int32)
+    counters = v["counters"].copy()
+    for b in range(B):
+        pc, _, raw = peaks(v["votes"][b], T_v, K_max)
+        r = refined_peaks(v["votes"][b], sums[b], pc, F, H, W)
+        a = assign_image(emb[b], None if fg is None else fg[b], bins_w, bins_h, pc, tau, peak_emb=r["peak_emb"])
+        k = pc.shape[0]
+        count[b] = k
+        pc_all[b, :k] = pc
+        centroids[b, :k] = r["centroids"]
+        peak_emb[b, :k] = r["peak_emb"]
+        labels[b], best[b], second[b] = a["labels"], a["best"], a["second"]
+        counters[b, CNT_RAW_PEAKS] = raw
+        counters[b, CNT_TRUNCATED] = raw - k
+        counters[b, CNT_TAU_REJECTED] = a["tau_rejected"]
+    return {"labels": labels, "centroids": centroids, "count": count, "votes": v["votes"], "sums": sums,
+            "peak_cell": pc_all, "peak_emb": peak_emb, "best": best, "second": second, "counters": counters}
 
 
 def soft_votes(emb: np.ndarray, fg, bins_w: int, bins_h: int, sample_cells=None) -> np.ndarray:

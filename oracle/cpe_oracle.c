@@ -300,7 +300,7 @@ void cpe_oracle_centroid_px(int cx, int cy, int bins_w, int bins_h, int H, int W
 int cpe_oracle_assign_image(const void* emb_img, int dtype, const uint8_t* fg_img, int H, int W, int F,
                             const float* Pw, const float* Ph, int bins_w, const int32_t* peak_cell, int count,
                             double tau, const int64_t* idx, int64_t n_idx, int32_t* labels, double* best,
-                            double* second, int64_t* tau_rejected) {
+                            double* second, int64_t* tau_rejected, const float* peak_emb) {
   size_t HW = (size_t)H * W;
   int64_t N = idx ? n_idx : (int64_t)HW;
   int64_t rejected = 0;
@@ -328,8 +328,9 @@ int cpe_oracle_assign_image(const void* emb_img, int dtype, const uint8_t* fg_im
     if (!finite) continue;
     for (int k = 0; k < count; ++k) {
       int cx = peak_cell[k] % bins_w, cy = peak_cell[k] / bins_w;
-      const float* ex = Pw + (size_t)cx * 2 * F;
-      const float* ey = Ph + (size_t)cy * 2 * F;
+      /* candidates are the palette rows of the peak's bin (Eq. 7), unless the caller hands in refined ones */
+      const float* ex = peak_emb ? peak_emb + (size_t)k * 4 * F : Pw + (size_t)cx * 2 * F;
+      const float* ey = peak_emb ? peak_emb + (size_t)k * 4 * F + 2 * F : Ph + (size_t)cy * 2 * F;
       double sx = 0.0, sy = 0.0;
       for (int c = 0; c < 2 * F; ++c) {
         double dx = xh[c] - (double)ex[c];
@@ -466,7 +467,7 @@ int cpe_oracle_decode(const void* emb, const uint8_t* fg, int B, int H, int W, i
     cpe_oracle_assign_image((const char*)emb + (size_t)b * 4 * F * HW * esz, dtype, fg ? fg + b * HW : NULL, H, W,
                             F, Pw, Ph, bins_w, peak_cell + (size_t)b * K_max, kept, tau, NULL, 0,
                             out_labels + b * HW, best ? best + b * HW : NULL, second ? second + b * HW : NULL,
-                            &rejected);
+                            &rejected, NULL);
     if (counters) {
       counters[b * CNT_N + CNT_RAW_PEAKS] = raw;
       counters[b * CNT_N + CNT_TRUNCATED] = raw - kept;
@@ -475,5 +476,71 @@ int cpe_oracle_decode(const void* emb, const uint8_t* fg, int B, int H, int W, i
   }
   free(Pw);
   free(Ph);
+  return 0;
+}
+
+/* ------------------------------- sub-cell refined centroids (an extension of Sec. 3.2 / Eq. 7) ---- */
+
+/*
+ * The paper's candidates are bin positions, so a candidate is off the voted centroid by up to half a bin.  The
+ * refinement keeps, next to every bin's count, the sum of the estimates that fell into it, and moves each peak to
+ * the mean estimate of its 3x3 neighbourhood (a strict peak has no other peak there, so those votes are its own).
+ *
+ * Sums are integers so that they do not depend on the order of addition: every estimate is taken as the fixed-point
+ * number rint(p * 2^24) (|p| <= 1: exact for |p| >= 1/4, otherwise rounded to 2^-24).
+ *   est  [B][H*W][2] binary32 estimates and cell [B][H*W] (-1 = no vote), as cpe_oracle_votes returns them
+ *   sums [B][cells][2] int64 (x, y)
+ */
+#define REFINE_SCALE 16777216.0 /* 2^24 */
+
+int cpe_oracle_vote_sums(const float* est, const int32_t* cell, int B, int H, int W, int cells, int64_t* sums) {
+  if (!est || !cell || !sums) return -1;
+  size_t HW = (size_t)H * W;
+  memset(sums, 0, sizeof(int64_t) * 2 * (size_t)cells * B);
+  for (size_t b = 0; b < (size_t)B; ++b)
+    for (size_t pix = 0; pix < HW; ++pix) {
+      int32_t c = cell[b * HW + pix];
+      if (c < 0) continue;
+      for (int a = 0; a < 2; ++a)
+        sums[(b * cells + (size_t)c) * 2 + a] += (int64_t)llrint((double)est[(b * HW + pix) * 2 + a] * REFINE_SCALE);
+    }
+  return 0;
+}
+
+/*
+ * One image: for each listed peak, mean = (sum over the 3x3 window of sums) / (2^24 * sum over it of votes), per
+ * axis, in binary64; the refined candidate is gamma(mean) of Eq. 2 (binary64 sin/cos, one rounding to binary32, the
+ * way the palette of Eq. 9 is made) and the refined centroid is mean in pixel units.
+ *   peak_emb [count][4F] (x block then y block), centroids [count][2], mean [count][2] (optional)
+ */
+int cpe_oracle_refined_peaks(const uint32_t* votes_img, const int64_t* sums_img, int bins_w, int bins_h,
+                             const int32_t* peak_cell, int count, int F, int H, int W, float* peak_emb,
+                             float* centroids, double* mean) {
+  if (!votes_img || !sums_img || !peak_cell || !peak_emb || !centroids) return -1;
+  for (int k = 0; k < count; ++k) {
+    int cx = peak_cell[k] % bins_w, cy = peak_cell[k] / bins_w;
+    int64_t s[2] = {0, 0}, n = 0;
+    for (int dy = -1; dy <= 1; ++dy)
+      for (int dx = -1; dx <= 1; ++dx) {
+        int x = cx + dx, y = cy + dy;
+        if (x < 0 || x >= bins_w || y < 0 || y >= bins_h) continue;
+        size_t c = (size_t)y * bins_w + x;
+        n += votes_img[c];
+        s[0] += sums_img[2 * c];
+        s[1] += sums_img[2 * c + 1];
+      }
+    double m[2];
+    for (int a = 0; a < 2; ++a) {
+      m[a] = (double)s[a] / ((double)n * REFINE_SCALE);
+      if (mean) mean[2 * k + a] = m[a];
+      for (int l = 0; l < F; ++l) {
+        double arg = ORACLE_PI * ldexp(1.0, l) * m[a];
+        peak_emb[(size_t)k * 4 * F + (size_t)a * 2 * F + 2 * l + 0] = (float)sin(arg);
+        peak_emb[(size_t)k * 4 * F + (size_t)a * 2 * F + 2 * l + 1] = (float)cos(arg);
+      }
+    }
+    centroids[2 * k + 0] = (float)(((m[0] + 1.0) * (double)W - 1.0) * 0.5);
+    centroids[2 * k + 1] = (float)(((m[1] + 1.0) * (double)H - 1.0) * 0.5);
+  }
   return 0;
 }

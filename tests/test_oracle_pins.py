@@ -605,3 +605,95 @@ def test_instance_masks_partition_the_labelled_pixels_and_count_them():
     assert np.array_equal(back, np.where(labels <= 5, labels, 0))
     assert oracle.instance_masks(labels, 7, want_planes=False)[0] is None
     assert np.array_equal(oracle.instance_masks(labels, 7, want_planes=False)[1][:, :5], pixels)
+
+
+# ---------------------------------------------------------------- sub-cell refined centroids
+
+def test_vote_sums_equal_a_numpy_scatter_add_of_fixed_point_estimates():
+    # definition: sums[cell] = sum of rint(p * 2^24) over the pixels that voted into the cell (integers: any order)
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=72, W=88, B=2, K=5, bins_w=24, bins_h=20)
+    fr = wl.make_frame(cfg, 3)
+    v = oracle.votes(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, want_est=True, want_cell=True)
+    got = oracle.vote_sums(v["est"], v["cell"], cfg.bins_w, cfg.bins_h)
+    want = np.zeros((cfg.B, cfg.bins_w * cfg.bins_h, 2), np.int64)
+    for b in range(cfg.B):
+        c = v["cell"][b].ravel()
+        take = c >= 0
+        fixed = np.rint(v["est"][b].reshape(-1, 2)[take].astype(np.float64) * 2.0 ** 24).astype(np.int64)
+        np.add.at(want[b], c[take], fixed)
+    assert np.array_equal(got.reshape(want.shape), want)
+    assert (got.reshape(want.shape)[v["votes"].reshape(cfg.B, -1) == 0] == 0).all()
+    # |p| <= 1 bounds every cell's sum by its count
+    assert (np.abs(got.reshape(want.shape)) <= v["votes"].reshape(cfg.B, -1, 1).astype(np.int64) << 24).all()
+
+
+def test_refined_peaks_recover_off_bin_centroids_of_clean_encodings():
+    # exact encodings of centroids placed anywhere inside a bin: every estimate equals the centroid (to binary32
+    # rounding of the estimate), so the mean does too, while the unrefined candidate is off by up to half a bin.
+    H, W, F, bw, bh = 64, 96, 4, 32, 32
+    boxes = [(0, 30, 0, 40), (0, 30, 40, 96), (30, 64, 0, 25), (30, 64, 25, 70), (34, 60, 72, 94)]
+    inst = _toy_instances(H, W, boxes)
+    cents = np.array([[-0.713, -0.801], [0.2291, -0.6502], [-0.8333, 0.5477], [-0.2412, 0.2468], [0.8, 0.74]])
+    emb = wl.encode(inst, cents, F, 0.0, None, np.float32)[None]
+    fg = (inst > 0).astype(np.uint8)[None]
+    res = oracle.decode_refined(emb, fg, bw, bh, T_v=8, K_max=16)
+    assert res["count"][0] == 5
+    lin = np.array([oracle.cell_of(cy, bh) * bw + oracle.cell_of(cx, bw) for cx, cy in cents])
+    order = np.argsort(lin)
+    assert res["peak_cell"][0, :5].tolist() == lin[order].tolist()
+    for j, k in enumerate(order):
+        want_px = ((cents[k, 0] + 1) * W - 1) / 2, ((cents[k, 1] + 1) * H - 1) / 2
+        np.testing.assert_allclose(res["centroids"][0, j], want_px, atol=2e-4)      # 2e-6 of the unit range
+        np.testing.assert_allclose(res["peak_emb"][0, j, :2 * F], gamma(cents[k, 0], F), atol=2e-6 * 2 ** F)
+        np.testing.assert_allclose(res["peak_emb"][0, j, 2 * F:], gamma(cents[k, 1], F), atol=2e-6 * 2 ** F)
+    relabel = np.zeros(6, np.int32)
+    relabel[order + 1] = np.arange(1, 6)
+    assert np.array_equal(res["labels"][0], relabel[inst])
+    assert res["best"][0][inst > 0].max() < 1e-4          # every pixel sits on its refined candidate
+    # the unrefined chain leaves a distance of the order of the bin offset
+    plain = oracle.decode(emb, fg, bw, bh, T_v=8, K_max=16)
+    assert plain["best"][0][inst > 0].max() > 0.05
+
+
+def test_refined_mean_pools_the_3x3_window_and_stays_on_the_unit_torus():
+    # hand-made maps: a blob straddling a cell border is pooled over the window; window clipped at the map edge
+    bw, bh, F, H, W = 6, 5, 3, 40, 60
+    V = np.zeros((bh, bw), np.uint32)
+    S = np.zeros((bh, bw, 2), np.int64)
+    one = 1 << 24
+    V[2, 2], S[2, 2] = 10, (int(10 * -0.10 * one), int(10 * 0.05 * one))
+    V[2, 3], S[2, 3] = 6, (int(6 * 0.02 * one), int(6 * 0.07 * one))
+    V[1, 2], S[1, 2] = 4, (int(4 * -0.12 * one), int(4 * -0.20 * one))
+    V[0, 5], S[0, 5] = 9, (int(9 * 0.90 * one), int(9 * -0.95 * one))      # corner cell: 4-cell window
+    V[4, 0], S[4, 0] = 1, (123, -456)                                      # outside both windows
+    pc = np.array([0 * bw + 5, 2 * bw + 2], np.int32)
+    r = oracle.refined_peaks(V, S, pc, F, H, W)
+    want1 = np.array([(10 * -0.10 + 6 * 0.02 + 4 * -0.12) / 20, (10 * 0.05 + 6 * 0.07 + 4 * -0.20) / 20])
+    np.testing.assert_allclose(r["mean"][0], [0.90, -0.95], atol=1e-7)
+    np.testing.assert_allclose(r["mean"][1], want1, atol=1e-7)
+    for k in range(2):
+        for a in range(2):
+            np.testing.assert_allclose(r["peak_emb"][k, a * 2 * F:(a + 1) * 2 * F], gamma(r["mean"][k, a], F),
+                                       atol=1.5e-7)
+        s, c = r["peak_emb"][k, 0::2].astype(np.float64), r["peak_emb"][k, 1::2].astype(np.float64)
+        np.testing.assert_allclose(s * s + c * c, 1.0, atol=3e-7)
+        np.testing.assert_allclose(r["centroids"][k], [((r["mean"][k, 0] + 1) * W - 1) / 2,
+                                                       ((r["mean"][k, 1] + 1) * H - 1) / 2], rtol=1e-6)
+
+
+def test_explicit_candidates_reduce_to_the_palette_case_and_to_brute_force():
+    # handing the palette rows in explicitly changes nothing; arbitrary rows agree with a direct Eq. 7 in numpy
+    emb, fg, cells, bw, bh, F = _tiny_problem(5)
+    Pw, Ph = oracle.palette(bw, F), oracle.palette(bh, F)
+    rows = np.concatenate([Pw[cells % bw], Ph[cells // bw]], axis=1)
+    a0 = oracle.assign_image(emb, fg, bw, bh, cells)
+    a1 = oracle.assign_image(emb, fg, bw, bh, cells, peak_emb=rows)
+    assert np.array_equal(a0["labels"], a1["labels"]) and np.array_equal(a0["best"], a1["best"])
+    rng = np.random.default_rng(11)
+    rows2 = rng.standard_normal(rows.shape).astype(np.float32)
+    a2 = oracle.assign_image(emb, None, bw, bh, cells, peak_emb=rows2)
+    x = emb.astype(np.float64).reshape(4 * F, -1).T                                  # [HW, 4F]
+    d = (np.sqrt(((x[:, None, :2 * F] - rows2[None, :, :2 * F].astype(np.float64)) ** 2).sum(-1)) +
+         np.sqrt(((x[:, None, 2 * F:] - rows2[None, :, 2 * F:].astype(np.float64)) ** 2).sum(-1)))
+    assert np.array_equal(a2["labels"].ravel(), d.argmin(1) + 1)
+    np.testing.assert_allclose(a2["best"].ravel(), d.min(1), rtol=1e-12)
