@@ -60,9 +60,19 @@ enum {
                                  filtering with the tensor cores first; same results, for cross-checking */
   CPE_FLAG_FILTER_ASSIGN = 8u,/* use the tensor-core filtered kernel for every image, however few peaks it has
                                  (by default images with few peaks take the all-pairs kernel); same results   */
-  CPE_FLAG_KEEP_VOTES = 4u    /* leave the vote map readable after the decode (CPE_INT_VOTES).  Without it the
+  CPE_FLAG_KEEP_VOTES = 4u,   /* leave the vote map readable after the decode (CPE_INT_VOTES).  Without it the
                                  last kernel of a decode re-zeroes the map for the next decode, which saves the
                                  clearing pass at the start; with it every decode starts with that pass.       */
+  CPE_FLAG_REFINE = 16u       /* sub-cell refined centroids (an extension: the paper's candidates of Eq. 7 are the
+                                 bin positions of Eq. 9, up to half a bin off the voted centroid).  Next to its
+                                 count every bin keeps the sum of the estimates that fell into it, as integers
+                                 rint(p * 2^24) so that the sums do not depend on the order of addition
+                                 (CPE_INT_VOTE_SUMS).  A peak is then placed at the mean estimate of its 3x3
+                                 neighbourhood, mean = (sum of the sums) / (2^24 * sum of the counts) in binary64:
+                                 out_centroids holds that mean in pixel units and the peak's candidate embedding
+                                 is gamma(mean) of Eq. 2 (binary64 sin/cos, rounded once) instead of the palette
+                                 rows.  Peak detection and everything else are unchanged.  Needs a larger
+                                 workspace (16 bytes per bin and image) and one clearing pass per decode.      */
 };
 
 /* bits of the per-image device status words */
@@ -91,14 +101,17 @@ enum {
   CPE_INT_VOTES = 0,        /* uint32 [B][bins_h][bins_w]       hard-vote map (CPE_FLAG_KEEP_VOTES)  */
   CPE_INT_PEAK_CELLS = 1,   /* int32  [B][max_instances]        linear bin cy*bins_w+cx, ascending */
   CPE_INT_PEAK_VOTES = 2,   /* uint32 [B][max_instances]        votes of each kept peak         */
-  CPE_INT_PEAK_EMB = 3,     /* float  [B][max_instances][4F]    concat(P_w[cx], P_h[cy])        */
+  CPE_INT_PEAK_EMB = 3,     /* float  [B][max_instances][4F]    concat(P_w[cx], P_h[cy]); with
+                                                                CPE_FLAG_REFINE gamma of the refined position */
   CPE_INT_PALETTE_W = 4,    /* float  [bins_w][2F]              Eq. 9                           */
   CPE_INT_PALETTE_H = 5,    /* float  [bins_h][2F]                                              */
   CPE_INT_BEST_SCORE = 6,   /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
   CPE_INT_SECOND_SCORE = 7, /* float  [B][H][W]  (CPE_FLAG_WRITE_SCORES) +inf where none        */
   CPE_INT_STATUS = 8,       /* uint32 [B]                       CPE_STATUS_* bits of each image      */
   CPE_INT_COUNTERS = 9,     /* uint32 [B][CPE_CNT_N]                                            */
-  CPE_INT_N = 10
+  CPE_INT_VOTE_SUMS = 10,   /* int64  [B][bins_h][bins_w][2]    fixed-point (2^-24) sums of the x and y
+                                                                estimates per bin (CPE_FLAG_REFINE)  */
+  CPE_INT_N = 11
 };
 
 /* stages reported by cpe_profile_decode */

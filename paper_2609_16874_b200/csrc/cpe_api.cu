@@ -61,7 +61,7 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
 
 template <typename T>
 int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                       uint32_t* votes, uint32_t* acc) {
+                       uint32_t* votes, uint32_t* acc, long long* sums) {
   const T* e = static_cast<const T*>(emb);
   constexpr int V = cpe::Elem<T>::kVec;
   // 128-bit plane loads: every plane of every image must start on a 16-byte boundary
@@ -70,9 +70,13 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
   if (vec) {
     const long long groups = (long long)HW / V;
     dim3 grid((unsigned)((groups + cpe::kVecGroups - 1) / cpe::kVecGroups), (unsigned)B);
-#define CPE_LAUNCH_VOTE(FT_)                                                                                   \
-  cpe::decode_vote_vec_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,      \
-                                                                         p->bins_h, votes, acc)
+#define CPE_LAUNCH_VOTE(FT_)                                                                                          \
+  if (sums)                                                                                                            \
+    cpe::decode_vote_vec_kernel<T, FT_, true><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,     \
+                                                                                 p->bins_h, votes, acc, sums);        \
+  else                                                                                                                 \
+    cpe::decode_vote_vec_kernel<T, FT_, false><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,    \
+                                                                                  p->bins_h, votes, acc, nullptr)
     switch (F) {
       case 4: CPE_LAUNCH_VOTE(4); break;
       case 8: CPE_LAUNCH_VOTE(8); break;
@@ -83,9 +87,13 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
     // 64-bit mask loads need every image's mask to start on an 8-byte boundary
     const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
     dim3 grid((unsigned)(((long long)HW + cpe::kVoteSpan - 1) / cpe::kVoteSpan), (unsigned)B);
-#define CPE_LAUNCH_VOTE(FT_)                                                                                       \
-  cpe::decode_vote_scalar_kernel<T, FT_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, F, p->levels, p->bins_w,    \
-                                                                            p->bins_h, vec_mask, votes, acc)
+#define CPE_LAUNCH_VOTE(FT_)                                                                                             \
+  if (sums)                                                                                                               \
+    cpe::decode_vote_scalar_kernel<T, FT_, true><<<grid, cpe::kVoteThreads, 0, st>>>(                                     \
+        e, fg, HW, F, p->levels, p->bins_w, p->bins_h, vec_mask, votes, acc, sums);                                       \
+  else                                                                                                                    \
+    cpe::decode_vote_scalar_kernel<T, FT_, false><<<grid, cpe::kVoteThreads, 0, st>>>(                                    \
+        e, fg, HW, F, p->levels, p->bins_w, p->bins_h, vec_mask, votes, acc, nullptr)
     switch (F) {
       case 4: CPE_LAUNCH_VOTE(4); break;
       case 8: CPE_LAUNCH_VOTE(8); break;
@@ -300,10 +308,13 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_CLEAR], st));
   // Normally the map is already zero (cpe_init_workspace, then the previous decode's last kernel).
   if (keep_votes) CPE_CUDA(cudaMemsetAsync(ws + L.votes, 0, L.votes_end - L.votes, st));
+  // The per-bin sums of the refinement stay readable after the decode, so they are cleared here.
+  long long* sums = (p->flags & CPE_FLAG_REFINE) ? reinterpret_cast<long long*>(ws + L.sums) : nullptr;
+  if (sums) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
-  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, acc)
-                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, acc);
+  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, acc, sums)
+                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, acc, sums);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
@@ -316,7 +327,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     cpe::peaks_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
                                                           (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W,
                                                           pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids,
-                                                          out_count, acc, counters, status);
+                                                          out_count, acc, counters, status, sums);
     CPE_CUDA(cudaGetLastError());
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
@@ -424,6 +435,11 @@ int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int 
       break;
     case CPE_INT_STATUS: off = L.status; sz = 4 * (size_t)B; break;
     case CPE_INT_COUNTERS: off = L.counters; sz = 4 * (size_t)CPE_CNT_N * B; break;
+    case CPE_INT_VOTE_SUMS:
+      if (!(params->flags & CPE_FLAG_REFINE)) return CPE_ERR_WHICH;
+      off = L.sums;
+      sz = 16 * (size_t)L.cells * B;
+      break;
     default: return CPE_ERR_WHICH;
   }
   *device_ptr = static_cast<char*>(params->workspace) + off;

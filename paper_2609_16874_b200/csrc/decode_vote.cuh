@@ -37,6 +37,36 @@ __device__ __forceinline__ void vote_cache_add(uint32_t* keys, uint32_t* cnts, u
   atomicAdd(&votes_img[cell], n);
 }
 
+// Sub-cell refinement: next to the count, a bin also gets the sum of the estimates that fell into it, as integers so
+// that the result does not depend on the order of addition.  An estimate p in [-1, 1) is taken as rint(p * 2^24)
+// (exact for |p| >= 1/4).  Lanes of the warp that name the same bin are summed first (at most 32 x 2^24 fits in 32
+// bits), then one lane per distinct bin adds the pair to the bin's 64-bit sums in global memory (fire-and-forget
+// reductions).  Called by all 32 lanes; cell < 0 = this lane has no vote.
+constexpr float kRefineScale = 16777216.0f;  // 2^24
+
+__device__ __forceinline__ void vote_sums_add(long long* __restrict__ sums_img, int cell, float px, float py,
+                                              bool one_bin, uint32_t voters) {
+  const int lane = threadIdx.x & 31;
+  const int fx = cell >= 0 ? __float2int_rn(__fmul_rn(px, kRefineScale)) : 0;
+  const int fy = cell >= 0 ? __float2int_rn(__fmul_rn(py, kRefineScale)) : 0;
+  if (one_bin) {
+    const int sx = __reduce_add_sync(0xffffffffu, fx), sy = __reduce_add_sync(0xffffffffu, fy);
+    if (lane == __ffs(voters) - 1) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(sums_img + 2 * (size_t)cell), (unsigned long long)(long long)sx);
+      atomicAdd(reinterpret_cast<unsigned long long*>(sums_img + 2 * (size_t)cell + 1),
+                (unsigned long long)(long long)sy);
+    }
+  } else {
+    const uint32_t same = __match_any_sync(0xffffffffu, cell);   // the lanes without a vote form a group of their own
+    const int sx = __reduce_add_sync(same, fx), sy = __reduce_add_sync(same, fy);
+    if (cell >= 0 && lane == __ffs(same) - 1) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(sums_img + 2 * (size_t)cell), (unsigned long long)(long long)sx);
+      atomicAdd(reinterpret_cast<unsigned long long*>(sums_img + 2 * (size_t)cell + 1),
+                (unsigned long long)(long long)sy);
+    }
+  }
+}
+
 // Compacts the participating pixels of the CTA's span into s_list (offsets within the span, ascending).
 // Returns the number of entries.  `fg` may be NULL (all pixels participate).  Uses s_scan[9] as scratch.
 __device__ __forceinline__ int compact_span(const uint8_t* __restrict__ fg_img, long long span0, int HW, bool vec_mask,
@@ -92,11 +122,11 @@ __device__ __forceinline__ int compact_span(const uint8_t* __restrict__ fg_img, 
 }
 
 // Scalar-load variant: any F, any alignment, any H*W.  FT > 0 fixes F at compile time.
-template <typename T, int FT>
+template <typename T, int FT, bool REFINE>
 __global__ void __launch_bounds__(kVoteThreads)
 decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
                    int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
-                   uint32_t* __restrict__ acc) {
+                   uint32_t* __restrict__ acc, long long* __restrict__ sums) {
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
   const int b = blockIdx.y;
@@ -106,6 +136,7 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
   const T* e = emb + (size_t)b * 4 * F * plane;
   const uint8_t* fg_img = fg ? fg + (size_t)b * plane : nullptr;
   uint32_t* votes_img = votes + (size_t)b * bins_w * bins_h;
+  long long* sums_img = REFINE ? sums + (size_t)b * bins_w * bins_h * 2 : nullptr;
   const long long span0 = (long long)blockIdx.x * kVoteSpan;
 
   __shared__ uint32_t s_keys[kHashSlots];
@@ -165,10 +196,13 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 #pragma unroll
     for (int q = 0; q < kVotePix; ++q) {
       int cell = -1;
+      float ux = 0.0f, uy = 0.0f;
       if (have[q]) {
         if (fin[q] == fin[q]) {
-          const int cx = cell_of(wrap_unit(__fmul_rn(p[q][0], unscale)), half_w, bins_w);
-          const int cy = cell_of(wrap_unit(__fmul_rn(p[q][1], unscale)), half_h, bins_h);
+          ux = wrap_unit(__fmul_rn(p[q][0], unscale));
+          uy = wrap_unit(__fmul_rn(p[q][1], unscale));
+          const int cx = cell_of(ux, half_w, bins_w);
+          const int cy = cell_of(uy, half_h, bins_h);
           cell = cy * bins_w + cx;
           ++voted;
         } else {
@@ -180,7 +214,9 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
       if (voters) {
         const int leader = __ffs(voters) - 1;
         const int ref = __shfl_sync(0xffffffffu, cell, leader);
-        if (__all_sync(0xffffffffu, cell < 0 || cell == ref)) {
+        const bool one_bin = __all_sync(0xffffffffu, cell < 0 || cell == ref);
+        if constexpr (REFINE) vote_sums_add(sums_img, cell, ux, uy, one_bin, voters);
+        if (one_bin) {
           if (lane == leader) vote_cache_add(s_keys, s_cnts, (uint32_t)ref, (uint32_t)__popc(voters), votes_img);
         } else {
           const uint32_t same = __match_any_sync(0xffffffffu, cell);
@@ -219,10 +255,11 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 constexpr int kVecGroups = 256;      // groups per CTA
 constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight together (2 loads each)
 
-template <typename T, int FT>
+template <typename T, int FT, bool REFINE>
 __global__ void __launch_bounds__(kVoteThreads, 3)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
-                       int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc) {
+                       int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
+                       long long* __restrict__ sums) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int F = FT;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
@@ -231,6 +268,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
   const size_t plane = (size_t)HW;
   const T* e = emb + (size_t)b * 4 * F * plane;
   uint32_t* votes_img = votes + (size_t)b * bins_w * bins_h;
+  long long* sums_img = REFINE ? sums + (size_t)b * bins_w * bins_h * 2 : nullptr;
   const long long span0 = (long long)blockIdx.x * kVecGroups * VEC;
 
   __shared__ uint32_t s_keys[kHashSlots];
@@ -351,8 +389,10 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
       int cell = -1;
       if (have && ((take >> j) & 1u)) {
         if ((ok_both >> j) & 1u) {
-          const int cx = cell_of(wrap_unit(px), half_w, bins_w);
-          const int cy = cell_of(wrap_unit(py), half_h, bins_h);
+          px = wrap_unit(px);
+          py = wrap_unit(py);
+          const int cx = cell_of(px, half_w, bins_w);
+          const int cy = cell_of(py, half_h, bins_h);
           cell = cy * bins_w + cx;
           ++voted;
         } else {
@@ -363,7 +403,9 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
       if (voters) {
         const int leader = __ffs(voters) - 1;
         const int ref = __shfl_sync(0xffffffffu, cell, leader);
-        if (__all_sync(0xffffffffu, cell < 0 || cell == ref)) {
+        const bool one_bin = __all_sync(0xffffffffu, cell < 0 || cell == ref);
+        if constexpr (REFINE) vote_sums_add(sums_img, cell, px, py, one_bin, voters);
+        if (one_bin) {
           if (lane == leader) vote_cache_add(s_keys, s_cnts, (uint32_t)ref, (uint32_t)__popc(voters), votes_img);
         } else {
           const uint32_t same = __match_any_sync(0xffffffffu, cell);

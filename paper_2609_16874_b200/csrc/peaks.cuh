@@ -7,6 +7,7 @@
 namespace cpe {
 
 constexpr int kPeakThreads = 1024;   // wide CTAs: the last one of an image does the whole compaction
+constexpr int kRefineChunk = 1024;     // peaks whose refined positions are staged in shared memory at a time
 
 // Phase 1 (every CTA): one thread per bin, one warp per 32 consecutive bins; the warp's ballot is one word
 // of the peak indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it
@@ -18,12 +19,18 @@ constexpr int kPeakThreads = 1024;   // wide CTAs: the last one of an image does
 // order, so the list is ascending in the linear bin index and, when there are more than K_max peaks, exactly
 // the first K_max are kept.  Then the centroids (bin positions of Eq. 9 in pixel units) and the peak
 // embeddings concat(P_w[cx], P_h[cy]) are gathered, and the image's counters and status word are written.
+//
+// With `sums` (sub-cell refinement; int64 [B][cells][2], the fixed-point sums of the estimates that fell into each
+// bin) a peak is moved from its bin position to the mean estimate of its 3x3 neighbourhood -- a strict peak has no
+// other peak there, so those votes are its own -- and its embedding is gamma(mean) of Eq. 2, evaluated in binary64
+// and rounded once, the way the palette rows are made.
 __global__ void __launch_bounds__(kPeakThreads)
 peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
              uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
-             uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status) {
+             uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
+             const long long* __restrict__ sums) {
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int cells = bins_w * bins_h;
@@ -141,6 +148,47 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
 
   const int D = 4 * F;
   float* pe = peak_emb + (size_t)b * K_max * D;
+  if (sums) {
+    __shared__ double s_mean[2 * kRefineChunk];
+    const long long* S = sums + (size_t)b * cells * 2;
+    for (int k0 = 0; k0 < count; k0 += kRefineChunk) {
+      const int nk = min(kRefineChunk, count - k0);
+      for (int i = tid; i < 2 * nk; i += kPeakThreads) {       // (peak, axis): pooled mean of the 3x3 window
+        const int k = k0 + (i >> 1), axis = i & 1;
+        const int lin = pc[k];
+        const int cy = lin / bins_w, cx = lin - cy * bins_w;
+        long long s = 0, n = 0;
+#pragma unroll
+        for (int dy = -1; dy <= 1; ++dy) {
+#pragma unroll
+          for (int dx = -1; dx <= 1; ++dx) {
+            const int ny = cy + dy, nx = cx + dx;
+            if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+            const int nlin = ny * bins_w + nx;
+            n += (long long)V[nlin];
+            s += __ldcg(S + 2 * (size_t)nlin + axis);
+          }
+        }
+        const double m = __ddiv_rn((double)s, __dmul_rn((double)n, 16777216.0));
+        s_mean[i] = m;
+        // pixel centres sit at x = -1 + (2 col + 1)/W
+        out_centroids[((size_t)b * K_max + k) * 2 + axis] =
+            (float)__dmul_rn(__dadd_rn(__dmul_rn(__dadd_rn(m, 1.0), (double)(axis ? H : W)), -1.0), 0.5);
+      }
+      __syncthreads();
+      for (int i = tid; i < 2 * F * nk; i += kPeakThreads) {   // (peak, axis, harmonic): sin and cos of pi 2^l mean
+        const int kk = i / (2 * F), r = i - kk * 2 * F;
+        const int axis = r / F, l = r - axis * F;
+        double sn, cs;
+        sincospi(scalbn(s_mean[2 * kk + axis], l), &sn, &cs);
+        float* o = pe + (size_t)(k0 + kk) * D + axis * 2 * F + 2 * l;
+        o[0] = (float)sn;
+        o[1] = (float)cs;
+      }
+      __syncthreads();
+    }
+    return;
+  }
   for (int i = tid; i < count * D; i += kPeakThreads) {
     const int k = i / D, c = i - k * D;
     const int lin = pc[k];

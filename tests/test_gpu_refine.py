@@ -1,0 +1,136 @@
+"""Sub-cell refined centroids (CPE_FLAG_REFINE): CUDA path vs CPU oracle through the C ABI.  Needs a B200.
+
+Integer work (votes, per-bin fixed-point sums, peak list, counts) must agree bit for bit; so must the refined
+centroids, which both sides derive from the same integers with the same correctly rounded binary64 operations.
+The refined candidate embeddings go through sin/cos of different libraries: one unit in the last place of
+binary32.  Labels and scores follow the usual rule (exact except where the oracle's top-2 margin is a near-tie).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_16874_b200 import binding as cb
+from paper_2609_16874_b200 import workloads as wl
+
+from gpu_util import REL, compare_labels
+
+pytestmark = pytest.mark.gpu
+
+EMB_ATOL = 1.5e-7     # |sin|, |cos| <= 1: one binary32 ulp below 1 is 6e-8, two libraries may round apart by one
+
+
+def run_refined(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, scores=True, mode="direct", **flags):
+    import torch
+    B, D, H, W = emb.shape
+    F = D // 4
+    dec = cb.Decoder(B, H, W, F, "f32" if emb.dtype == np.float32 else "f16", bins_w, bins_h, T_v, float(tau), K_max,
+                     0, write_scores=scores, keep_votes=True, refine=True, **flags)
+    d_emb = torch.from_numpy(emb).cuda()
+    d_fg = None if fg is None else torch.from_numpy(np.ascontiguousarray(fg, np.uint8)).cuda()
+    if mode == "direct":
+        dec.decode(d_emb, d_fg)
+        dec.decode(d_emb, d_fg)        # the sums are cleared at the start of every decode
+    else:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = dec.capture(d_emb, d_fg, stream=side)
+        dec.labels.fill_(-7)
+        dec.replay(g, stream=side)
+        dec.replay(g, stream=side)
+        side.synchronize()
+    torch.cuda.synchronize()
+    out = {
+        "labels": dec.labels.cpu().numpy(),
+        "centroids": dec.centroids.cpu().numpy(),
+        "count": dec.count.cpu().numpy(),
+        "votes": dec.intermediate(cb.CPE_INT_VOTES).cpu().numpy().view(np.uint32),
+        "sums": dec.intermediate(cb.CPE_INT_VOTE_SUMS).cpu().numpy(),
+        "peak_cell": dec.intermediate(cb.CPE_INT_PEAK_CELLS).cpu().numpy(),
+        "peak_emb": dec.intermediate(cb.CPE_INT_PEAK_EMB).cpu().numpy(),
+        "status": int(np.bitwise_or.reduce(dec.intermediate(cb.CPE_INT_STATUS).cpu().numpy())),
+        "counters": dec.intermediate(cb.CPE_INT_COUNTERS).cpu().numpy().astype(np.int64),
+    }
+    if scores:
+        out["best"] = dec.intermediate(cb.CPE_INT_BEST_SCORE).cpu().numpy()
+        out["second"] = dec.intermediate(cb.CPE_INT_SECOND_SCORE).cpu().numpy()
+    dec.close()
+    return out
+
+
+def compare_refined(gpu, ora):
+    assert not (gpu["status"] & cb.CPE_STATUS_INTERNAL), hex(gpu["status"])
+    assert np.array_equal(gpu["votes"], ora["votes"]), "vote map differs"
+    assert np.array_equal(gpu["sums"], ora["sums"]), "per-bin sums differ"
+    assert np.array_equal(gpu["count"], ora["count"])
+    for b in range(len(ora["count"])):
+        n = int(ora["count"][b])
+        assert np.array_equal(gpu["peak_cell"][b, :n], ora["peak_cell"][b, :n])
+        assert np.array_equal(gpu["centroids"][b, :n].view(np.uint32), ora["centroids"][b, :n].view(np.uint32))
+        np.testing.assert_allclose(gpu["peak_emb"][b, :n], ora["peak_emb"][b, :n], rtol=0, atol=EMB_ATOL)
+    for c in (cb.CPE_CNT_VOTING, cb.CPE_CNT_NONFINITE, cb.CPE_CNT_RAW_PEAKS, cb.CPE_CNT_TRUNCATED):
+        assert np.array_equal(gpu["counters"][:, c], ora["counters"][:, c]), c
+    return compare_labels(gpu["labels"], gpu.get("best"), gpu.get("second"), ora["labels"], ora["best"],
+                          ora["second"])
+
+
+CASES = [
+    ("c1", dict()),                                                        # vector-load vote kernel, fp32
+    ("c1", dict(H=67, W=93)),                                              # scalar-load vote kernel
+    ("c2", dict(H=192, W=256, K=12)),
+    ("c3", dict(H=256, W=384, K=24, bins_w=96, bins_h=64)),                # fp16
+    ("c3", dict(H=99, W=121, K=8, bins_w=64, bins_h=32)),                  # fp16, scalar path
+    ("c4", dict(B=3, H=160, W=168, K=30, bins_w=40, bins_h=40)),           # batch, touching instances
+    ("c5", dict(H=256, W=256, K=40, bins_w=128, bins_h=128)),              # F = 16
+]
+
+
+@pytest.mark.parametrize("name,over", CASES, ids=[f"{n}-{i}" for i, (n, _) in enumerate(CASES)])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_refined_decode_matches_oracle(name, over, mode):
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 0)
+    ora = oracle.decode_refined(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    assert ora["count"].min() >= 1
+    gpu = run_refined(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, mode=mode)
+    rep = compare_refined(gpu, ora)
+    # production configuration (no scores) and the tensor-core filtered kernel forced on
+    fast = run_refined(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=False, mode=mode)
+    compare_refined(fast, ora)
+    for sc in (True, False):
+        filt = run_refined(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=sc,
+                           mode=mode, filter_assign=True)
+        compare_refined(filt, ora)
+    print(name, over, rep)
+
+
+def test_refined_centroids_are_closer_to_the_truth_than_bin_centres():
+    # what the mode is for: on the noisy c2 recipe the refined centroid is well inside a bin width of the instance's
+    # true centroid, and the pixels' distances to their candidate drop
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=256, W=256, K=10)
+    fr = wl.make_frame(cfg, 4)
+    gpu = run_refined(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    plain = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    n = int(gpu["count"][0])
+    assert n == int(plain["count"][0]) >= 1
+    truth = fr["centroids"][0]                                   # [K, 2] in [-1, 1)
+    truth_px = np.stack([((truth[:, 0] + 1) * cfg.W - 1) / 2, ((truth[:, 1] + 1) * cfg.H - 1) / 2], 1)
+
+    def err(cent):
+        d = np.linalg.norm(cent[:, None, :] - truth_px[None], axis=2)
+        return np.nanmin(d, axis=1)
+    e_ref, e_bin = err(gpu["centroids"][0, :n]), err(plain["centroids"][0, :n])
+    assert np.median(e_ref) < 0.5 * np.median(e_bin)
+    fgm = fr["fg"][0] > 0
+    assert np.median(gpu["best"][0][fgm]) < np.median(plain["best"][0][fgm])
+
+
+def test_refine_intermediate_needs_the_flag_and_workspace_grows_by_the_sums():
+    p0 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, 0)
+    p1 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, cb.CPE_FLAG_REFINE)
+    n0, n1 = cb.cpe_workspace_size(2, 96, 128, 4, p0), cb.cpe_workspace_size(2, 96, 128, 4, p1)
+    assert n1 - n0 == 16 * 64 * 48 * 2
+    import torch
+    ws = torch.empty(n0, dtype=torch.uint8, device="cuda")
+    p0.workspace, p0.workspace_bytes = ws.data_ptr(), n0
+    rc, _, _ = cb.cpe_get_intermediate(p0, cb.CPE_INT_VOTE_SUMS, 2, 96, 128, 4)
+    assert rc == cb.CPE_ERR_WHICH
