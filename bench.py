@@ -393,6 +393,11 @@ def run_ours(args, cfg):
             except Exception as exc:   # a parity-test workload must not take the headline line down with it
                 others[name] = {"error": repr(exc)}
         line["other_configs"] = others
+        try:   # the same decode with sub-cell refined centroids (per-bin sums, gamma(mean) candidates)
+            line["refined_centroids"] = {n: measure_other(wl.CONFIGS[n], 50, 5, dev, refine=True)
+                                         for n in sorted({cfg.name, "c3", "c5"})}
+        except Exception as exc:
+            line["refined_centroids"] = {"error": repr(exc)}
         try:
             line["soft_votes"] = measure_soft_votes(cfg, max(20, min(K, 100)), max(3, min(Wm, 10)), dev)
         except Exception as exc:
@@ -409,8 +414,9 @@ def run_ours(args, cfg):
     dist_util.shutdown()
 
 
-def measure_other(cfg, steps, warmup, dev):
-    """Graph-replay timing of one more workload (no host leg, no CPU baseline): p50, MP/s, per-stage times."""
+def measure_other(cfg, steps, warmup, dev, refine=False):
+    """Graph-replay timing of one more workload (no host leg, no CPU baseline): p50, MP/s, per-stage times.
+    `refine`: with sub-cell refined centroids (CPE_FLAG_REFINE)."""
     import torch
     from paper_2609_16874_b200 import binding as cb
     n_frames = frames_needed(cfg)
@@ -418,7 +424,8 @@ def measure_other(cfg, steps, warmup, dev):
     d_emb = [torch.from_numpy(f["emb"]).to(dev) for f in frames]
     d_fg = [torch.from_numpy(f["fg"]).to(dev) for f in frames]
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if n_frames * cfg.emb_bytes < 2 * L2_BYTES else None
-    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev,
+                     refine=refine)
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         graphs = [dec.capture(d_emb[i], d_fg[i], stream=stream) for i in range(n_frames)]
