@@ -82,6 +82,7 @@ assign_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW,
               const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau,
               int32_t* __restrict__ labels, float* __restrict__ best, float* __restrict__ second,
               uint32_t* __restrict__ counters, uint32_t* __restrict__ votes, int cells, int k_limit) {
+  grid_dependency_sync();
   constexpr int DT = FT > 0 ? 4 * FT : 64;
   const int F = FT > 0 ? FT : F_rt;
   const int D = 4 * F;

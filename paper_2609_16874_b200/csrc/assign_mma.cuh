@@ -869,6 +869,7 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
                   int peak_cap, int span, int vec_mask, int vec_gather, int32_t* __restrict__ labels, float* __restrict__ best,
                   float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
                   uint32_t* __restrict__ votes, int cells, int k_min) {
+  grid_dependency_sync();
   assign_mma_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status_all, votes, cells, k_min);
 }
 

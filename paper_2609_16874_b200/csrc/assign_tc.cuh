@@ -1038,6 +1038,7 @@ assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, 
                      uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all, uint32_t* __restrict__ votes, int cells,
                      int k_min, uint32_t* __restrict__ acc) {
   static_assert(kTcThreads == kAmThreads, "both bodies run with the same block size");
+  grid_dependency_sync();
   if (count_ptr[blockIdx.y] <= tc_k_max)
     assign_tc_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, tc_peak_cap, tc_vec_mask, labels,
                                  best, second, counters, status_all, votes, cells, k_min, tc_k_max, acc);

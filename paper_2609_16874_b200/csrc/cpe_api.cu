@@ -59,6 +59,25 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
   return CPE_OK;
 }
 
+// Launch of a kernel that consumes what the kernel before it in the stream wrote, with programmatic stream
+// serialisation: its CTAs may be scheduled while the predecessor is still running and wait on the device
+// (grid_dependency_sync at the top of every kernel of the chain).  CPE_PDL=0 in the environment launches plainly.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+  static const bool plain = [] { const char* e = getenv("CPE_PDL"); return e && e[0] == '0'; }();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = plain ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 template <typename T>
 int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                        uint32_t* votes, uint32_t* acc, long long* sums) {
@@ -127,10 +146,9 @@ int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int
   const long long n_blocks = ((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads;
   const long long per_image = std::max(1, (8 * sm_count() + B - 1) / B);
   dim3 grid((unsigned)std::min(n_blocks, per_image), (unsigned)B);
-#define CPE_LAUNCH_ASSIGN(FT_)                                                                                  \
-  cpe::assign_kernel<T, FT_><<<grid, cpe::kAssignThreads, 0, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, \
-                                                                  p->tau, labels, best, second, counters, votes_to_zero, cells, \
-                                                                  k_limit)
+#define CPE_LAUNCH_ASSIGN(FT_)                                                                                     \
+  CPE_CUDA(launch_dependent(cpe::assign_kernel<T, FT_>, grid, cpe::kAssignThreads, 0, st, e, fg, HW, F, p->max_instances, \
+                            peak_emb, count, p->tau, labels, best, second, counters, votes_to_zero, cells, k_limit))
   switch (F) {
     case 4: CPE_LAUNCH_ASSIGN(4); break;
     case 8: CPE_LAUNCH_ASSIGN(8); break;
@@ -169,10 +187,9 @@ int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, i
   dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
   const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
   const int need_exact = p->tau < INFINITY ? 1 : 0;
-  kern<<<grid, cpe::kAmThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact,
-                                            peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status,
-                                            votes_to_zero,
-                                            cells, k_min);
+  CPE_CUDA(launch_dependent(kern, grid, cpe::kAmThreads, smem, st, e, fg, HW, F, p->max_instances, peak_emb, count, p->tau,
+                            need_exact, peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status,
+                            votes_to_zero, cells, k_min));
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -213,9 +230,9 @@ int launch_assign_filter_t(cudaStream_t st, const T* e, const uint8_t* fg, int B
   dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
   const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
   const int need_exact = p->tau < INFINITY ? 1 : 0;
-  kern<<<grid, cpe::kTcThreads, smem, st>>>(e, fg, HW, F, p->max_instances, peak_emb, count, p->tau, need_exact, tc_cap, tc_k_max,
-                                            vec_mask, mma_cap, span, vec_mask, vec_gather, labels, best, second, counters,
-                                            status, votes_to_zero, cells, k_min, acc);
+  CPE_CUDA(launch_dependent(kern, grid, cpe::kTcThreads, smem, st, e, fg, HW, F, p->max_instances, peak_emb, count, p->tau,
+                            need_exact, tc_cap, tc_k_max, vec_mask, mma_cap, span, vec_mask, vec_gather, labels, best, second,
+                            counters, status, votes_to_zero, cells, k_min, acc));
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -324,10 +341,9 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     // small maps: one CTA per image does both phases without the cross-CTA hand-over
     const int ctas = L.words <= 8 * warps_per_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
     dim3 grid((unsigned)ctas, (unsigned)B);
-    cpe::peaks_kernel<<<grid, cpe::kPeakThreads, 0, st>>>(votes, p->bins_w, p->bins_h, L.words,
-                                                          (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W,
-                                                          pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids,
-                                                          out_count, acc, counters, status, sums);
+    CPE_CUDA(launch_dependent(cpe::peaks_kernel, grid, cpe::kPeakThreads, 0, st, votes, p->bins_w, p->bins_h, L.words,
+                              (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W, pal_w, pal_h, peak_cell,
+                              peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums));
     CPE_CUDA(cudaGetLastError());
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;

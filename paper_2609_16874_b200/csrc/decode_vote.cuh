@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(kVoteThreads)
 decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
                    int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
                    uint32_t* __restrict__ acc, long long* __restrict__ sums) {
+  grid_dependency_sync();
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
   const int b = blockIdx.y;
@@ -260,6 +261,7 @@ __global__ void __launch_bounds__(kVoteThreads, 3)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
                        int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
                        long long* __restrict__ sums) {
+  grid_dependency_sync();
   constexpr int VEC = Elem<T>::kVec;
   constexpr int F = FT;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
