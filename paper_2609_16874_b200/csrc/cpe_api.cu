@@ -59,6 +59,8 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
   return CPE_OK;
 }
 
+int sm_count();
+
 // Launch of a kernel that consumes what the kernel before it in the stream wrote, with programmatic stream
 // serialisation: its CTAs may be scheduled while the predecessor is still running and wait on the device
 // (grid_dependency_sync at the top of every kernel of the chain).  CPE_PDL=0 in the environment launches plainly.
@@ -88,20 +90,29 @@ int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                    (F == 4 || F == 8 || F == 16);
   if (vec) {
     const long long groups = (long long)HW / V;
-    dim3 grid((unsigned)((groups + cpe::kVecGroups - 1) / cpe::kVecGroups), (unsigned)B);
+    // the largest span that still gives one full wave of CTAs (three resident per SM), else the smallest
+    const long long wave = 3LL * sm_count();
+    const int span = (groups + 255) / 256 * B >= wave ? 256 : (groups + 127) / 128 * B >= wave ? 128 : 64;
+    dim3 grid((unsigned)((groups + span - 1) / span), (unsigned)B);
+#define CPE_LAUNCH_VOTE_G(FT_, RF_, G_)                                                                              \
+  cpe::decode_vote_vec_kernel<T, FT_, RF_, G_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,   \
+                                                                                  p->bins_h, votes, acc, sums)
+#define CPE_LAUNCH_VOTE_R(FT_, RF_)                                                                                   \
+  switch (span) {                                                                                                     \
+    case 256: CPE_LAUNCH_VOTE_G(FT_, RF_, 256); break;                                                                \
+    case 128: CPE_LAUNCH_VOTE_G(FT_, RF_, 128); break;                                                                \
+    default: CPE_LAUNCH_VOTE_G(FT_, RF_, 64); break;                                                                  \
+  }
 #define CPE_LAUNCH_VOTE(FT_)                                                                                          \
-  if (sums)                                                                                                            \
-    cpe::decode_vote_vec_kernel<T, FT_, true><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,     \
-                                                                                 p->bins_h, votes, acc, sums);        \
-  else                                                                                                                 \
-    cpe::decode_vote_vec_kernel<T, FT_, false><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,    \
-                                                                                  p->bins_h, votes, acc, nullptr)
+  if (sums) { CPE_LAUNCH_VOTE_R(FT_, true) } else { CPE_LAUNCH_VOTE_R(FT_, false) }
     switch (F) {
       case 4: CPE_LAUNCH_VOTE(4); break;
       case 8: CPE_LAUNCH_VOTE(8); break;
       default: CPE_LAUNCH_VOTE(16); break;
     }
 #undef CPE_LAUNCH_VOTE
+#undef CPE_LAUNCH_VOTE_R
+#undef CPE_LAUNCH_VOTE_G
   } else {
     // 64-bit mask loads need every image's mask to start on an 8-byte boundary
     const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);

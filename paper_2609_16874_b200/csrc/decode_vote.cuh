@@ -253,10 +253,12 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 // participating pixel, then each thread takes one (group, axis) item: it issues all 2F plane loads of
 // its axis at once (the only long-latency step), runs the coarse-to-fine estimate for its VEC pixels,
 // swaps results with its partner lane (same group, other axis) and turns half of the pixels into bins.
-constexpr int kVecGroups = 256;      // groups per CTA
+constexpr int kVecGroupsMax = 256;   // groups per CTA: 256, 128 or 64 (template parameter GROUPS; the launcher takes the
+                                     // largest that still gives a full wave of CTAs -- small images are latency-bound
+                                     // and want many short CTAs, large ones want fewer fixed costs)
 constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight together (2 loads each)
 
-template <typename T, int FT, bool REFINE>
+template <typename T, int FT, bool REFINE, int GROUPS>
 __global__ void __launch_bounds__(kVoteThreads, 3)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
                        int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
@@ -271,11 +273,12 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
   const T* e = emb + (size_t)b * 4 * F * plane;
   uint32_t* votes_img = votes + (size_t)b * bins_w * bins_h;
   long long* sums_img = REFINE ? sums + (size_t)b * bins_w * bins_h * 2 : nullptr;
-  const long long span0 = (long long)blockIdx.x * kVecGroups * VEC;
+  static_assert(GROUPS <= kVecGroupsMax && GROUPS <= kVoteThreads, "one thread looks at one group");
+  const long long span0 = (long long)blockIdx.x * GROUPS * VEC;
 
   __shared__ uint32_t s_keys[kHashSlots];
   __shared__ uint32_t s_cnts[kHashSlots];
-  __shared__ uint16_t s_grp[kVecGroups];   // low 8 bits: group index in the span; high 8 bits: participation bits
+  __shared__ uint16_t s_grp[GROUPS];   // low 8 bits: group index in the span; high 8 bits: participation bits
   __shared__ int s_scan[kVoteThreads / 32 + 1];
   __shared__ uint32_t s_nonfinite, s_voting;
   for (int i = tid; i < kHashSlots; i += kVoteThreads) {
@@ -288,7 +291,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
   uint32_t bits = 0;
   {
     const long long p0 = span0 + (long long)tid * VEC;
-    if (p0 < HW) {  // H*W is a multiple of VEC: a group is never cut by the end of the image
+    if (tid < GROUPS && p0 < HW) {  // H*W is a multiple of VEC: a group is never cut by the end of the image
       if (!fg) {
         bits = (1u << VEC) - 1u;
       } else {
