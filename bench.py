@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 # (smsp__inst_executed.sum), which is what an instruction-bound kernel is measured against.
 NCU = {
     # (workload, stage): {"traffic": bytes, "warp_inst": count, "kernel": name}
-    ("c2", "assign"): {"traffic": 22046464, "warp_inst": 10145531, "kernel": "assign_kernel<float,8>"},
-    ("c2", "decode_vote"): {"traffic": 22059520, "warp_inst": 4131965, "kernel": "decode_vote_vec_kernel<float,8>"},
+    ("c2", "assign"): {"traffic": 22046464, "warp_inst": 10155003, "kernel": "assign_kernel<float,8>"},
+    ("c2", "decode_vote"): {"traffic": 22059520, "warp_inst": 4782767, "kernel": "decode_vote_vec_kernel<float,8,false,128>"},
     ("c3", "assign"): {"traffic": 95789568, "warp_inst": 46424257, "kernel": "assign_filter_kernel<__half,16,false>"},
     ("c3", "decode_vote"): {"traffic": 89585408, "warp_inst": 26567474, "kernel": "decode_vote_vec_kernel<__half,8>"},
 }
