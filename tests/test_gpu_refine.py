@@ -134,3 +134,34 @@ def test_refine_intermediate_needs_the_flag_and_workspace_grows_by_the_sums():
     p0.workspace, p0.workspace_bytes = ws.data_ptr(), n0
     rc, _, _ = cb.cpe_get_intermediate(p0, cb.CPE_INT_VOTE_SUMS, 2, 96, 128, 4)
     assert rc == cb.CPE_ERR_WHICH
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c5"])
+def test_refined_full_size_configs(name):
+    """Full-size inputs, graph replay as the benchmark runs it: votes, per-bin sums, peak list, refined centroids and
+    candidate embeddings against the full oracle; labels and scores on sampled pixels; label-map properties on all."""
+    cfg = wl.CONFIGS[name]
+    fr = wl.make_frame(cfg, 0)
+    emb, fg = fr["emb"], fr["fg"]
+    gpu = run_refined(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, mode="graph")
+    ov = oracle.votes(emb, fg, cfg.bins_w, cfg.bins_h, want_est=True, want_cell=True)
+    sums = oracle.vote_sums(ov["est"], ov["cell"], cfg.bins_w, cfg.bins_h)
+    assert np.array_equal(gpu["votes"], ov["votes"])
+    assert np.array_equal(gpu["sums"], sums)
+    rng = np.random.default_rng(7)
+    n_sample = {"c2": 60000, "c3": 40000, "c5": 12000}[name]
+    for b in range(cfg.B):
+        cells, _, raw = oracle.peaks(ov["votes"][b], cfg.T_v, cfg.K_max)
+        n = len(cells)
+        assert gpu["count"][b] == n and np.array_equal(gpu["peak_cell"][b, :n], cells)
+        r = oracle.refined_peaks(ov["votes"][b], sums[b], cells, cfg.F, cfg.H, cfg.W)
+        assert np.array_equal(gpu["centroids"][b, :n].view(np.uint32), r["centroids"].view(np.uint32))
+        np.testing.assert_allclose(gpu["peak_emb"][b, :n], r["peak_emb"], rtol=0, atol=EMB_ATOL)
+        idx = np.sort(rng.choice(cfg.H * cfg.W, n_sample, replace=False)).astype(np.int64)
+        res = oracle.assign_image(emb[b], fg[b], cfg.bins_w, cfg.bins_h, cells, cfg.tau, idx=idx, peak_emb=r["peak_emb"])
+        rep = compare_labels(gpu["labels"][b].ravel()[idx], gpu["best"][b].ravel()[idx], gpu["second"][b].ravel()[idx],
+                             res["labels"], res["best"], res["second"])
+        lab = gpu["labels"][b]
+        assert ((lab > 0) == (fg[b] > 0)).all() and lab.max() <= n
+        print(name, "peaks", n, rep)
+    assert gpu["status"] == 0
