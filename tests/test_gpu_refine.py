@@ -165,3 +165,39 @@ def test_refined_full_size_configs(name):
         assert ((lab > 0) == (fg[b] > 0)).all() and lab.max() <= n
         print(name, "peaks", n, rep)
     assert gpu["status"] == 0
+
+
+def test_refined_edge_cases_empty_truncated_nonfinite_and_border_peaks():
+    # no foreground: no votes, zero sums, no peaks, all labels 0
+    cfg = wl.scaled(wl.CONFIGS["c3"], H=64, W=128, K=4, bins_w=32, bins_h=16)
+    fr = wl.make_frame(cfg, 0)
+    fg0 = np.zeros_like(fr["fg"])
+    gpu = run_refined(fr["emb"], fg0, cfg.bins_w, cfg.bins_h)
+    assert gpu["count"][0] == 0 and (gpu["labels"] == 0).all() and not gpu["sums"].any() and not gpu["votes"].any()
+
+    # more peaks than K_max: the first K_max in bin order are kept and refined; non-finite pixels neither vote nor add
+    cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=96, W=112, K=12, bins_w=28, bins_h=24)
+    fr = wl.make_frame(cfg, 1)
+    emb = fr["emb"].copy()
+    ys, xs = np.nonzero(fr["fg"][1])
+    emb[1, 3, ys[::17], xs[::17]] = np.nan
+    emb[1, 20, ys[5::29], xs[5::29]] = np.inf
+    ora = oracle.decode_refined(emb, fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, K_max=5)
+    assert ora["counters"][:, oracle.CNT_TRUNCATED].min() > 0 and ora["counters"][1, oracle.CNT_NONFINITE] > 0
+    gpu = run_refined(emb, fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, K_max=5)
+    compare_refined(gpu, ora)
+    assert gpu["status"] & cb.CPE_STATUS_PEAK_OVERFLOW and gpu["status"] & cb.CPE_STATUS_NONFINITE
+
+    # instances whose centroids sit in the border bins (clipped 3x3 windows, estimates near -1 and +1)
+    H, W, F, bw, bh = 64, 96, 4, 16, 12
+    inst = np.zeros((H, W), np.int32)
+    inst[:30, :40], inst[:30, 56:], inst[34:, :40], inst[34:, 56:] = 1, 2, 3, 4
+    cents = np.array([[-0.93, -0.90], [0.94, -0.91], [-0.95, 0.92], [0.96, 0.93]])
+    emb = wl.encode(inst, cents, F, 0.02, np.random.default_rng(5), np.float32)[None]
+    fg = (inst > 0).astype(np.uint8)[None]
+    ora = oracle.decode_refined(emb, fg, bw, bh, T_v=8, K_max=8)
+    assert ora["count"][0] == 4
+    cells = ora["peak_cell"][0, :4]
+    assert set((cells % bw).tolist()) <= {0, bw - 1} and set((cells // bw).tolist()) <= {0, bh - 1}
+    gpu = run_refined(emb, fg, bw, bh, T_v=8, K_max=8)
+    compare_refined(gpu, ora)
