@@ -425,7 +425,8 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
   const uint32_t pk_lbo = (uint32_t)peak_cap * 16u; // bytes between core matrices along K in the peak operand
   const bool score_all = WANT2 || need_exact;       // scores wanted: every row is re-scored
   const int R1 = (K + kTcRound - 1) / kTcRound;     // rounds of 64 peaks
-  const bool combined = R1 == 1;                    // one round serves both passes
+  const bool both = R1 == 2;                        // up to 128 peaks: the two stages together hold one round of all peaks
+  const bool combined = R1 <= 2;                    // one round serves both passes
   const int n_rounds = combined ? 1 : 2 * R1;       // per tile: pass 1 rounds (S only), then pass 2 rounds (S and Delta)
 
   // ---- one-time set-up: tensor memory, barriers, zeroed tiles (padding k-slots must stay zero), peak operand
@@ -754,7 +755,8 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
       const uint32_t tq = q / (uint32_t)n_rounds;
       const int r = (int)(q - tq * (uint32_t)n_rounds);
       const int us = (int)(tq % kTiles);
-      const uint32_t as = q & 1u;
+      const uint32_t as = both ? 0u : (q & 1u);
+      const uint32_t uses = both ? q : (q >> 1);    // how often the stage has been used before
       // wait for the tile's operand -- or for the news that the tiles ended before this one
       {
         bool ready = false;
@@ -769,19 +771,21 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
         if (!ready) return false;
       }
       if (*reinterpret_cast<volatile uint32_t*>(s_rflags + us * kTcRows) & kRfEnd) return true;
-      if (!mbar_wait(mb_free + 8 * as, ((q >> 1) & 1u) ^ 1u, s_abort)) return false;
+      if (!mbar_wait(mb_free + 8 * as, (uses & 1u) ^ 1u, s_abort)) return false;
       tc_fence_after();
       const bool with_delta = combined || r >= R1;
       const uint64_t da = da0 + (uint64_t)(((uint32_t)us * (kTileHalves * 2)) >> 4);
-      const uint64_t db = db0 + (uint64_t)(((uint32_t)((r % R1) * kTcRound) * 16u) >> 4);
+      for (int h = 0; h < (both ? 2 : 1); ++h) {     // `both`: peaks 0..63 into stage 0, 64..127 into stage 1
+        const uint64_t db = db0 + (uint64_t)(((uint32_t)((r % R1 + h) * kTcRound) * 16u) >> 4);
 #pragma unroll
-      for (int acc = 0; acc < 2; ++acc) {
-        if (acc == 1 && !with_delta) continue;
+        for (int acc = 0; acc < 2; ++acc) {
+          if (acc == 1 && !with_delta) continue;
 #pragma unroll
-        for (int ks = 0; ks < 2 * KS; ++ks) {
-          const uint32_t id = (acc == 1 && ks >= KS) ? (kTcIdesc | kTcNegB) : kTcIdesc;
-          tc_mma(tmem + as * 128u + (uint32_t)(acc * 64), da + (uint64_t)((ks * 2u * kTileLbo) >> 4),
-                 db + (uint64_t)((ks * 2u * pk_lbo) >> 4), id, ks > 0);
+          for (int ks = 0; ks < 2 * KS; ++ks) {
+            const uint32_t id = (acc == 1 && ks >= KS) ? (kTcIdesc | kTcNegB) : kTcIdesc;
+            tc_mma(tmem + (as + (uint32_t)h) * 128u + (uint32_t)(acc * 64), da + (uint64_t)((ks * 2u * kTileLbo) >> 4),
+                   db + (uint64_t)((ks * 2u * pk_lbo) >> 4), id, ks > 0);
+          }
         }
       }
       tc_commit(mb_done + 8 * as);
@@ -790,13 +794,13 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
     };
     // This warp is through with round q's stage.  The last of the four warps to say so issues round q + 2 into it.
     auto release_stage = [&](uint32_t q) {
-      const uint32_t as = q & 1u;
+      const uint32_t as = both ? 0u : (q & 1u);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(mb_free + 8 * as);
         const uint32_t old = atomicAdd(&s_relcnt[as], 1u);
-        if ((old & 3u) == 3u && !issue_round(q + 2)) {
+        if ((old & 3u) == 3u && !issue_round(q + (both ? 1u : 2u))) {
           *s_abort = 1;
           am_ok(false, 11u, status);
         }
@@ -805,7 +809,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
     };
     // the first two rounds have nobody to release their stages
     if (tid == 0) {
-      if (!issue_round(0) || !issue_round(1)) {
+      if (!issue_round(0) || (!both && !issue_round(1))) {
         *s_abort = 1;
         am_ok(false, 11u, status);
       }
@@ -828,13 +832,16 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
       float s1 = inf, s2 = inf;
       uint32_t as = 0;
       for (int r = 0; r < R1; ++r) {
-        as = rc & 1u;
-        if (!wait_all(mb_done + 8 * as, (rc >> 1) & 1u)) { bad = true; break; }
-        tc_fence_after();
+        if (!both || r == 0) {
+          as = both ? 0u : (rc & 1u);
+          if (!wait_all(mb_done + 8 * as, (both ? rc : (rc >> 1)) & 1u)) { bad = true; break; }
+          tc_fence_after();
+        }
+        const uint32_t st = as + (both ? (uint32_t)r : 0u);      // the stage that holds this round's columns
         const int kn = K - r * kTcRound;
         for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
           float vS[32];
-          tc_ld32(t_lane + as * 128u + (uint32_t)c0, vS);
+          tc_ld32(t_lane + st * 128u + (uint32_t)c0, vS);
           if constexpr (WANT2) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -882,10 +889,11 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
           if (!wait_all(mb_done + 8 * as, (rc >> 1) & 1u)) { bad = true; break; }
           tc_fence_after();
         }
+        const uint32_t st = as + (both ? (uint32_t)r : 0u);
         const int kn = K - r * kTcRound;
         for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
           float vS[32], vD[32];
-          tc_ld32x2(t_lane + as * 128u + (uint32_t)c0, t_lane + as * 128u + 64u + (uint32_t)c0, vS, vD);
+          tc_ld32x2(t_lane + st * 128u + (uint32_t)c0, t_lane + st * 128u + 64u + (uint32_t)c0, vS, vD);
           uint32_t mk = 0, mk2 = 0;     // two chains: the OR into one mask would serialise the loop
           float xs = 0.0f, xd = 0.0f;   // S and Delta of the last column that passed
 #pragma unroll
@@ -921,8 +929,10 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
             }
           }
         }
-        release_stage(rc);
-        ++rc;
+        if (!both || r == R1 - 1) {
+          release_stage(rc);
+          ++rc;
+        }
       }
       if (bad) break;
       // what is left of the list once U is final (the order, ascending k, is kept)

@@ -217,9 +217,12 @@ int launch_assign_filter_t(cudaStream_t st, const T* e, const uint8_t* fg, int B
   int tc_cap = (p->max_instances + cpe::kTcRound - 1) / cpe::kTcRound * cpe::kTcRound;
   const int tc_fixed = cpe::tc_smem_layout(KA, 0).total;
   tc_cap = std::max(cpe::kTcRound, std::min(tc_cap, (budget - tc_fixed) / (2 * KA * 2) / cpe::kTcRound * cpe::kTcRound));
-  // beyond one round the mma.sync body is the faster one (CPE_ASSIGN_PATH=tc lifts the limit: tests, comparisons)
+  // up to 128 peaks fit the two tensor-memory stages at once; beyond that the mma.sync body is the faster one
+  // (CPE_ASSIGN_PATH=tc lifts the limit: tests, comparisons; CPE_ASSIGN_PATH=tc64 keeps it at one stage)
   static const char* path = getenv("CPE_ASSIGN_PATH");
-  const int tc_k_max = (path && strcmp(path, "tc") == 0) ? tc_cap : std::min(tc_cap, cpe::kTcRound);
+  const int tc_k_max = (path && strcmp(path, "tc") == 0)     ? tc_cap
+                       : (path && strcmp(path, "tc64") == 0) ? std::min(tc_cap, cpe::kTcRound)
+                                                             : std::min(tc_cap, 2 * cpe::kTcRound);
   const int tc_smem = cpe::tc_smem_layout(KA, tc_cap).total;
   // mma.sync body
   const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
