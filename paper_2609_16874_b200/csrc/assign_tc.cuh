@@ -15,7 +15,9 @@
 //            so a peak with L_k > thr cannot be the arg-min.                             1/2 instruction per pair
 //   pass 2   L_k <= thr as a bit mask per row, 4 instructions per pair.  A peak that passes gets bounds
 //            dlo <= d_k <= dhi from its S and Delta; the smallest dhi bounds the best distance, and the row's
-//            candidates are the peaks with dlo below it.
+//            candidates are the peaks with dlo below it.  (The sweep runs as four chains, one per column number
+//            mod 4, each remembering the values of its last passing column: registers cannot be indexed by a
+//            run-time column number, and this way several passing columns of a block still have theirs at hand.)
 //   A row with one candidate is decided (no scores wanted, tau = +inf).  The others are queued, per warp, and
 //   worked off when the queue fills up, and at the end by all warps: one lane per (pixel, candidate) pair scores it
 //   in binary32 in the one fixed operation order that defines the result, then one lane per pixel picks the winner.
@@ -34,7 +36,11 @@
 //                         the MMAs of the round after next into it (one lane: {S, Delta} x 4F/16 k-steps of M=128,
 //                         N=64, committed to the stage's mbarrier and, with the tile's last round, to the tile
 //                         buffer's).
-// Two tensor-memory stages of 128 columns, four tile buffers (two for F > 8); two CTAs per SM.  Every wait is
+// Two tensor-memory stages of 128 columns, four tile buffers (two for F > 8); two CTAs per SM.  Up to 64 peaks a
+// tile takes one stage while the other one is filled for the next tile; 65 to 128 peaks take both stages for one tile
+// (one round over all peaks: the MMAs of the next tile then wait for the release, the SM's other CTA fills the gap);
+// more peaks than that go round by round, pass 1 over all rounds and then pass 2 (slower than the mma.sync kernel,
+// which the launcher therefore prefers there).  Every wait is
 // bounded; a wait that runs out raises a flag that every other wait polls, the status word records it, and the
 // kernel winds down.  (A CTA of a kernel that uses tensor memory keeps the SM to itself until it has given up its
 // right to allocate: hence the relinquish right after the allocation.)
@@ -894,37 +900,50 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
         for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
           float vS[32], vD[32];
           tc_ld32x2(t_lane + st * 128u + (uint32_t)c0, t_lane + st * 128u + 64u + (uint32_t)c0, vS, vD);
-          uint32_t mk = 0, mk2 = 0;     // two chains: the OR into one mask would serialise the loop
-          float xs = 0.0f, xd = 0.0f;   // S and Delta of the last column that passed
+          // Four chains, one per column number mod 4: the OR into one mask would serialise the loop, and each chain
+          // remembers S and Delta of its last column that passed -- so up to four columns that pass in one block of
+          // 32 still have their values at hand as long as their numbers differ mod 4 (peaks next to each other in
+          // the list, which are next to each other on the map, always do).
+          uint32_t mq[4] = {0u, 0u, 0u, 0u};
+          float xs[4] = {0.0f, 0.0f, 0.0f, 0.0f}, xd[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float d0 = vD[j] + cD, d1 = vD[j + 1] + cD;
-            if (fmaf(2.0f, vS[j], -fabsf(d0)) <= thr) { mk |= 1u << j; xs = vS[j]; xd = d0; }
-            if (fmaf(2.0f, vS[j + 1], -fabsf(d1)) <= thr) { mk2 |= 1u << (j + 1); xs = vS[j + 1]; xd = d1; }
+          for (int j = 0; j < 32; j += 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float d = vD[j + i] + cD;
+              if (fmaf(2.0f, vS[j + i], -fabsf(d)) <= thr) { mq[i] |= 1u << (j + i); xs[i] = vS[j + i]; xd[i] = d; }
+            }
           }
-          mk |= mk2;
           const int rem = kn - c0;
-          if (rem < 32) mk &= (1u << rem) - 1u;
+          const uint32_t valid = rem < 32 ? (1u << rem) - 1u : 0xffffffffu;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mq[i] &= valid;
+          uint32_t mk = (mq[0] | mq[1]) | (mq[2] | mq[3]);
           if (mk) {
             const int kbase = r * kTcRound + c0;
             n_pairs += (uint32_t)__popc(mk);
-            if ((mk & (mk - 1)) == 0) {
-              // the only one of these 32 columns: its S and Delta are at hand
-              const float Slo = cS + xs;
-              const float e = dS + 4e-6f * (fabsf(Slo) + fabsf(xd));           // |S - S_lo - e| <= e, |Delta - xd| <= e
-              const float a_lo = 0.5f * (Slo + xd - e), b_lo = 0.5f * (Slo - xd - e);
-              const float dlo = (__fsqrt_rn(fmaxf(a_lo, 0.0f)) + __fsqrt_rn(fmaxf(b_lo, 0.0f))) * (1.0f - 2e-6f);
-              const float dhi = (__fsqrt_rn(fmaxf(a_lo + 2.0f * e, 0.0f)) + __fsqrt_rn(fmaxf(b_lo + 2.0f * e, 0.0f))) * (1.0f + 2e-6f);
-              if (dhi < U1) { U2 = U1; U1 = dhi; }
-              else if (dhi < U2) { U2 = dhi; }
-              const float Uref = WANT2 ? U2 : U1;
-              if (dlo <= Uref * (1.0f + 4e-5f) + 1e-6f) append(kbase + __ffs(mk) - 1, dlo);
-            } else {
-              // several in one block of columns: kept without bounds
-              lost = true;
-              while (mk) {
-                append(kbase + __ffs(mk) - 1, 0.0f);
-                mk &= mk - 1;
+            while (mk) {                       // in ascending k: the list keeps that order
+              const int j = __ffs(mk) - 1;
+              mk &= mk - 1;
+              const int i = j & 3;
+              const uint32_t mi = i == 0 ? mq[0] : i == 1 ? mq[1] : i == 2 ? mq[2] : mq[3];
+              if ((mi & (mi - 1)) == 0) {
+                // the only one of its chain: bounds dlo <= d <= dhi from its S and Delta
+                const float xs_ = i == 0 ? xs[0] : i == 1 ? xs[1] : i == 2 ? xs[2] : xs[3];
+                const float xd_ = i == 0 ? xd[0] : i == 1 ? xd[1] : i == 2 ? xd[2] : xd[3];
+                const float Slo = cS + xs_;
+                const float e = dS + 4e-6f * (fabsf(Slo) + fabsf(xd_));           // |S - S_lo - e| <= e, |Delta - xd| <= e
+                const float a_lo = 0.5f * (Slo + xd_ - e), b_lo = 0.5f * (Slo - xd_ - e);
+                const float dlo = (__fsqrt_rn(fmaxf(a_lo, 0.0f)) + __fsqrt_rn(fmaxf(b_lo, 0.0f))) * (1.0f - 2e-6f);
+                const float dhi = (__fsqrt_rn(fmaxf(a_lo + 2.0f * e, 0.0f)) + __fsqrt_rn(fmaxf(b_lo + 2.0f * e, 0.0f))) * (1.0f + 2e-6f);
+                if (dhi < U1) { U2 = U1; U1 = dhi; }
+                else if (dhi < U2) { U2 = dhi; }
+                const float Uref = WANT2 ? U2 : U1;
+                if (dlo <= Uref * (1.0f + 4e-5f) + 1e-6f) append(kbase + j, dlo);
+              } else {
+                // several of one chain: kept without bounds
+                lost = true;
+                append(kbase + j, 0.0f);
               }
             }
           }
