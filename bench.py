@@ -45,8 +45,8 @@ NCU = {
     # (workload, stage): {"traffic": bytes, "warp_inst": count, "kernel": name}
     ("c2", "assign"): {"traffic": 22046464, "warp_inst": 10155003, "kernel": "assign_kernel<float,8>"},
     ("c2", "decode_vote"): {"traffic": 22059520, "warp_inst": 4782767, "kernel": "decode_vote_vec_kernel<float,8,false,128>"},
-    ("c3", "assign"): {"traffic": 95789568, "warp_inst": 46424257, "kernel": "assign_filter_kernel<__half,16,false>"},
-    ("c3", "decode_vote"): {"traffic": 89585408, "warp_inst": 26567474, "kernel": "decode_vote_vec_kernel<__half,8>"},
+    ("c3", "assign"): {"traffic": 95092992, "warp_inst": 48988454, "kernel": "assign_filter_kernel<__half,16,false>"},
+    ("c3", "decode_vote"): {"traffic": 87389696, "warp_inst": 26583472, "kernel": "decode_vote_vec_kernel<__half,8,false,256>"},
 }
 # Ceiling for instruction-bound kernels: 148 SMs x 4 schedulers x 1 warp instruction per clock x 1.965 GHz.
 ALU_PEAK_GWARPINST = 148 * 4 * 1.965
