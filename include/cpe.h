@@ -50,7 +50,9 @@ enum {
   CPE_ERR_CUDA = -7,       /* a CUDA runtime call failed (see cpe_last_cuda_error)         */
   CPE_ERR_WHICH = -8,      /* unknown intermediate id, or it was not requested by flags    */
   CPE_ERR_NOMEM = -9,      /* host or device allocation failed (context helpers only)      */
-  CPE_ERR_STATIC_LIMIT = -10 /* the problem needs more scratch than cpe_decode_static has       */
+  CPE_ERR_STATIC_LIMIT = -10, /* the problem needs more scratch than cpe_decode_static has      */
+  CPE_ERR_BUSY = -11       /* host front end: two calls are already in flight (or, for the
+                              synchronous call, one is)                                    */
 };
 
 /* cpe_params.flags */
@@ -218,17 +220,28 @@ int cpe_profile_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_m
 /* ------------------------------------------------------------------ host-buffer front end --- */
 
 /*
- * End-to-end call for callers whose data lives in host memory.  The context owns its device buffers
- * (input, mask, outputs, workspace), a stream and a captured graph for fixed B, H, W, F and params
- * (params->workspace is ignored).  cpe_host_decode copies emb and fg_mask to the device, replays the
- * graph, copies labels, centroids and counts back and returns when they have arrived.  Host buffers
- * should be page-locked for full copy bandwidth; pageable memory works.  fg_mask_host may be NULL only
- * if the context was created with has_mask = 0.
+ * End-to-end calls for callers whose data lives in host memory.  The context owns two slots, each with its
+ * device buffers (input, mask, outputs, workspace), a stream and a captured graph for fixed B, H, W, F and
+ * params (params->workspace is ignored).
+ *   cpe_host_decode  copies emb and fg_mask to the device, replays the graph, copies labels, centroids and
+ *                    counts back and returns when they have arrived.
+ *   cpe_host_submit  enqueues the same work on the next slot and returns at once; cpe_host_wait returns when
+ *                    the OLDEST submission's results have arrived in the host buffers it was given.  Up to two
+ *                    submissions may be in flight (a third returns CPE_ERR_BUSY and enqueues nothing), so the
+ *                    copy of one step's inputs overlaps the decode and read-back of the step before.  The host
+ *                    buffers of a submission must stay valid and untouched until its wait returns.
+ * cpe_host_wait with nothing in flight returns CPE_ERR_PARAM; cpe_host_decode while something is in flight
+ * returns CPE_ERR_BUSY.  A context is not thread-safe.  Host buffers should be page-locked for full copy
+ * bandwidth and for the overlap (pageable memory works, its copies are staged by the driver).  fg_mask_host
+ * may be NULL only if the context was created with has_mask = 0.
  */
 typedef struct cpe_host_ctx cpe_host_ctx;
 int cpe_host_ctx_create(int B, int H, int W, int F, const cpe_params* params, int has_mask, cpe_host_ctx** out_ctx);
 int cpe_host_decode(cpe_host_ctx* ctx, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
                     float* centroids_host, int32_t* count_host);
+int cpe_host_submit(cpe_host_ctx* ctx, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
+                    float* centroids_host, int32_t* count_host);
+int cpe_host_wait(cpe_host_ctx* ctx);
 /* Bytes moved per cpe_host_decode call in each direction. */
 int cpe_host_ctx_traffic(const cpe_host_ctx* ctx, size_t* h2d_bytes, size_t* d2h_bytes);
 void cpe_host_ctx_destroy(cpe_host_ctx* ctx);

@@ -20,6 +20,7 @@ CPE_F32, CPE_F16 = 0, 1
 CPE_OK = 0
 CPE_ERR_NULL, CPE_ERR_SIZE, CPE_ERR_DTYPE, CPE_ERR_ALIGN, CPE_ERR_WORKSPACE = -1, -2, -3, -4, -5
 CPE_ERR_PARAM, CPE_ERR_CUDA, CPE_ERR_WHICH, CPE_ERR_NOMEM, CPE_ERR_STATIC_LIMIT = -6, -7, -8, -9, -10
+CPE_ERR_BUSY = -11
 CPE_STATIC_SCRATCH_BYTES = 8 << 20
 CPE_STATIC_MAX_BINS = 1024
 CPE_FLAG_WRITE_SCORES = 1
@@ -38,7 +39,8 @@ CPE_STAGE_N = 5
 EXPORTS = (
     "cpe_workspace_size", "cpe_init_workspace", "cpe_decode", "cpe_get_intermediate", "cpe_strerror",
     "cpe_last_cuda_error", "cpe_graph_create", "cpe_graph_launch", "cpe_graph_destroy", "cpe_graph_kernel_nodes",
-    "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
+    "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_submit", "cpe_host_wait",
+    "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
     "cpe_decode_static", "cpe_soft_votes", "cpe_instance_masks", "cpe_channels_last_to_planar",
 )
 
@@ -116,6 +118,10 @@ def load() -> ctypes.CDLL:
     lib.cpe_host_ctx_create.restype = ci
     lib.cpe_host_decode.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.cpe_host_decode.restype = ci
+    lib.cpe_host_submit.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.cpe_host_submit.restype = ci
+    lib.cpe_host_wait.argtypes = [vp]
+    lib.cpe_host_wait.restype = ci
     lib.cpe_host_ctx_traffic.argtypes = [vp, ctypes.POINTER(cs), ctypes.POINTER(cs)]
     lib.cpe_host_ctx_traffic.restype = ci
     lib.cpe_host_ctx_destroy.argtypes = [vp]
@@ -222,6 +228,14 @@ def cpe_host_ctx_create(B, H, W, F, params: cpe_params, has_mask: bool):
 
 def cpe_host_decode(ctx, emb_host, fg_mask_host, labels_host, centroids_host, count_host) -> int:
     return int(load().cpe_host_decode(ctx, emb_host, fg_mask_host or None, labels_host, centroids_host, count_host))
+
+
+def cpe_host_submit(ctx, emb_host, fg_mask_host, labels_host, centroids_host, count_host) -> int:
+    return int(load().cpe_host_submit(ctx, emb_host, fg_mask_host or None, labels_host, centroids_host, count_host))
+
+
+def cpe_host_wait(ctx) -> int:
+    return int(load().cpe_host_wait(ctx))
 
 
 def cpe_host_ctx_traffic(ctx):
@@ -386,6 +400,15 @@ class HostDecoder:
         """numpy (or pinned torch CPU) arrays, contiguous, of the context's shapes."""
         ptr = lambda a: 0 if a is None else (a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data)
         self.decode_ptrs(ptr(emb), ptr(fg), ptr(labels), ptr(centroids), ptr(count))
+
+    def submit(self, emb, fg, labels, centroids, count):
+        """Enqueue a decode (at most two in flight); the arrays must stay alive and untouched until `wait`."""
+        ptr = lambda a: 0 if a is None else (a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data)
+        _check(cpe_host_submit(self.ctx, ptr(emb), ptr(fg), ptr(labels), ptr(centroids), ptr(count)), "cpe_host_submit")
+
+    def wait(self):
+        """Return when the oldest submission's results have arrived."""
+        _check(cpe_host_wait(self.ctx), "cpe_host_wait")
 
     def close(self):
         if self.ctx:

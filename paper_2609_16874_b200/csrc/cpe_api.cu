@@ -383,8 +383,7 @@ struct cpe_graph {
   int kernel_nodes = 0;
 };
 
-struct cpe_host_ctx {
-  int B = 0, H = 0, W = 0, F = 0, has_mask = 0;
+struct HostSlot {
   cpe_params params{};
   cudaStream_t stream = nullptr;
   void* d_emb = nullptr;
@@ -394,6 +393,14 @@ struct cpe_host_ctx {
   int32_t* d_count = nullptr;
   void* d_ws = nullptr;
   cpe_graph* graph = nullptr;
+};
+
+// Two slots, each with its own stream, device buffers, workspace and captured graph: while one slot's decode and
+// read-back run, the other slot's inputs are already on their way to the device.
+struct cpe_host_ctx {
+  int B = 0, H = 0, W = 0, F = 0, has_mask = 0;
+  HostSlot slot[2];
+  unsigned submitted = 0, waited = 0;     // calls so far; submitted - waited <= 2 are in flight
   size_t emb_bytes = 0, fg_bytes = 0, labels_bytes = 0, centroids_bytes = 0, count_bytes = 0;
 };
 
@@ -490,6 +497,7 @@ const char* cpe_strerror(int code) {
     case CPE_ERR_WHICH: return "unknown or unavailable intermediate";
     case CPE_ERR_NOMEM: return "allocation failed";
     case CPE_ERR_STATIC_LIMIT: return "the problem needs more scratch (or more bins) than cpe_decode_static provides";
+    case CPE_ERR_BUSY: return "the host front end already has its two calls in flight";
     default: return "unknown error code";
   }
 }
@@ -587,14 +595,17 @@ int cpe_profile_decode(cpe_stream_t stream, const void* emb, const uint8_t* fg_m
 
 void cpe_host_ctx_destroy(cpe_host_ctx* c) {
   if (!c) return;
-  if (c->graph) cpe_graph_destroy(c->graph);
-  cudaFree(c->d_emb);
-  cudaFree(c->d_fg);
-  cudaFree(c->d_labels);
-  cudaFree(c->d_centroids);
-  cudaFree(c->d_count);
-  cudaFree(c->d_ws);
-  if (c->stream) cudaStreamDestroy(c->stream);
+  for (HostSlot& sl : c->slot) {
+    if (sl.stream) cudaStreamSynchronize(sl.stream);
+    if (sl.graph) cpe_graph_destroy(sl.graph);
+    cudaFree(sl.d_emb);
+    cudaFree(sl.d_fg);
+    cudaFree(sl.d_labels);
+    cudaFree(sl.d_centroids);
+    cudaFree(sl.d_count);
+    cudaFree(sl.d_ws);
+    if (sl.stream) cudaStreamDestroy(sl.stream);
+  }
   delete c;
 }
 
@@ -606,51 +617,73 @@ int cpe_host_ctx_create(int B, int H, int W, int F, const cpe_params* params, in
   cpe_host_ctx* c = new (std::nothrow) cpe_host_ctx();
   if (!c) return CPE_ERR_NOMEM;
   c->B = B; c->H = H; c->W = W; c->F = F; c->has_mask = has_mask ? 1 : 0;
-  c->params = *params;
   const size_t HW = (size_t)H * W;
   c->emb_bytes = (size_t)B * 4 * F * HW * elem_size(params->dtype);
   c->fg_bytes = has_mask ? (size_t)B * HW : 0;
   c->labels_bytes = (size_t)B * HW * 4;
   c->centroids_bytes = (size_t)B * params->max_instances * 2 * 4;
   c->count_bytes = (size_t)B * 4;
-  c->params.workspace_bytes = cpe::make_layout(B, H, W, F, params).total;
-  cudaError_t e = cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking);
-  if (e == cudaSuccess) e = cudaMalloc(&c->d_emb, c->emb_bytes);
-  if (e == cudaSuccess && has_mask) e = cudaMalloc((void**)&c->d_fg, c->fg_bytes);
-  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_labels, c->labels_bytes);
-  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_centroids, c->centroids_bytes);
-  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_count, c->count_bytes);
-  if (e == cudaSuccess) e = cudaMalloc(&c->d_ws, c->params.workspace_bytes);
-  if (e != cudaSuccess) {
-    cuda_fail(e);
-    cpe_host_ctx_destroy(c);
-    return e == cudaErrorMemoryAllocation ? CPE_ERR_NOMEM : CPE_ERR_CUDA;
+  for (HostSlot& sl : c->slot) {
+    sl.params = *params;
+    sl.params.workspace_bytes = cpe::make_layout(B, H, W, F, params).total;
+    cudaError_t e = cudaStreamCreateWithFlags(&sl.stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaMalloc(&sl.d_emb, c->emb_bytes);
+    if (e == cudaSuccess && has_mask) e = cudaMalloc((void**)&sl.d_fg, c->fg_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&sl.d_labels, c->labels_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&sl.d_centroids, c->centroids_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&sl.d_count, c->count_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&sl.d_ws, sl.params.workspace_bytes);
+    if (e != cudaSuccess) {
+      cuda_fail(e);
+      cpe_host_ctx_destroy(c);
+      return e == cudaErrorMemoryAllocation ? CPE_ERR_NOMEM : CPE_ERR_CUDA;
+    }
+    sl.params.workspace = sl.d_ws;
+    cpe_stream_t s = reinterpret_cast<cpe_stream_t>(sl.stream);
+    rc = cpe_init_workspace(s, B, H, W, F, &sl.params);
+    if (rc == CPE_OK && cudaMemsetAsync(sl.d_centroids, 0, c->centroids_bytes, sl.stream) != cudaSuccess) rc = CPE_ERR_CUDA;
+    if (rc == CPE_OK)
+      rc = cpe_graph_create(s, sl.d_emb, sl.d_fg, B, H, W, F, &sl.params, sl.d_labels, sl.d_centroids, sl.d_count,
+                            &sl.graph);
+    if (rc != CPE_OK) { cpe_host_ctx_destroy(c); return rc; }
   }
-  c->params.workspace = c->d_ws;
-  cpe_stream_t s = reinterpret_cast<cpe_stream_t>(c->stream);
-  rc = cpe_init_workspace(s, B, H, W, F, &c->params);
-  if (rc == CPE_OK && cudaMemsetAsync(c->d_centroids, 0, c->centroids_bytes, c->stream) != cudaSuccess) rc = CPE_ERR_CUDA;
-  if (rc == CPE_OK)
-    rc = cpe_graph_create(s, c->d_emb, c->d_fg, B, H, W, F, &c->params, c->d_labels, c->d_centroids, c->d_count,
-                          &c->graph);
-  if (rc != CPE_OK) { cpe_host_ctx_destroy(c); return rc; }
   *out_ctx = c;
+  return CPE_OK;
+}
+
+int cpe_host_submit(cpe_host_ctx* c, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
+                    float* centroids_host, int32_t* count_host) {
+  if (!c || !emb_host || !labels_host || !centroids_host || !count_host) return CPE_ERR_NULL;
+  if (c->has_mask && !fg_mask_host) return CPE_ERR_NULL;
+  if (c->submitted - c->waited >= 2u) return CPE_ERR_BUSY;
+  HostSlot& sl = c->slot[c->submitted & 1u];
+  CPE_CUDA(cudaMemcpyAsync(sl.d_emb, emb_host, c->emb_bytes, cudaMemcpyHostToDevice, sl.stream));
+  if (c->has_mask) CPE_CUDA(cudaMemcpyAsync(sl.d_fg, fg_mask_host, c->fg_bytes, cudaMemcpyHostToDevice, sl.stream));
+  int rc = cpe_graph_launch(sl.graph, reinterpret_cast<cpe_stream_t>(sl.stream));
+  if (rc) return rc;
+  CPE_CUDA(cudaMemcpyAsync(labels_host, sl.d_labels, c->labels_bytes, cudaMemcpyDeviceToHost, sl.stream));
+  CPE_CUDA(cudaMemcpyAsync(centroids_host, sl.d_centroids, c->centroids_bytes, cudaMemcpyDeviceToHost, sl.stream));
+  CPE_CUDA(cudaMemcpyAsync(count_host, sl.d_count, c->count_bytes, cudaMemcpyDeviceToHost, sl.stream));
+  ++c->submitted;
+  return CPE_OK;
+}
+
+int cpe_host_wait(cpe_host_ctx* c) {
+  if (!c) return CPE_ERR_NULL;
+  if (c->submitted == c->waited) return CPE_ERR_PARAM;
+  HostSlot& sl = c->slot[c->waited & 1u];
+  ++c->waited;
+  CPE_CUDA(cudaStreamSynchronize(sl.stream));
   return CPE_OK;
 }
 
 int cpe_host_decode(cpe_host_ctx* c, const void* emb_host, const uint8_t* fg_mask_host, int32_t* labels_host,
                     float* centroids_host, int32_t* count_host) {
-  if (!c || !emb_host || !labels_host || !centroids_host || !count_host) return CPE_ERR_NULL;
-  if (c->has_mask && !fg_mask_host) return CPE_ERR_NULL;
-  CPE_CUDA(cudaMemcpyAsync(c->d_emb, emb_host, c->emb_bytes, cudaMemcpyHostToDevice, c->stream));
-  if (c->has_mask) CPE_CUDA(cudaMemcpyAsync(c->d_fg, fg_mask_host, c->fg_bytes, cudaMemcpyHostToDevice, c->stream));
-  int rc = cpe_graph_launch(c->graph, reinterpret_cast<cpe_stream_t>(c->stream));
+  if (!c) return CPE_ERR_NULL;
+  if (c->submitted != c->waited) return CPE_ERR_BUSY;
+  int rc = cpe_host_submit(c, emb_host, fg_mask_host, labels_host, centroids_host, count_host);
   if (rc) return rc;
-  CPE_CUDA(cudaMemcpyAsync(labels_host, c->d_labels, c->labels_bytes, cudaMemcpyDeviceToHost, c->stream));
-  CPE_CUDA(cudaMemcpyAsync(centroids_host, c->d_centroids, c->centroids_bytes, cudaMemcpyDeviceToHost, c->stream));
-  CPE_CUDA(cudaMemcpyAsync(count_host, c->d_count, c->count_bytes, cudaMemcpyDeviceToHost, c->stream));
-  CPE_CUDA(cudaStreamSynchronize(c->stream));
-  return CPE_OK;
+  return cpe_host_wait(c);
 }
 
 int cpe_host_ctx_traffic(const cpe_host_ctx* c, size_t* h2d_bytes, size_t* d2h_bytes) {

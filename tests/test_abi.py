@@ -93,11 +93,11 @@ def test_intermediate_addresses_are_inside_the_workspace_and_disjoint():
 
 def test_strerror_covers_every_code():
     seen = set()
-    for code in range(0, -10, -1):
+    for code in range(0, -12, -1):
         s = cb.cpe_strerror(code)
         assert s and s != "unknown error code"
         seen.add(s)
-    assert len(seen) == 10
+    assert len(seen) == 12
     assert cb.cpe_strerror(-99) == "unknown error code"
     assert cb.cpe_graph_launch(0, 0) == cb.CPE_ERR_NULL
     assert cb.cpe_graph_kernel_nodes(0) == 0

@@ -213,6 +213,39 @@ def test_host_front_end_matches_device_path():
     hd.close()
 
 
+def test_host_front_end_pipelined_submissions_keep_their_order_and_results():
+    import torch
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=128, W=160, K=7, bins_w=32, bins_h=32)
+    frames = [wl.make_frame(cfg, i) for i in range(5)]
+    want = [oracle.decode(f["emb"], f["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max) for f in frames]
+    hd = cb.HostDecoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    emb = [torch.from_numpy(f["emb"]).pin_memory() for f in frames]
+    fg = [torch.from_numpy(f["fg"]).pin_memory() for f in frames]
+    out = [(torch.full((cfg.B, cfg.H, cfg.W), -1, dtype=torch.int32).pin_memory(),
+            torch.zeros((cfg.B, cfg.K_max, 2), dtype=torch.float32).pin_memory(),
+            torch.zeros((cfg.B,), dtype=torch.int32).pin_memory()) for _ in frames]
+    assert cb.cpe_host_wait(hd.ctx) == cb.CPE_ERR_PARAM                      # nothing in flight
+    hd.submit(emb[0], fg[0], *out[0])
+    hd.submit(emb[1], fg[1], *out[1])
+    ptr = lambda a: a.data_ptr()
+    assert cb.cpe_host_submit(hd.ctx, ptr(emb[2]), ptr(fg[2]), *[ptr(o) for o in out[2]]) == cb.CPE_ERR_BUSY
+    assert cb.cpe_host_decode(hd.ctx, ptr(emb[2]), ptr(fg[2]), *[ptr(o) for o in out[2]]) == cb.CPE_ERR_BUSY
+    for i in range(2, 5):                                                     # steady state: two in flight
+        hd.wait()
+        hd.submit(emb[i], fg[i], *out[i])
+    hd.wait()
+    hd.wait()
+    for i in range(5):
+        lab, cen, cnt = (o.numpy() for o in out[i])
+        assert np.array_equal(cnt, want[i]["count"]), i
+        compare_labels(lab, None, None, want[i]["labels"], want[i]["best"], want[i]["second"])
+        n = int(cnt[0])
+        np.testing.assert_allclose(cen[0, :n], want[i]["centroids"][0, :n], rtol=1e-4, atol=1e-4)
+    hd.decode(emb[3], fg[3], *out[0])                                         # the synchronous call still works afterwards
+    assert np.array_equal(out[0][0].numpy(), out[3][0].numpy())
+    hd.close()
+
+
 def test_profile_entry_point_reports_all_stages():
     import torch
     cfg = wl.scaled(wl.CONFIGS["c2"], H=128, W=128, K=6, bins_w=32, bins_h=32)
