@@ -339,12 +339,17 @@ def run_ours(args, cfg):
         alu = {"achieved": a, "peak": ALU_PEAK_GWARPINST, "unit": "G warp-instructions/s", "frac": a / ALU_PEAK_GWARPINST,
                "warp_instructions_per_launch": ncu["warp_inst"],
                "note": "instruction count from the ncu capture under profiles/; duration measured here"}
+    hbm = {"achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_src}
+    # The dominant kernels of this path are instruction-bound: the headline figures are warp instructions issued per
+    # second against the issue-slot ceiling (148 SMs x 4 schedulers x 1.965 GHz); the `hbm` object says how far the
+    # kernel is from the memory roofline it would have to reach.  Without an instruction count the HBM figures lead.
+    lead = alu if alu else hbm
     roofline = {
-        # the dominant kernels of this path are instruction-bound: the HBM figures say how far the
-        # kernel is from the memory roofline it would have to reach, the `alu` object how busy the issue slots are
-        "bound": "alu" if alu else "hbm", "kernel": ncu.get("kernel", dominant), "achieved": achieved, "peak": peak_gbs,
-        "unit": "GB/s", "frac": achieved / peak_gbs, "traffic": ncu.get("traffic"), "alu": alu,
-        "peak_source": peak_src, "algorithmic_bytes_per_launch": alg[dominant],
+        "bound": "alu" if alu else "hbm", "kernel": ncu.get("kernel", dominant), "achieved": lead["achieved"],
+        "peak": lead["peak"], "unit": lead["unit"], "frac": lead["frac"], "traffic": ncu.get("traffic"),
+        "alu": alu, "hbm": hbm,
+        "peak_source": peak_src if not alu else "derived: SMs x schedulers x clocks.max.sm (issue slots); HBM: " + peak_src,
+        "algorithmic_bytes_per_launch": alg[dominant],
         "kernel_ms": stage_ms[dominant],
         "stage_ms": stage_ms,
         "stage_frac_of_peak": {k: (alg[k] / (v * 1e-3) / 1e9 / peak_gbs if v > 0 else None) for k, v in stage_ms.items()},
