@@ -334,3 +334,15 @@ print("ok")
     env = dict(os.environ, CPE_ASSIGN_PATH="tc")
     out = subprocess.run([sys.executable, "-c", code, root], env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "ok" in out.stdout, out.stdout[-2000:] + out.stderr[-4000:]
+
+
+@pytest.mark.parametrize("name,over", [("c2", dict(H=384, W=384, K=90, bins_w=96, bins_h=96)),              # fp32, F = 8
+                                       ("c5", dict(H=320, W=352, K=100, bins_w=128, bins_h=128)),           # fp16, F = 16
+                                       ("c4", dict(B=2, H=320, W=320, K=70, bins_w=80, bins_h=80))])        # fp16, F = 8
+def test_between_65_and_128_peaks_both_tensor_memory_stages_serve_one_tile(name, over):
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 2)
+    gpu, ora, rep = check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, mode="graph")
+    assert 64 < ora["count"].max() <= 128, ora["count"]
+    assert gpu["status"] == 0
+    print(name, over, ora["count"].tolist(), rep)
