@@ -75,7 +75,7 @@ constexpr uint32_t kRfHard = 8u;      // binary32 pixel beyond the binary16 rang
 constexpr uint32_t kRfEnd = 16u;      // no more tiles
 
 struct TcSmem {
-  int tiles, peaks, queue, hardq, cand, clo, ring, ringbits, rpix, rslack, rcs, rcd, rflags, misc, total;
+  int tiles, peaks, queue, hardq, cand, clo, bmin, ring, ringbits, rpix, rslack, rcs, rcd, rflags, misc, total;
 };
 
 // peak_cap must be a multiple of kTcRound
@@ -90,6 +90,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int KA, int peak_cap) {
   s.hardq = off;    off += 4 * kTcHardQueue * 4;
   s.cand = off;     off += kTcCand * kTcRows * 2;
   s.clo = off;      off += kTcCand * kTcRows * 4;
+  s.bmin = off;     off += 4 * kTcRows * 4;
   s.ring = off;     off += kTcRing * 4;
   s.ringbits = off; off += kTcRing;
   s.rpix = off;     off += tc_tiles(KA) * kTcRows * 4;
@@ -393,6 +394,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
   uint32_t* s_hardq = reinterpret_cast<uint32_t*>(tc_smem + L.hardq);
   uint16_t* s_cand = reinterpret_cast<uint16_t*>(tc_smem + L.cand);       // [slot][row]: the peaks that passed, per row
   float* s_clo = reinterpret_cast<float*>(tc_smem + L.clo);               // [slot][row]: their lower bounds of the distance
+  float* s_bmin = reinterpret_cast<float*>(tc_smem + L.bmin);             // [block of 32 columns][row]: smallest S of pass 1
   uint32_t* s_ring = reinterpret_cast<uint32_t*>(tc_smem + L.ring);       // participating 8-pixel groups, in pixel order
   uint8_t* s_ringbits = reinterpret_cast<uint8_t*>(tc_smem + L.ringbits); // which of a group's 8 pixels participate
   uint32_t* s_rpix = reinterpret_cast<uint32_t*>(tc_smem + L.rpix);       // per tile buffer and row: pixel index
@@ -848,17 +850,20 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
         for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
           float vS[32];
           tc_ld32(t_lane + st * 128u + (uint32_t)c0, vS);
+          float bm = inf;               // the block's own minimum: pass 2 skips blocks that cannot hold a candidate
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) bm = min3f(bm, vS[j], vS[j + 1]);   // columns beyond the last peak are NaN
+          if (combined) s_bmin[(2 * r + (c0 >> 5)) * kTcRows + tid] = bm;
           if constexpr (WANT2) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const float v = (vS[j] == vS[j]) ? vS[j] : inf;   // columns beyond the last peak are NaN
+              const float v = (vS[j] == vS[j]) ? vS[j] : inf;
               const float lo = fminf(s1, v), hi = fmaxf(s1, v);
               s1 = lo;
               s2 = fminf(s2, hi);
             }
           } else {
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) s1 = min3f(s1, vS[j], vS[j + 1]);
+            s1 = fminf(s1, bm);
           }
         }
         if (!combined) {
@@ -875,6 +880,10 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
       const float sref = (WANT2 ? s2 : s1) + cS;
       const float thr_full = (2.0f * (sref + 2.0f * dS) * (1.0f + 1e-5f) + 1e-6f) + dS;
       const float thr = live ? (thr_full - 2.0f * cS) + 1e-5f * (fabsf(thr_full) + 2.0f * cS) : qnan;
+      // |Delta_c| <= S_lo + 3 dS = cS + S_acc + 3 dS, so what pass 2 tests is at least S_acc - cS - 3 dS: a column
+      // can only pass if S_acc <= thrS, and a block of 32 columns whose smallest S_acc is above it for every row of
+      // the warp is not looked at again (neighbouring pixels have the same few peaks close by: most blocks go).
+      const float thrS = (thr + cS + 3.0f * dS) + 1e-5f * (fabsf(thr) + cS);
 
       // ---- pass 2: L_k <= thr as a bit mask.  A peak that passes gets bounds dlo <= d <= dhi from its S and Delta
       // (A = (S + Delta) / 2, B = (S - Delta) / 2); the smallest dhi, U, bounds the best distance, and the candidates
@@ -898,6 +907,10 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
         const uint32_t st = as + (both ? (uint32_t)r : 0u);
         const int kn = K - r * kTcRound;
         for (int c0 = 0; c0 < kTcRound && c0 < kn; c0 += 32) {
+          if (combined) {
+            const bool need = live && s_bmin[(2 * r + (c0 >> 5)) * kTcRows + tid] <= thrS;
+            if (!__any_sync(0xffffffffu, need)) continue;
+          }
           float vS[32], vD[32];
           tc_ld32x2(t_lane + st * 128u + (uint32_t)c0, t_lane + st * 128u + 64u + (uint32_t)c0, vS, vD);
           // Four chains, one per column number mod 4: the OR into one mask would serialise the loop, and each chain
