@@ -13,6 +13,8 @@
 // (binary16 rounding of the palette and, for binary32 inputs, of the pixel; accumulation):
 //   pass 1   the smallest S_k (the second smallest when the runner-up is wanted): d_best^2 <= 2 (S_min + slack) =: thr,
 //            so a peak with L_k > thr cannot be the arg-min.                             1/2 instruction per pair
+//            The minimum of every block of 32 columns is kept as well: |Delta| <= S bounds what pass 2 computes from
+//            below by S alone, so a block whose minimum is too large for every row of the warp is skipped there.
 //   pass 2   L_k <= thr as a bit mask per row, 4 instructions per pair.  A peak that passes gets bounds
 //            dlo <= d_k <= dhi from its S and Delta; the smallest dhi bounds the best distance, and the row's
 //            candidates are the peaks with dlo below it.  (The sweep runs as four chains, one per column number
