@@ -859,6 +859,23 @@ extern "C" int cpe_channels_last_to_planar(cpe_stream_t stream, const void* emb_
   // base does; a plane piece does iff the base, the plane pitch H * W and the tile start are multiples of 16 bytes
   const int vec_in = (uintptr_t)emb_nhwc % 16 == 0 && ((size_t)HW * D * esz) % 16 == 0;
   const int vec_out = (uintptr_t)emb_planar % 16 == 0 && ((size_t)HW * esz) % 16 == 0;
+  // aligned inputs with whole tiles and a power-of-two number of 4-channel units take the unit-wise kernels
+  const int U = D / 4;
+  const bool pow2_units = (U & (U - 1)) == 0;
+  if (vec_in && vec_out && pow2_units && dtype == CPE_F16 && U >= 2 && HW % cpe::kLyFastPixels16 == 0) {
+    dim3 g((unsigned)(HW / cpe::kLyFastPixels16), (unsigned)B);
+    cpe::channels_last_to_planar_f16_kernel<<<g, cpe::kLyThreads, (size_t)cpe::kLyFastPixels16 * D * 2, st>>>(
+        static_cast<const uint16_t*>(emb_nhwc), static_cast<uint16_t*>(emb_planar), HW, D);
+    CPE_CUDA(cudaGetLastError());
+    return CPE_OK;
+  }
+  if (vec_in && vec_out && pow2_units && dtype == CPE_F32 && HW % cpe::kLyFastPixels32 == 0) {
+    dim3 g((unsigned)(HW / cpe::kLyFastPixels32), (unsigned)B);
+    cpe::channels_last_to_planar_f32_kernel<<<g, cpe::kLyThreads, (size_t)cpe::kLyFastPixels32 * D * 4, st>>>(
+        static_cast<const float*>(emb_nhwc), static_cast<float*>(emb_planar), HW, D);
+    CPE_CUDA(cudaGetLastError());
+    return CPE_OK;
+  }
   if (dtype == CPE_F32)
     cpe::channels_last_to_planar_kernel<float><<<grid, cpe::kLyThreads, smem, st>>>(
         static_cast<const float*>(emb_nhwc), static_cast<float*>(emb_planar), HW, D, vec_in, vec_out);

@@ -10,7 +10,12 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("shape,dtype", [((2, 12, 37, 53), np.float32), ((1, 64, 64, 96), np.float16),
-                                         ((3, 4, 1, 7), np.float16), ((1, 20, 130, 64), np.float32)])
+                                         ((3, 4, 1, 7), np.float16), ((1, 20, 130, 64), np.float32),
+                                         # aligned, whole tiles, power-of-two channel units: the unit-wise kernels
+                                         ((2, 32, 64, 64), np.float32), ((1, 32, 32, 64), np.float16),
+                                         ((2, 8, 16, 64), np.float16), ((1, 16, 8, 48), np.float32),
+                                         ((1, 64, 32, 32), np.float32), ((2, 16, 48, 32), np.float16),
+                                         ((1, 4, 16, 16), np.float32)])
 def test_conversion_is_a_transpose(shape, dtype):
     import torch
     B, D, H, W = shape
