@@ -74,7 +74,8 @@ enum {
                                  out_centroids holds that mean in pixel units and the peak's candidate embedding
                                  is gamma(mean) of Eq. 2 (binary64 sin/cos, rounded once) instead of the palette
                                  rows.  Peak detection and everything else are unchanged.  Needs a larger
-                                 workspace (16 bytes per bin and image) and one clearing pass per decode.      */
+                                 workspace (16 bytes per bin and image); maps of more than 8192 bins, and decodes
+                                 with CPE_FLAG_KEEP_VOTES, add one clearing pass per decode.                  */
 };
 
 /* bits of the per-image device status words */
@@ -112,7 +113,8 @@ enum {
   CPE_INT_STATUS = 8,       /* uint32 [B]                       CPE_STATUS_* bits of each image      */
   CPE_INT_COUNTERS = 9,     /* uint32 [B][CPE_CNT_N]                                            */
   CPE_INT_VOTE_SUMS = 10,   /* int64  [B][bins_h][bins_w][2]    fixed-point (2^-24) sums of the x and y
-                                                                estimates per bin (CPE_FLAG_REFINE)  */
+                                                                estimates per bin (CPE_FLAG_REFINE and
+                                                                CPE_FLAG_KEEP_VOTES)                 */
   CPE_INT_N = 11
 };
 

@@ -339,9 +339,12 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_CLEAR], st));
   // Normally the map is already zero (cpe_init_workspace, then the previous decode's last kernel).
   if (keep_votes) CPE_CUDA(cudaMemsetAsync(ws + L.votes, 0, L.votes_end - L.votes, st));
-  // The per-bin sums of the refinement stay readable after the decode, so they are cleared here.
+  // The per-bin sums of the refinement: a small map, which one CTA of the peak kernel handles per image, is cleared
+  // by that CTA after its last read; otherwise (or when the intermediates are to stay readable) they are cleared here.
   long long* sums = (p->flags & CPE_FLAG_REFINE) ? reinterpret_cast<long long*>(ws + L.sums) : nullptr;
-  if (sums) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
+  const bool one_peak_cta = L.words <= 8 * (cpe::kPeakThreads / 32);
+  const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes;
+  if (sums && !sums_cleared_by_peaks) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
   rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, acc, sums)
@@ -353,11 +356,12 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   {
     const int warps_per_cta = cpe::kPeakThreads / 32;
     // small maps: one CTA per image does both phases without the cross-CTA hand-over
-    const int ctas = L.words <= 8 * warps_per_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
+    const int ctas = one_peak_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
     dim3 grid((unsigned)ctas, (unsigned)B);
     CPE_CUDA(launch_dependent(cpe::peaks_kernel, grid, cpe::kPeakThreads, 0, st, votes, p->bins_w, p->bins_h, L.words,
                               (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W, pal_w, pal_h, peak_cell,
-                              peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums));
+                              peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums,
+                              sums_cleared_by_peaks ? 1 : 0));
     CPE_CUDA(cudaGetLastError());
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
@@ -473,7 +477,7 @@ int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int 
     case CPE_INT_STATUS: off = L.status; sz = 4 * (size_t)B; break;
     case CPE_INT_COUNTERS: off = L.counters; sz = 4 * (size_t)CPE_CNT_N * B; break;
     case CPE_INT_VOTE_SUMS:
-      if (!(params->flags & CPE_FLAG_REFINE)) return CPE_ERR_WHICH;
+      if (!(params->flags & CPE_FLAG_REFINE) || !(params->flags & CPE_FLAG_KEEP_VOTES)) return CPE_ERR_WHICH;
       off = L.sums;
       sz = 16 * (size_t)L.cells * B;
       break;

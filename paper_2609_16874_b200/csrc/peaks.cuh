@@ -23,14 +23,15 @@ constexpr int kRefineChunk = 1024;     // peaks whose refined positions are stag
 // With `sums` (sub-cell refinement; int64 [B][cells][2], the fixed-point sums of the estimates that fell into each
 // bin) a peak is moved from its bin position to the mean estimate of its 3x3 neighbourhood -- a strict peak has no
 // other peak there, so those votes are its own -- and its embedding is gamma(mean) of Eq. 2, evaluated in binary64
-// and rounded once, the way the palette rows are made.
+// and rounded once, the way the palette rows are made.  `zero_sums` (only with one CTA per image): the sums are cleared
+// at the end, so that the decode needs no clearing pass for them.
 __global__ void __launch_bounds__(kPeakThreads)
 peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
              uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
              uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
-             const long long* __restrict__ sums) {
+             long long* __restrict__ sums, int zero_sums) {
   grid_dependency_sync();
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -151,7 +152,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   float* pe = peak_emb + (size_t)b * K_max * D;
   if (sums) {
     __shared__ double s_mean[2 * kRefineChunk];
-    const long long* S = sums + (size_t)b * cells * 2;
+    long long* S = sums + (size_t)b * cells * 2;
     for (int k0 = 0; k0 < count; k0 += kRefineChunk) {
       const int nk = min(kRefineChunk, count - k0);
       for (int i = tid; i < 2 * nk; i += kPeakThreads) {       // (peak, axis): pooled mean of the 3x3 window
@@ -188,6 +189,9 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
       }
       __syncthreads();
     }
+    // small maps (this CTA does the whole image): the sums have no reader left and are left zero for the next decode
+    if (zero_sums)
+      for (int i = tid; i < 2 * cells; i += kPeakThreads) S[i] = 0;
     return;
   }
   for (int i = tid; i < count * D; i += kPeakThreads) {
