@@ -4,8 +4,10 @@
 //   GEMM 1   D_x = Xhat (-2 P_w)^T  [128 pixels x 128 bins], D_y likewise: binary16 operands split into a high and a
 //            low part (pixel and palette), three tcgen05.mma per k-step, binary32 accumulators in tensor memory, so
 //            that ||xhat - P_w[a]||^2 = ||xhat||^2 + F + D_x is good to ~1e-6 relative before the square root.
-//   epilogue a thread that owns one pixel row reads its D row (tcgen05.ld), forms exp(-sqrt(.)) and stores it,
-//            rounded to binary16, straight into the operand layout of GEMM 2 (bin-major core matrices).
+//   epilogue two threads own one pixel row (one per axis, in warps that share the row's tensor-memory lanes): each
+//            reads its D row (tcgen05.ld), forms exp(-sqrt(.)) and stores it, rounded to binary16, straight into the
+//            operand layout of GEMM 2 (bin-major core matrices).  Two warps per scheduler keep the special-function
+//            unit, which bounds this kernel, busier than one can.
 //   GEMM 2   H_block += E_x^T E_y  [128 x 128 bins], K = the tile's 128 pixels, accumulated in tensor memory over all
 //            the tiles that the CTA sees; at the end the block is added to the histogram in global memory
 //            (binary32 atomics: the split over CTAs is a split-K reduction whose order is not fixed).
@@ -20,7 +22,8 @@
 
 namespace cpe {
 
-constexpr int kSvThreads = 256;     // warps 0-3: pixel rows (epilogues, MMA issue), warps 4-7: producers
+constexpr int kSvThreads = 384;     // warps 0-3: pixel rows, x axis (and MMA issue); warps 4-7: producers;
+                                    // warps 8-11: the same pixel rows, y axis
 constexpr int kSvBins = 128;        // bins per block side
 constexpr int kSvTiles = 2;         // pixel tile buffers
 constexpr int kSvCols = 512;        // tensor-memory columns: D_x [0,128), D_y [128,256), H block [256,384)
@@ -51,8 +54,8 @@ __host__ __device__ inline SvSmem sv_smem_layout(int KA) {
 constexpr uint32_t kSvIdesc1 = (1u << 4) | (1u << 15) | ((uint32_t)(kSvBins >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t kSvIdesc2 = kSvIdesc1 | (1u << 16);
 
-// Barrier among the 128 consumer threads (barrier resource 2)
-__device__ __forceinline__ void sv_consumers_sync() { asm volatile("barrier.cta.sync 2, 128;" ::: "memory"); }
+// Barrier among the 256 row threads of both axes (barrier resource 2)
+__device__ __forceinline__ void sv_consumers_sync() { asm volatile("barrier.cta.sync 2, 256;" ::: "memory"); }
 
 template <typename T, int KA>
 __global__ void __launch_bounds__(kSvThreads, 1)
@@ -136,7 +139,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  if (wid >= 4) {
+  if (wid >= 4 && wid < 8) {
     // =============================================================================================== producers
     const int ptid = tid - 128, pw = ptid >> 5;
     const int gl = ptid >> 3, cq = ptid & 7;        // lane cq fetches channels cq, cq+8, ... of group gl, owns row ptid
@@ -273,7 +276,9 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     }
   } else {
     // =============================================================================================== pixel rows
-    const uint32_t t_lane = tmem + ((uint32_t)(wid * 32) << 16);
+    const int axis_y = wid >= 8 ? 1 : 0;                 // which of the two distance accumulators this thread reads
+    const int row = tid & 127;                           // warps 8-11 start at thread 256
+    const uint32_t t_lane = tmem + ((uint32_t)((wid & 3) * 32) << 16);
     const uint64_t d_tile0 = tc_desc((uint32_t)__cvta_generic_to_shared(s_tiles), kTileLbo, 128u);
     const uint64_t d_pw = tc_desc((uint32_t)__cvta_generic_to_shared(s_pw), kPalLbo, 128u);
     const uint64_t d_ph = tc_desc((uint32_t)__cvta_generic_to_shared(s_ph), kPalLbo, 128u);
@@ -308,10 +313,10 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
         const bool ok = mbar_wait(mb_meta + 8 * us, (t / kSvTiles) & 1u, s_abort);
         if (!__all_sync(0xffffffffu, ok)) { bad = true; break; }
       }
-      const uint32_t flags = s_rflags[us * kTcRows + tid];
+      const uint32_t flags = s_rflags[us * kTcRows + row];
       if (flags & kRfEnd) break;
       const bool live = (flags & kRfLive) != 0;
-      const float cx = s_rnx[us * kTcRows + tid] + (float)F, cy = s_rny[us * kTcRows + tid] + (float)F;
+      const float cn = (axis_y ? s_rny : s_rnx)[us * kTcRows + row] + (float)F;
       tc_fence_before();
       sv_consumers_sync();        // every row has its data; the D columns and (after GEMM 2) the E tiles are free
       if (tid == 0) {
@@ -346,22 +351,15 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       // ---- epilogue: this row's weights into the operand tiles of GEMM 2: element (bin n, pixel p) at
       // (p / 8) * kELbo + (n / 8) * 128 + (p % 8) * 16 + (n % 8) * 2 bytes
       {
-        unsigned char* ex_row = reinterpret_cast<unsigned char*>(s_ex) + (tid >> 3) * kELbo + (tid & 7) * 16;
-        unsigned char* ey_row = reinterpret_cast<unsigned char*>(s_ey) + (tid >> 3) * kELbo + (tid & 7) * 16;
+        unsigned char* e_row = reinterpret_cast<unsigned char*>(axis_y ? s_ey : s_ex) + (row >> 3) * kELbo + (row & 7) * 16;
         // only the bins that exist (in steps of 32): the rest of the E tiles stays zero
-        for (int c0 = 0; c0 < max(na, nb); c0 += 32) {
-          float vx[32], vy[32];
-          tc_ld32x2(t_lane + (uint32_t)c0, t_lane + 128u + (uint32_t)c0, vx, vy);
-          if (c0 < na) {
+        const int nbins = axis_y ? nb : na;
+        for (int c0 = 0; c0 < nbins; c0 += 32) {
+          float v[32];
+          tc_ld32(t_lane + (uint32_t)(axis_y * 128 + c0), v);
 #pragma unroll
-            for (int g = 0; g < 4; ++g)
-              *reinterpret_cast<uint4*>(ex_row + ((c0 >> 3) + g) * 128) = weights8(vx + 8 * g, cx, live);
-          }
-          if (c0 < nb) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-              *reinterpret_cast<uint4*>(ey_row + ((c0 >> 3) + g) * 128) = weights8(vy + 8 * g, cy, live);
-          }
+          for (int g = 0; g < 4; ++g)
+            *reinterpret_cast<uint4*>(e_row + ((c0 >> 3) + g) * 128) = weights8(v + 8 * g, cn, live);
         }
       }
       fence_async_smem();
@@ -387,9 +385,10 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     }
     if (!bad && t > 0) {
       tc_fence_after();
-      const int a = a0 + tid;
+      const int a = a0 + row;
       float* h_img = hist + (size_t)img * bins_w * bins_h;
-      for (int c0 = 0; c0 < kSvBins; c0 += 32) {
+      // the two threads of a row share its columns
+      for (int c0 = axis_y * (kSvBins / 2); c0 < (axis_y + 1) * (kSvBins / 2); c0 += 32) {
         float v[32];
         tc_ld32(t_lane + 256u + (uint32_t)c0, v);
         if (a < bins_w) {
