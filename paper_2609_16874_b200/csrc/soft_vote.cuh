@@ -292,59 +292,76 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     const int na = min(kSvBins, bins_w - a0), nb = min(kSvBins, bins_h - b0);   // bins of this block that exist
 
     // exp(-sqrt(max(c + D, 0))) for 8 consecutive bins, rounded to binary16.  The special-function unit's
-    // approximations (sqrt, 2^x: about 2^-22 relative each) are far inside the binary16 rounding that follows.
+    // approximations (sqrt, 2^x: about 2^-22 relative each) are far inside the binary16 rounding that follows; the
+    // flush-to-zero forms are single instructions (a subnormal argument or result is below anything binary16 holds:
+    // its smallest subnormal is e^-16.6).  A row without a pixel is masked after packing.
     auto weights8 = [&](const float* v, float c, bool live) -> uint4 {
-      __half2 h[4];
+      uint32_t w[4];
+      const uint32_t keep = live ? 0xffffffffu : 0u;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float d0, d1, e0, e1;
-        asm("sqrt.approx.f32 %0, %1;" : "=f"(d0) : "f"(fmaxf(c + v[2 * i], 0.0f)));
-        asm("sqrt.approx.f32 %0, %1;" : "=f"(d1) : "f"(fmaxf(c + v[2 * i + 1], 0.0f)));
-        asm("ex2.approx.f32 %0, %1;" : "=f"(e0) : "f"(-d0 * log2e));
-        asm("ex2.approx.f32 %0, %1;" : "=f"(e1) : "f"(-d1 * log2e));
-        h[i] = __floats2half2_rn(live ? e0 : 0.0f, live ? e1 : 0.0f);
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d0) : "f"(fmaxf(c + v[2 * i], 0.0f)));
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d1) : "f"(fmaxf(c + v[2 * i + 1], 0.0f)));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-d0 * log2e));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-d1 * log2e));
+        const __half2 h = __floats2half2_rn(e0, e1);
+        w[i] = *reinterpret_cast<const uint32_t*>(&h) & keep;
       }
-      return *reinterpret_cast<const uint4*>(h);
+      return make_uint4(w[0], w[1], w[2], w[3]);
     };
 
-    while (true) {
-      const int us = (int)(t % kSvTiles);
-      {
-        const bool ok = mbar_wait(mb_meta + 8 * us, (t / kSvTiles) & 1u, s_abort);
-        if (!__all_sync(0xffffffffu, ok)) { bad = true; break; }
+    // GEMM 1 of tile `tt` (buffer `us`): D_x, D_y = pixel tile (high [+ low]) x palette block (high + low)
+    auto issue_gemm1 = [&](int us) {
+      const uint64_t da = d_tile0 + (uint64_t)(((uint32_t)us * 2u * (kPartHalves * 2)) >> 4);
+#pragma unroll
+      for (int axis = 0; axis < 2; ++axis) {
+        const uint64_t db = axis ? d_ph : d_pw;
+        bool acc = false;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          const uint64_t ka = da + (uint64_t)(((axis * KS + ks) * 2u * kTileLbo) >> 4);
+          const uint64_t kb = db + (uint64_t)((ks * 2u * kPalLbo) >> 4);
+          tc_mma(tmem + (uint32_t)(axis * 128), ka, kb, kSvIdesc1, acc);
+          acc = true;
+          tc_mma(tmem + (uint32_t)(axis * 128), ka, kb + kLoPal, kSvIdesc1, true);
+          if (kSplitPixel) tc_mma(tmem + (uint32_t)(axis * 128), ka + kLoTile, kb, kSvIdesc1, true);
+        }
       }
-      const uint32_t flags = s_rflags[us * kTcRows + row];
-      if (flags & kRfEnd) break;
-      const bool live = (flags & kRfLive) != 0;
-      const float cn = (axis_y ? s_rny : s_rnx)[us * kTcRows + row] + (float)F;
+      tc_commit(mb_d);
+      tc_commit(mb_tile + 8 * us);
+    };
+    // row data of tile `tt`: false when the wait ran out
+    uint32_t flags = 0;
+    float cn = 0.0f;
+    auto fetch_row = [&](uint32_t tt) -> bool {
+      const int us = (int)(tt % kSvTiles);
+      const bool ok = mbar_wait(mb_meta + 8 * us, (tt / kSvTiles) & 1u, s_abort);
+      if (!__all_sync(0xffffffffu, ok)) return false;
+      flags = s_rflags[us * kTcRows + row];
+      cn = (axis_y ? s_rny : s_rnx)[us * kTcRows + row] + (float)F;
+      return true;
+    };
+
+    // The loop is software-pipelined by one tile: the thread that issues GEMM 2 of tile t issues GEMM 1 of tile t + 1
+    // right behind it, so the tensor pipe runs them back to back while the row threads are between two epilogues,
+    // and one wait (GEMM 1 done: the MMAs complete in issue order, so GEMM 2 of the tile before is done as well)
+    // and one barrier per tile are enough.
+    if (!fetch_row(0)) bad = true;
+    if (!bad && !(flags & kRfEnd)) {
       tc_fence_before();
-      sv_consumers_sync();        // every row has its data; the D columns and (after GEMM 2) the E tiles are free
+      sv_consumers_sync();        // every row thread has read its row data
       if (tid == 0) {
         tc_fence_after();
-        // GEMM 1: D_x, D_y = pixel tile (high [+ low]) x palette block (high + low)
-        const uint64_t da = d_tile0 + (uint64_t)(((uint32_t)us * 2u * (kPartHalves * 2)) >> 4);
-#pragma unroll
-        for (int axis = 0; axis < 2; ++axis) {
-          const uint64_t db = axis ? d_ph : d_pw;
-          bool acc = false;
-#pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            const uint64_t ka = da + (uint64_t)(((axis * KS + ks) * 2u * kTileLbo) >> 4);
-            const uint64_t kb = db + (uint64_t)((ks * 2u * kPalLbo) >> 4);
-            tc_mma(tmem + (uint32_t)(axis * 128), ka, kb, kSvIdesc1, acc);
-            acc = true;
-            tc_mma(tmem + (uint32_t)(axis * 128), ka, kb + kLoPal, kSvIdesc1, true);
-            if (kSplitPixel) tc_mma(tmem + (uint32_t)(axis * 128), ka + kLoTile, kb, kSvIdesc1, true);
-          }
-        }
-        tc_commit(mb_d);
-        tc_commit(mb_tile + 8 * us);
+        issue_gemm1(0);
       }
       __syncwarp();
+    }
+    while (!bad && !(flags & kRfEnd)) {
+      const bool live = (flags & kRfLive) != 0;
+      const float c_row = cn;
       {
-        bool ok = mbar_wait(mb_d, t & 1u, s_abort);
-        // the E tiles are still being read by GEMM 2 of the previous tile
-        if (t > 0) ok = mbar_wait(mb_e, (t - 1) & 1u, s_abort) && ok;
+        const bool ok = mbar_wait(mb_d, t & 1u, s_abort);   // GEMM 1 of this tile (and every MMA before it) is done
         if (!__all_sync(0xffffffffu, ok)) { bad = true; break; }
       }
       tc_fence_after();
@@ -359,9 +376,11 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
           tc_ld32(t_lane + (uint32_t)(axis_y * 128 + c0), v);
 #pragma unroll
           for (int g = 0; g < 4; ++g)
-            *reinterpret_cast<uint4*>(e_row + ((c0 >> 3) + g) * 128) = weights8(v + 8 * g, cn, live);
+            *reinterpret_cast<uint4*>(e_row + ((c0 >> 3) + g) * 128) = weights8(v + 8 * g, c_row, live);
         }
       }
+      // the next tile's row data (the producers are a tile ahead), before the barrier that frees D and publishes E
+      if (!fetch_row(t + 1)) { bad = true; break; }
       fence_async_smem();
       tc_fence_before();
       sv_consumers_sync();
@@ -374,6 +393,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
           tc_mma(tmem + 256u, d_ex + o, d_ey + o, kSvIdesc2, t > 0 || ks > 0);
         }
         tc_commit(mb_e);
+        if (!(flags & kRfEnd)) issue_gemm1((int)((t + 1) % kSvTiles));
       }
       __syncwarp();
       ++t;
