@@ -120,18 +120,31 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
   }
   // -2 P rows of this block, split into binary16 high and low parts; K-major core matrices: (bin n, slot s) at
   // (s / 8) * (128 * 8) + n * 8 + s % 8.  Bins beyond the map are zero rows (their H entries are never stored).
-  for (int i = tid; i < 2 * kSvBins * KA; i += kSvThreads) {
-    const int axis = i / (kSvBins * KA), j = i - axis * kSvBins * KA;
-    const int n = j / KA, s = j - n * KA;
-    const int bin = (axis ? b0 : a0) + n, nbins = axis ? bins_h : bins_w;
-    float v = 0.0f;
-    if (bin < nbins && s < 2 * F) v = -2.0f * (axis ? pal_h : pal_w)[(size_t)bin * 2 * F + s];
-    const __half hi = __float2half_rn(v);
-    const __half lo = __float2half_rn(v - __half2float(hi));
-    __half* dst = axis ? s_ph : s_pw;
-    const int o = (s >> 3) * (kSvBins * 8) + n * 8 + (s & 7);
-    dst[o] = hi;
-    dst[kSvBins * KA + o] = lo;
+  // (four elements per thread and round, so that their loads are in flight together)
+  for (int i0 = tid; i0 < 2 * kSvBins * KA; i0 += 4 * kSvThreads) {
+    float v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * kSvThreads;
+      const int axis = i / (kSvBins * KA), j = i - axis * kSvBins * KA;
+      const int n = j / KA, s = j - n * KA;
+      const int bin = (axis ? b0 : a0) + n, nbins = axis ? bins_h : bins_w;
+      v[u] = 0.0f;
+      if (i < 2 * kSvBins * KA && bin < nbins && s < 2 * F) v[u] = -2.0f * __ldg((axis ? pal_h : pal_w) + (size_t)bin * 2 * F + s);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * kSvThreads;
+      if (i >= 2 * kSvBins * KA) break;
+      const int axis = i / (kSvBins * KA), j = i - axis * kSvBins * KA;
+      const int n = j / KA, s = j - n * KA;
+      const __half hi = __float2half_rn(v[u]);
+      const __half lo = __float2half_rn(v[u] - __half2float(hi));
+      __half* dst = axis ? s_ph : s_pw;
+      const int o = (s >> 3) * (kSvBins * 8) + n * 8 + (s & 7);
+      dst[o] = hi;
+      dst[kSvBins * KA + o] = lo;
+    }
   }
   fence_async_smem();
   tc_fence_before();
@@ -169,10 +182,29 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
         const uint32_t grp = s_ring[(ring_head + gl) & (kTcRing - 1)];
         bits = s_ringbits[(ring_head + gl) & (kTcRing - 1)];
         const T* src0 = e_img + (size_t)grp * 8;
-        for (int c = cq; c < D; c += 8) {
+        constexpr int kIt = 2 * KA / 8;                 // channels per lane at most (D <= 2 KA)
+        // every load of this lane is issued before the first value is used
+        uint4 raw[kIt * (sizeof(T) == 2 ? 1 : 2)];
+#pragma unroll
+        for (int it = 0; it < kIt; ++it) {
+          const int c = cq + 8 * it;
+          if (c < D) {
+            const uint4* src = reinterpret_cast<const uint4*>(src0 + (size_t)c * plane);
+            if constexpr (sizeof(T) == 2) {
+              raw[it] = __ldg(src);
+            } else {
+              raw[2 * it] = __ldg(src);
+              raw[2 * it + 1] = __ldg(src + 1);
+            }
+          }
+        }
+#pragma unroll
+        for (int it = 0; it < kIt; ++it) {
+          const int c = cq + 8 * it;
+          if (c >= D) break;
           float f[8];
           if constexpr (sizeof(T) == 2) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(src0 + (size_t)c * plane));
+            const uint4 q = raw[it];
             *reinterpret_cast<uint4*>(unit_ptr(tile, c)) = q;
             const __half2* h = reinterpret_cast<const __half2*>(&q);
 #pragma unroll
@@ -182,8 +214,8 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
               f[2 * i + 1] = v.y;
             }
           } else {
-            const float4* src = reinterpret_cast<const float4*>(src0 + (size_t)c * plane);
-            const float4 lo4 = __ldg(src), hi4 = __ldg(src + 1);
+            const float4 lo4 = *reinterpret_cast<const float4*>(&raw[2 * it]);
+            const float4 hi4 = *reinterpret_cast<const float4*>(&raw[2 * it + 1]);
             f[0] = lo4.x; f[1] = lo4.y; f[2] = lo4.z; f[3] = lo4.w;
             f[4] = hi4.x; f[5] = hi4.y; f[6] = hi4.z; f[7] = hi4.w;
             __half hh[8], hl[8];
