@@ -361,11 +361,15 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
           unpack_vec<T>(raw[2 * ll], s);
           unpack_vec<T>(raw[2 * ll + 1], c);
 #pragma unroll
-          for (int j = 0; j < VEC; ++j) {
-            fin[j] = fold_finite(fin[j], s[j], c[j]);
-            if (l < Fu) {
-              const float u = atan2_ht(s[j], c[j]);
-              p[j] = (l == 0) ? u : refine_scaled(p[j], u);
+          for (int j = 0; j < VEC; ++j) fin[j] = fold_finite(fin[j], s[j], c[j]);
+          if (l < Fu) {
+            // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
+#pragma unroll
+            for (int j = 0; j < VEC; j += 2) {
+              const float2 u = atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
+              const float2 v = (l == 0) ? u : refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
+              p[j] = v.x;
+              p[j + 1] = v.y;
             }
           }
         }
