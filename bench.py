@@ -416,6 +416,10 @@ def run_ours(args, cfg):
                                          for n in sorted({cfg.name, "c3", "c5"})}
         except Exception as exc:
             line["refined_centroids"] = {"error": repr(exc)}
+        try:   # what the chain of launches costs by itself
+            line["launch_floor"] = measure_launch_floor(cfg, 200, 10, dev)
+        except Exception as exc:
+            line["launch_floor"] = {"error": repr(exc)}
         try:
             line["soft_votes"] = measure_soft_votes(cfg, max(20, min(K, 100)), max(3, min(Wm, 10)), dev)
         except Exception as exc:
@@ -471,6 +475,35 @@ def measure_other(cfg, steps, warmup, dev, refine=False):
             "instances_found": count, "one_read_embedding_roofline_us": one_read_us,
             "frac_of_one_read_roofline": one_read_us / (p50 * 1e3),
             "frac_of_algorithmic_bytes_roofline": alg / (peak_gbs * 1e9) / (p50 * 1e-3)}
+
+
+def measure_launch_floor(cfg, steps, warmup, dev):
+    """The decode's graph on the workload's shape with an all-zero mask: no pixel votes, no peak is found, nothing is
+    scored; the kernels still start, synchronise with their predecessors, read the mask and write the (all-zero) label
+    map.  Its replay time is what the chain of four dependent launches costs before any of the method's arithmetic."""
+    import torch
+    from paper_2609_16874_b200 import binding as cb
+    dt = torch.float32 if cfg.dtype == "f32" else torch.float16
+    emb = torch.zeros(cfg.B, cfg.D, cfg.H, cfg.W, dtype=dt, device=dev)
+    fg = torch.zeros(cfg.B, cfg.H, cfg.W, dtype=torch.uint8, device=dev)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        graph = dec.capture(emb, fg, stream=stream)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(warmup + steps):
+            j = i - warmup
+            if j >= 0:
+                ev[j][0].record(stream)
+            dec.replay(graph, stream=stream)
+            if j >= 0:
+                ev[j][1].record(stream)
+        stream.synchronize()
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    dec.close()
+    return {"workload": cfg.name + " shape, all-zero mask", "steps": steps, "p50_ms": float(np.percentile(step_ms, 50)),
+            "mean_ms": float(step_ms.mean()),
+            "note": "same four-node graph; no votes, no peaks, no scoring; mask read and label map written"}
 
 
 # Ceiling of the special-function units: 148 SMs x 16 results per clock x 1.965 GHz.
