@@ -342,7 +342,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   // The per-bin sums of the refinement: a small map, which one CTA of the peak kernel handles per image, is cleared
   // by that CTA after its last read; otherwise (or when the intermediates are to stay readable) they are cleared here.
   long long* sums = (p->flags & CPE_FLAG_REFINE) ? reinterpret_cast<long long*>(ws + L.sums) : nullptr;
-  const bool one_peak_cta = L.words <= 8 * (cpe::kPeakThreads / 32);
+  const bool one_peak_cta = L.words <= cpe::kPeakStageWords;
   const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes;
   if (sums && !sums_cleared_by_peaks) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
@@ -358,10 +358,12 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     // small maps: one CTA per image does both phases without the cross-CTA hand-over
     const int ctas = one_peak_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
     dim3 grid((unsigned)ctas, (unsigned)B);
-    CPE_CUDA(launch_dependent(cpe::peaks_kernel, grid, cpe::kPeakThreads, 0, st, votes, p->bins_w, p->bins_h, L.words,
+    // one CTA per image: it works on a copy of the vote map in shared memory (at most 32 KB)
+    const size_t map_smem = one_peak_cta ? 4 * (size_t)L.cells : 0;
+    CPE_CUDA(launch_dependent(cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes, p->bins_w, p->bins_h, L.words,
                               (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W, pal_w, pal_h, peak_cell,
                               peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums,
-                              sums_cleared_by_peaks ? 1 : 0));
+                              sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0));
     CPE_CUDA(cudaGetLastError());
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;

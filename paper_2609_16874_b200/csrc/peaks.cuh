@@ -7,7 +7,9 @@
 namespace cpe {
 
 constexpr int kPeakThreads = 1024;   // wide CTAs: the last one of an image does the whole compaction
-constexpr int kRefineChunk = 1024;     // peaks whose refined positions are staged in shared memory at a time
+constexpr int kRefineChunk = 512;     // peaks whose refined positions are staged in shared memory at a time
+constexpr int kPeakStageWords = 8 * (kPeakThreads / 32);   // largest map (in bitmap words) that one CTA does alone
+constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared memory when one CTA does the image
 
 // Phase 1 (every CTA): one thread per bin, one warp per 32 consecutive bins; the warp's ballot is one word
 // of the peak indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it
@@ -25,26 +27,47 @@ constexpr int kRefineChunk = 1024;     // peaks whose refined positions are stag
 // other peak there, so those votes are its own -- and its embedding is gamma(mean) of Eq. 2, evaluated in binary64
 // and rounded once, the way the palette rows are made.  `zero_sums` (only with one CTA per image): the sums are cleared
 // at the end, so that the decode needs no clearing pass for them.
+//
+// `staged` (only with one CTA per image; needs 4 * bins_w * bins_h bytes of dynamic shared memory): the CTA first
+// copies the whole vote map into shared memory with independent loads -- one round trip to L2 instead of one or two
+// per 32-bin word and warp iteration -- and keeps the bitmap and the head of the peak list there as well, so that
+// the dependent steps of this latency-bound kernel stay on the SM.
 __global__ void __launch_bounds__(kPeakThreads)
 peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
              uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
              uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
-             long long* __restrict__ sums, int zero_sums) {
+             long long* __restrict__ sums, int zero_sums, int staged) {
+  extern __shared__ uint32_t s_map[];                 // [cells] when staged
+  __shared__ uint32_t s_bm[kPeakStageWords];
+  __shared__ int s_pc[kPeakListStage];
   grid_dependency_sync();
   const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int cells = bins_w * bins_h;
   const uint32_t* V = votes + (size_t)b * cells;
   uint32_t* bm = bitmap + (size_t)b * words;
+  // the voting kernel's accumulators are wanted by thread 0 near the end: fetched now, off the critical path
+  uint32_t acc_voting = 0, acc_nonfinite = 0;
+  if (tid == 0) {
+    acc_voting = __ldcg(&acc[b * kAccStride + kAccVoting]);
+    acc_nonfinite = __ldcg(&acc[b * kAccStride + kAccNonfinite]);
+  }
+  if (staged) {
+    for (int i = tid; i < cells; i += kPeakThreads) s_map[i] = __ldcg(V + i);
+    __syncthreads();
+  }
+  auto vote_at = [&](int i) -> uint32_t { return staged ? s_map[i] : __ldg(V + i); };
+  auto bitmap_at = [&](int w) -> uint32_t { return staged ? s_bm[w] : __ldcg(bm + w); };
+  auto cell_of = [&](const int32_t* list, int k) -> int { return (staged && k < kPeakListStage) ? s_pc[k] : list[k]; };
 
   // ---- phase 1 (a CTA takes the words blockIdx.x*32 + wid, then strides by the grid: one CTA per image for small maps)
   for (int warp = blockIdx.x * (kPeakThreads / 32) + wid; warp < words; warp += gridDim.x * (kPeakThreads / 32)) {
     const int lin = warp * 32 + lane;
     bool peak = false;
     if (lin < cells) {
-      const uint32_t v = __ldg(V + lin);
+      const uint32_t v = vote_at(lin);
       if (v > T_v) {
         const int cy = lin / bins_w, cx = lin - cy * bins_w;
         peak = true;
@@ -56,14 +79,17 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
             const int ny = cy + dy, nx = cx + dx;
             if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
             const int nlin = ny * bins_w + nx;
-            const uint32_t nv = __ldg(V + nlin);
+            const uint32_t nv = vote_at(nlin);
             if (nv > v || (nv == v && nlin < lin)) peak = false;
           }
         }
       }
     }
     const uint32_t word = __ballot_sync(0xffffffffu, peak);
-    if (lane == 0) bm[warp] = word;
+    if (lane == 0) {
+      bm[warp] = word;
+      if (staged) s_bm[warp] = word;
+    }
   }
 
   // ---- which CTA of this image is the last one?  (with one CTA per image there is nothing to ask)
@@ -88,7 +114,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   const int per = (words + kPeakThreads - 1) / kPeakThreads;
   const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
   int local = 0;
-  for (int w = w0; w < w1; ++w) local += __popc(__ldcg(bm + w));
+  for (int w = w0; w < w1; ++w) local += __popc(bitmap_at(w));
 
   __shared__ int s_warp[kPeakThreads / 32];
   __shared__ int s_total;
@@ -100,28 +126,31 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   }
   if (lane == 31) s_warp[wid] = incl;
   __syncthreads();
-  if (tid == 0) {
-    int run = 0;
+  if (wid == 0) {                      // exclusive scan of the 32 warp totals by the first warp
+    static_assert(kPeakThreads / 32 == 32, "one lane per warp total");
+    const int mine = s_warp[lane];
+    int inc = mine;
 #pragma unroll
-    for (int w = 0; w < kPeakThreads / 32; ++w) {
-      const int t = s_warp[w];
-      s_warp[w] = run;
-      run += t;
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += t;
     }
-    s_total = run;
+    s_warp[lane] = inc - mine;
+    if (lane == 31) s_total = inc;
   }
   __syncthreads();
   int slot = s_warp[wid] + incl - local;
   const int total = s_total;
 
   for (int w = w0; w < w1 && slot < K_max; ++w) {
-    uint32_t bits = __ldcg(bm + w);
+    uint32_t bits = bitmap_at(w);
     while (bits && slot < K_max) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
       const int lin = w * 32 + bit;
       pc[slot] = lin;
-      pv[slot] = V[lin];
+      if (staged && slot < kPeakListStage) s_pc[slot] = lin;
+      pv[slot] = vote_at(lin);
       ++slot;
     }
   }
@@ -129,7 +158,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   if (tid == 0) {
     out_count[b] = count;
     // fold the voting kernel's accumulators into this image's counters, and leave them zero for the next decode
-    const uint32_t voting = acc[b * kAccStride + kAccVoting], nonfinite = acc[b * kAccStride + kAccNonfinite];
+    const uint32_t voting = acc_voting, nonfinite = acc_nonfinite;
     acc[b * kAccStride + kAccVoting] = 0u;
     acc[b * kAccStride + kAccNonfinite] = 0u;
     acc[b * kAccStride + kAccTicket] = 0u;
@@ -157,7 +186,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
       const int nk = min(kRefineChunk, count - k0);
       for (int i = tid; i < 2 * nk; i += kPeakThreads) {       // (peak, axis): pooled mean of the 3x3 window
         const int k = k0 + (i >> 1), axis = i & 1;
-        const int lin = pc[k];
+        const int lin = cell_of(pc, k);
         const int cy = lin / bins_w, cx = lin - cy * bins_w;
         long long s = 0, n = 0;
 #pragma unroll
@@ -167,7 +196,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
             const int ny = cy + dy, nx = cx + dx;
             if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
             const int nlin = ny * bins_w + nx;
-            n += (long long)V[nlin];
+            n += (long long)vote_at(nlin);
             s += __ldcg(S + 2 * (size_t)nlin + axis);
           }
         }
@@ -196,12 +225,12 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   }
   for (int i = tid; i < count * D; i += kPeakThreads) {
     const int k = i / D, c = i - k * D;
-    const int lin = pc[k];
+    const int lin = cell_of(pc, k);
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     pe[i] = (c < 2 * F) ? pal_w[cx * 2 * F + c] : pal_h[cy * 2 * F + (c - 2 * F)];
   }
   for (int k = tid; k < count; k += kPeakThreads) {
-    const int lin = pc[k];
+    const int lin = cell_of(pc, k);
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     // bin position -1 + 2i/(n+1), i = c+1 (Eq. 9); pixel centres sit at x = -1 + (2 col + 1)/W
     const double x = -1.0 + 2.0 * (double)(cx + 1) / (double)(bins_w + 1);
