@@ -416,6 +416,11 @@ def run_ours(args, cfg):
                                          for n in sorted({cfg.name, "c3", "c5"})}
         except Exception as exc:
             line["refined_centroids"] = {"error": repr(exc)}
+        try:   # a caller that bounds its instance count inside the all-pairs range: one launch fewer
+            if cfg.name in ("c1", "c2"):
+                line["max_instances_32"] = measure_other(cfg, 200, 10, dev, k_max=32)
+        except Exception as exc:
+            line["max_instances_32"] = {"error": repr(exc)}
         try:   # what the chain of launches costs by itself
             line["launch_floor"] = measure_launch_floor(cfg, 200, 10, dev)
         except Exception as exc:
@@ -436,9 +441,9 @@ def run_ours(args, cfg):
     dist_util.shutdown()
 
 
-def measure_other(cfg, steps, warmup, dev, refine=False):
+def measure_other(cfg, steps, warmup, dev, refine=False, k_max=None):
     """Graph-replay timing of one more workload (no host leg, no CPU baseline): p50, MP/s, per-stage times.
-    `refine`: with sub-cell refined centroids (CPE_FLAG_REFINE)."""
+    `refine`: with sub-cell refined centroids (CPE_FLAG_REFINE); `k_max`: max_instances other than the workload's."""
     import torch
     from paper_2609_16874_b200 import binding as cb
     n_frames = frames_needed(cfg)
@@ -446,8 +451,8 @@ def measure_other(cfg, steps, warmup, dev, refine=False):
     d_emb = [torch.from_numpy(f["emb"]).to(dev) for f in frames]
     d_fg = [torch.from_numpy(f["fg"]).to(dev) for f in frames]
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if n_frames * cfg.emb_bytes < 2 * L2_BYTES else None
-    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, device=dev,
-                     refine=refine)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau,
+                     k_max if k_max else cfg.K_max, device=dev, refine=refine)
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         graphs = [dec.capture(d_emb[i], d_fg[i], stream=stream) for i in range(n_frames)]

@@ -135,7 +135,9 @@ typedef struct cpe_params {
   int32_t levels;          /* harmonics used by the centroid estimate; 0 or >= F means all F   */
   int32_t vote_threshold;  /* T_v >= 0: a peak needs V > T_v ("predefined threshold", Sec. 3.2) */
   float tau;               /* Eq. 8: a pixel keeps its label iff d < tau; +inf keeps every one */
-  int32_t max_instances;   /* K_max: capacity per image of the peak / centroid arrays          */
+  int32_t max_instances;   /* K_max: capacity per image of the peak / centroid arrays.  Up to 32
+                              (16 when F > 8) the decode enqueues one kernel fewer: no image can
+                              then need the tensor-core assignment.                            */
   uint32_t flags;          /* CPE_FLAG_*                                                       */
   void* workspace;         /* device memory, 256-byte aligned, owned by the caller             */
   size_t workspace_bytes;  /* >= cpe_workspace_size(...) for the same B, H, W, F and params    */

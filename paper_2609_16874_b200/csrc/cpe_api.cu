@@ -262,6 +262,11 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   // exactly one of them: all pairs on the plain ALUs when an image has few peaks (the fixed cost of the
   // tensor-core filter does not pay), the filtered kernel otherwise.  The other kernel's CTAs exit at once.
   const int k_limit = (p->flags & CPE_FLAG_FILTER_ASSIGN) ? 0 : (F <= 8 ? 32 : 16);
+  // A caller whose max_instances already is within the all-pairs range needs no second kernel: no image can have
+  // more peaks than that (the list is truncated to max_instances), so the chain is one launch shorter.
+  if (p->max_instances <= k_limit)
+    return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                  votes_to_zero, cells, 0x7fffffff);
   int rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
                                   cells, k_limit);
   if (rc) return rc;

@@ -346,3 +346,34 @@ def test_between_65_and_128_peaks_both_tensor_memory_stages_serve_one_tile(name,
     assert 64 < ora["count"].max() <= 128, ora["count"]
     assert gpu["status"] == 0
     print(name, over, ora["count"].tolist(), rep)
+
+
+def test_small_max_instances_takes_the_three_kernel_chain():
+    """With max_instances inside the all-pairs range no image can need the filtered kernel, so it is not enqueued:
+    the captured graph has three kernel nodes instead of four, results are the oracle's, and replays repeat them
+    (the all-pairs kernel then is the one that leaves the vote map zero for the next decode)."""
+    import torch
+    cfg = wl.scaled(wl.CONFIGS["c2"], H=192, W=256, K=12, bins_w=48, bins_h=32)
+    fr = wl.make_frame(cfg, 0)
+    check_case(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, K_max=32, mode="graph")
+    ora = oracle.decode(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, 32)
+    emb, fg = torch.from_numpy(fr["emb"]).cuda(), torch.from_numpy(fr["fg"]).cuda()
+    nodes = {}
+    for k_max in (32, 33):
+        dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, k_max)
+        stream = torch.cuda.Stream()          # capture needs a stream of its own, not the default one
+        torch.cuda.synchronize()
+        g = dec.capture(emb, fg, stream=stream)
+        nodes[k_max] = cb.cpe_graph_kernel_nodes(g)
+        for _ in range(3):
+            dec.replay(g, stream=stream)
+            torch.cuda.synchronize()
+            n = int(ora["count"][0])
+            assert int(dec.count.cpu()[0]) == n
+            assert np.array_equal(dec.intermediate(cb.CPE_INT_PEAK_CELLS).cpu().numpy()[0, :n], ora["peak_cell"][0, :n])
+            lab = dec.labels.cpu().numpy()
+            with np.errstate(invalid="ignore"):
+                near_tie = (ora["second"] - ora["best"]) < 1e-5
+            assert ((lab == ora["labels"]) | near_tie).all()
+        dec.close()
+    assert nodes[32] == nodes[33] - 1, nodes
