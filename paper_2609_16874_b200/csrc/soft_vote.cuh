@@ -320,23 +320,25 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     constexpr uint64_t kLoTile = (uint64_t)((kPartHalves * 2) >> 4);        // low part of a pixel tile
     uint32_t t = 0;
     bool bad = false;
-    const float log2e = 1.4426950408889634f;
+    const float log2e_sq = 2.0813689810056077f;         // log2(e)^2
     const int na = min(kSvBins, bins_w - a0), nb = min(kSvBins, bins_h - b0);   // bins of this block that exist
 
-    // exp(-sqrt(max(c + D, 0))) for 8 consecutive bins, rounded to binary16.  The special-function unit's
+    // exp(-sqrt(|c + D|)) for 8 consecutive bins, rounded to binary16, as 2^(-sqrt(|c + D| log2(e)^2)): one fused
+    // multiply-add, two special-function results.  (The squared distance is non-negative up to the rounding of its
+    // three terms, about 1e-6; its magnitude stands in for max(., 0) and costs nothing.)  The special-function unit's
     // approximations (sqrt, 2^x: about 2^-22 relative each) are far inside the binary16 rounding that follows; the
     // flush-to-zero forms are single instructions (a subnormal argument or result is below anything binary16 holds:
-    // its smallest subnormal is e^-16.6).  A row without a pixel is masked after packing.
-    auto weights8 = [&](const float* v, float c, bool live) -> uint4 {
+    // its smallest subnormal is e^-16.6).  A row without a pixel is masked after packing.  `ck` = c log2(e)^2.
+    auto weights8 = [&](const float* v, float ck, bool live) -> uint4 {
       uint32_t w[4];
       const uint32_t keep = live ? 0xffffffffu : 0u;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float d0, d1, e0, e1;
-        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d0) : "f"(fmaxf(c + v[2 * i], 0.0f)));
-        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d1) : "f"(fmaxf(c + v[2 * i + 1], 0.0f)));
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-d0 * log2e));
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-d1 * log2e));
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d0) : "f"(fabsf(fmaf(v[2 * i], log2e_sq, ck))));
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d1) : "f"(fabsf(fmaf(v[2 * i + 1], log2e_sq, ck))));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-d0));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-d1));
         const __half2 h = __floats2half2_rn(e0, e1);
         w[i] = *reinterpret_cast<const uint32_t*>(&h) & keep;
       }
@@ -391,7 +393,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     }
     while (!bad && !(flags & kRfEnd)) {
       const bool live = (flags & kRfLive) != 0;
-      const float c_row = cn;
+      const float c_row = cn * log2e_sq;
       {
         const bool ok = mbar_wait(mb_d, t & 1u, s_abort);   // GEMM 1 of this tile (and every MMA before it) is done
         if (!__all_sync(0xffffffffu, ok)) { bad = true; break; }
