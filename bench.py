@@ -81,22 +81,29 @@ class ClockSampler:
         except Exception:
             self.nv = None
 
-    def _poll(self):
+    def sample(self):
+        """One reading, now (also called from the timing loop itself, while the GPU works through the queued steps:
+        the polling thread gets few turns while the main thread is busy submitting)."""
         nv = self.nv
+        if nv is None:
+            return
+        try:
+            mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            try:
+                r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+            except Exception:
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            self.samples.append(mhz)
+            for bit, name in self.REASONS.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _poll(self):
         while not self._stop.is_set():
             if self._active.is_set():
-                try:
-                    mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
-                    try:
-                        r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
-                    except Exception:
-                        r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                    self.samples.append(mhz)
-                    for bit, name in self.REASONS.items():
-                        if r & bit:
-                            self.reasons.add(name)
-                except Exception:
-                    pass
+                self.sample()
             time.sleep(0.002)
 
     def start(self):
@@ -257,6 +264,9 @@ def run_ours(args, cfg):
         sampler.window(True)
         for i in range(K):
             step(i, *ev[i])
+            if i % 256 == 128:
+                sampler.sample()      # between two submissions; the steps are timed by their own events
+        sampler.sample()
         stream.synchronize()
         torch.cuda.synchronize(dev)
         sampler.window(False)
