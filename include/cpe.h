@@ -65,6 +65,16 @@ enum {
   CPE_FLAG_KEEP_VOTES = 4u,   /* leave the vote map readable after the decode (CPE_INT_VOTES).  Without it the
                                  last kernel of a decode re-zeroes the map for the next decode, which saves the
                                  clearing pass at the start; with it every decode starts with that pass.       */
+  CPE_FLAG_NO_PDL = 32u,      /* launch the kernels of a decode plainly, without programmatic stream serialisation
+                                 (A/B timing; same results)                                                    */
+  CPE_FLAG_TC_ALL_ROUNDS = 64u,   /* filtered assignment: let the tensor-memory (tcgen05) body take every image whose
+                                     peaks fit its shared-memory operand, in rounds of 64, instead of handing images
+                                     with more than 128 peaks to the mma.sync body (tests, comparisons; same results) */
+  CPE_FLAG_TC_ONE_STAGE = 128u,   /* ... or only images with at most 64 peaks (one tensor-memory stage per tile)     */
+  CPE_FLAG_MMA_ASSIGN = 256u,     /* filtered assignment: the mma.sync kernel for every image (comparisons)          */
+  CPE_FLAG_NO_PRUNE = 512u,       /* do not prune the candidates of Eq. 7 (see cpe_decode): every image with more peaks
+                                     than the all-pairs range goes to the tensor-core filtered kernels; same results  */
+  CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment for every image, however few peaks it has; same results    */
   CPE_FLAG_REFINE = 16u       /* sub-cell refined centroids (an extension: the paper's candidates of Eq. 7 are the
                                  bin positions of Eq. 9, up to half a bin off the voted centroid).  Next to its
                                  count every bin keeps the sum of the estimates that fell into it, as integers
@@ -115,7 +125,11 @@ enum {
   CPE_INT_VOTE_SUMS = 10,   /* int64  [B][bins_h][bins_w][2]    fixed-point (2^-24) sums of the x and y
                                                                 estimates per bin (CPE_FLAG_REFINE and
                                                                 CPE_FLAG_KEEP_VOTES)                 */
-  CPE_INT_N = 11
+  CPE_INT_PRUNE_STATE = 11, /* uint32 [B][8]  the pruned assignment's words of each image (only when it is enabled):
+                                                [0] pixels visited, [1] pixels whose candidate list did not settle them,
+                                                [2] non-zero: the image was handed to the tensor-core filtered kernel,
+                                                [4..7] that kernel's own counters (folded into CPE_INT_COUNTERS)  */
+  CPE_INT_N = 12
 };
 
 /* stages reported by cpe_profile_decode */
@@ -123,7 +137,7 @@ enum {
   CPE_STAGE_CLEAR = 0,      /* zeroing of the vote map (only with CPE_FLAG_KEEP_VOTES; else ~0)  */
   CPE_STAGE_DECODE_VOTE = 1,
   CPE_STAGE_PEAKS = 2,      /* local-maximum test, ordered peak list, centroids, peak embeddings */
-  CPE_STAGE_COMPACT = 3,    /* (merged into CPE_STAGE_PEAKS; reported as ~0)                     */
+  CPE_STAGE_LISTS = 3,      /* per-peak candidate lists of the pruned assignment (~0 without it) */
   CPE_STAGE_ASSIGN = 4,     /* assignment and label-map write                                    */
   CPE_STAGE_N = 5
 };

@@ -28,12 +28,19 @@ CPE_FLAG_EXACT_ASSIGN = 2
 CPE_FLAG_KEEP_VOTES = 4
 CPE_FLAG_FILTER_ASSIGN = 8
 CPE_FLAG_REFINE = 16
+CPE_FLAG_NO_PDL = 32
+CPE_FLAG_TC_ALL_ROUNDS = 64
+CPE_FLAG_TC_ONE_STAGE = 128
+CPE_FLAG_MMA_ASSIGN = 256
+CPE_FLAG_NO_PRUNE = 512
+CPE_FLAG_PRUNE_ALL = 1024
 CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL = 1, 2, 4
 CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
 CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8
 (CPE_INT_VOTES, CPE_INT_PEAK_CELLS, CPE_INT_PEAK_VOTES, CPE_INT_PEAK_EMB, CPE_INT_PALETTE_W, CPE_INT_PALETTE_H,
- CPE_INT_BEST_SCORE, CPE_INT_SECOND_SCORE, CPE_INT_STATUS, CPE_INT_COUNTERS, CPE_INT_VOTE_SUMS) = range(11)
-CPE_STAGE_NAMES = ("clear", "decode_vote", "peaks", "compact", "assign")
+ CPE_INT_BEST_SCORE, CPE_INT_SECOND_SCORE, CPE_INT_STATUS, CPE_INT_COUNTERS, CPE_INT_VOTE_SUMS,
+ CPE_INT_PRUNE_STATE) = range(12)
+CPE_STAGE_NAMES = ("clear", "decode_vote", "peaks", "lists", "assign")
 CPE_STAGE_N = 5
 
 EXPORTS = (
@@ -260,7 +267,7 @@ class Decoder:
 
     def __init__(self, B, H, W, F, dtype, bins_w, bins_h, vote_threshold=8, tau=math.inf, max_instances=1024,
                  levels=0, write_scores=False, device="cuda:0", exact_assign=False, keep_votes=False, filter_assign=False,
-                 refine=False):
+                 refine=False, flags=0):
         import torch
         self.torch = torch
         self.B, self.H, self.W, self.F = B, H, W, F
@@ -269,7 +276,7 @@ class Decoder:
         self.emb_dtype = torch.float32 if code == CPE_F32 else torch.float16
         flags = ((CPE_FLAG_WRITE_SCORES if write_scores else 0) | (CPE_FLAG_EXACT_ASSIGN if exact_assign else 0) |
                  (CPE_FLAG_KEEP_VOTES if keep_votes else 0) | (CPE_FLAG_FILTER_ASSIGN if filter_assign else 0) |
-                 (CPE_FLAG_REFINE if refine else 0))
+                 (CPE_FLAG_REFINE if refine else 0) | int(flags))
         self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances, flags)
         n = cpe_workspace_size(B, H, W, F, self.params)
         if n == 0:
@@ -362,6 +369,7 @@ class Decoder:
             CPE_INT_STATUS: (torch.int32, (self.B,)),
             CPE_INT_COUNTERS: (torch.int32, (self.B, CPE_CNT_N)),
             CPE_INT_VOTE_SUMS: (torch.int64, (self.B, bh, bw, 2)),
+            CPE_INT_PRUNE_STATE: (torch.int32, (self.B, 8)),
         }
         dt, shape = shapes[which]
         return raw.view(dt).view(shape)
@@ -382,10 +390,10 @@ class HostDecoder:
     """End-to-end front end for host buffers (``cpe_host_ctx_*``): numpy in, numpy out, copies included."""
 
     def __init__(self, B, H, W, F, dtype, bins_w, bins_h, vote_threshold=8, tau=math.inf, max_instances=1024,
-                 levels=0, has_mask=True, refine=False):
+                 levels=0, has_mask=True, refine=False, flags=0):
         code = {"f32": CPE_F32, "f16": CPE_F16}[dtype]
         self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances,
-                                  CPE_FLAG_REFINE if refine else 0)
+                                  (CPE_FLAG_REFINE if refine else 0) | int(flags))
         self.shape = (B, H, W, F)
         self.max_instances = max_instances
         rc, self.ctx = cpe_host_ctx_create(B, H, W, F, self.params, has_mask)

@@ -868,8 +868,13 @@ assign_mma_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int
                   const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
                   int peak_cap, int span, int vec_mask, int vec_gather, int32_t* __restrict__ labels, float* __restrict__ best,
                   float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
-                  uint32_t* __restrict__ votes, int cells, int k_min) {
+                  uint32_t* __restrict__ votes, int cells, int k_min, const uint32_t* __restrict__ near_state) {
   grid_dependency_sync();
+  // after the pruned assignment (near_state given) this kernel only takes the images which that one handed on
+  if (near_state) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) fold_near_counters(near_state, counters, blockIdx.y);
+    if (!near_state[blockIdx.y * kNearStride + kNearGiveUp]) k_min = 0x7fffffff;
+  }
   assign_mma_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status_all, votes, cells, k_min);
 }
 

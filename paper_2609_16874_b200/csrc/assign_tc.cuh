@@ -1080,9 +1080,14 @@ assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, 
                      int tc_peak_cap, int tc_k_max, int tc_vec_mask, int mma_peak_cap, int mma_span, int mma_vec_mask,
                      int mma_vec_gather, int32_t* __restrict__ labels, float* __restrict__ best, float* __restrict__ second,
                      uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all, uint32_t* __restrict__ votes, int cells,
-                     int k_min, uint32_t* __restrict__ acc) {
+                     int k_min, uint32_t* __restrict__ acc, const uint32_t* __restrict__ near_state) {
   static_assert(kTcThreads == kAmThreads, "both bodies run with the same block size");
   grid_dependency_sync();
+  // after the pruned assignment (near_state given) this kernel only takes the images which that one handed on
+  if (near_state) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) fold_near_counters(near_state, counters, blockIdx.y);
+    if (!near_state[blockIdx.y * kNearStride + kNearGiveUp]) k_min = 0x7fffffff;
+  }
   if (count_ptr[blockIdx.y] <= tc_k_max)
     assign_tc_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, tc_peak_cap, tc_vec_mask, labels,
                                  best, second, counters, status_all, votes, cells, k_min, tc_k_max, acc);
@@ -1092,7 +1097,7 @@ assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, 
     if (threadIdx.x < 32) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     assign_mma_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, mma_peak_cap, mma_span,
                                   mma_vec_mask, mma_vec_gather, labels, best, second, counters, status_all, votes, cells,
-                                  tc_k_max + 1);
+                                  max(k_min, tc_k_max + 1));
   }
 }
 

@@ -11,30 +11,46 @@
 #include <vector>
 
 #include "assign.cuh"
-#include "assign_mma.cuh"
-#include "assign_tc.cuh"
 #include "cpe.h"
 #include "cpe_common.cuh"
-#include "decode_vote.cuh"
 #include "instance_masks.cuh"
+#include "launch.h"
 #include "layout.cuh"
 #include "peaks.cuh"
-#include "soft_vote.cuh"
 
 namespace {
-
 thread_local int g_last_cuda = 0;
+}
 
-inline int cuda_fail(cudaError_t e) {
+namespace cpe {
+namespace host {
+
+int cuda_fail(cudaError_t e) {
   g_last_cuda = (int)e;
   return CPE_ERR_CUDA;
 }
 
-#define CPE_CUDA(call)                          \
-  do {                                          \
-    cudaError_t e_ = (call);                    \
-    if (e_ != cudaSuccess) return cuda_fail(e_); \
-  } while (0)
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+}  // namespace host
+}  // namespace cpe
+
+namespace {
+
+using cpe::host::cuda_fail;
+using cpe::host::launch_dependent;
+using cpe::host::plain_launch;
+using cpe::host::sm_count;
 
 inline size_t elem_size(int dtype) { return dtype == CPE_F32 ? 4 : 2; }
 
@@ -59,95 +75,6 @@ int check_workspace(int B, int H, int W, int F, const cpe_params* p, cpe::Layout
   return CPE_OK;
 }
 
-int sm_count();
-
-// Launch of a kernel that consumes what the kernel before it in the stream wrote, with programmatic stream
-// serialisation: its CTAs may be scheduled while the predecessor is still running and wait on the device
-// (grid_dependency_sync at the top of every kernel of the chain).  CPE_PDL=0 in the environment launches plainly.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
-  static const bool plain = [] { const char* e = getenv("CPE_PDL"); return e && e[0] == '0'; }();
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = dim3((unsigned)threads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = plain ? 0 : 1;
-  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
-}
-
-template <typename T>
-int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                       uint32_t* votes, uint32_t* acc, long long* sums) {
-  const T* e = static_cast<const T*>(emb);
-  constexpr int V = cpe::Elem<T>::kVec;
-  // 128-bit plane loads: every plane of every image must start on a 16-byte boundary
-  const bool vec = ((uintptr_t)emb % 16 == 0) && (HW % V == 0) && (!fg || (uintptr_t)fg % V == 0) &&
-                   (F == 4 || F == 8 || F == 16);
-  if (vec) {
-    const long long groups = (long long)HW / V;
-    // the largest span that still gives one full wave of CTAs (three resident per SM), else the smallest
-    const long long wave = 3LL * sm_count();
-    const int span = (groups + 255) / 256 * B >= wave ? 256 : (groups + 127) / 128 * B >= wave ? 128 : 64;
-    dim3 grid((unsigned)((groups + span - 1) / span), (unsigned)B);
-#define CPE_LAUNCH_VOTE_G(FT_, RF_, G_)                                                                              \
-  cpe::decode_vote_vec_kernel<T, FT_, RF_, G_><<<grid, cpe::kVoteThreads, 0, st>>>(e, fg, HW, p->levels, p->bins_w,   \
-                                                                                  p->bins_h, votes, acc, sums)
-#define CPE_LAUNCH_VOTE_R(FT_, RF_)                                                                                   \
-  switch (span) {                                                                                                     \
-    case 256: CPE_LAUNCH_VOTE_G(FT_, RF_, 256); break;                                                                \
-    case 128: CPE_LAUNCH_VOTE_G(FT_, RF_, 128); break;                                                                \
-    default: CPE_LAUNCH_VOTE_G(FT_, RF_, 64); break;                                                                  \
-  }
-#define CPE_LAUNCH_VOTE(FT_)                                                                                          \
-  if (sums) { CPE_LAUNCH_VOTE_R(FT_, true) } else { CPE_LAUNCH_VOTE_R(FT_, false) }
-    switch (F) {
-      case 4: CPE_LAUNCH_VOTE(4); break;
-      case 8: CPE_LAUNCH_VOTE(8); break;
-      default: CPE_LAUNCH_VOTE(16); break;
-    }
-#undef CPE_LAUNCH_VOTE
-#undef CPE_LAUNCH_VOTE_R
-#undef CPE_LAUNCH_VOTE_G
-  } else {
-    // 64-bit mask loads need every image's mask to start on an 8-byte boundary
-    const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
-    dim3 grid((unsigned)(((long long)HW + cpe::kVoteSpan - 1) / cpe::kVoteSpan), (unsigned)B);
-#define CPE_LAUNCH_VOTE(FT_)                                                                                             \
-  if (sums)                                                                                                               \
-    cpe::decode_vote_scalar_kernel<T, FT_, true><<<grid, cpe::kVoteThreads, 0, st>>>(                                     \
-        e, fg, HW, F, p->levels, p->bins_w, p->bins_h, vec_mask, votes, acc, sums);                                       \
-  else                                                                                                                    \
-    cpe::decode_vote_scalar_kernel<T, FT_, false><<<grid, cpe::kVoteThreads, 0, st>>>(                                    \
-        e, fg, HW, F, p->levels, p->bins_w, p->bins_h, vec_mask, votes, acc, nullptr)
-    switch (F) {
-      case 4: CPE_LAUNCH_VOTE(4); break;
-      case 8: CPE_LAUNCH_VOTE(8); break;
-      case 16: CPE_LAUNCH_VOTE(16); break;
-      default: CPE_LAUNCH_VOTE(0); break;
-    }
-#undef CPE_LAUNCH_VOTE
-  }
-  CPE_CUDA(cudaGetLastError());
-  return CPE_OK;
-}
-
-int sm_count() {
-  static int cached[64] = {0};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (!cached[dev]) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
-
 template <typename T>
 int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                         const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
@@ -157,9 +84,10 @@ int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int
   const long long n_blocks = ((long long)HW + cpe::kAssignThreads - 1) / cpe::kAssignThreads;
   const long long per_image = std::max(1, (8 * sm_count() + B - 1) / B);
   dim3 grid((unsigned)std::min(n_blocks, per_image), (unsigned)B);
-#define CPE_LAUNCH_ASSIGN(FT_)                                                                                     \
-  CPE_CUDA(launch_dependent(cpe::assign_kernel<T, FT_>, grid, cpe::kAssignThreads, 0, st, e, fg, HW, F, p->max_instances, \
-                            peak_emb, count, p->tau, labels, best, second, counters, votes_to_zero, cells, k_limit))
+#define CPE_LAUNCH_ASSIGN(FT_)                                                                                          \
+  CPE_CUDA(launch_dependent(plain_launch(p), cpe::assign_kernel<T, FT_>, grid, cpe::kAssignThreads, 0, st, e, fg, HW, F, \
+                            p->max_instances, peak_emb, count, p->tau, labels, best, second, counters, votes_to_zero,   \
+                            cells, k_limit))
   switch (F) {
     case 4: CPE_LAUNCH_ASSIGN(4); break;
     case 8: CPE_LAUNCH_ASSIGN(8); break;
@@ -171,139 +99,69 @@ int launch_assign_exact(cudaStream_t st, const void* emb, const uint8_t* fg, int
   return CPE_OK;
 }
 
+// What the pruned assignment reads and writes besides the outputs (all inside the workspace).
+struct PruneArgs {
+  const float* ref_emb = nullptr;
+  float* ref2 = nullptr;
+  float* cand2 = nullptr;
+  uint32_t* nbr = nullptr;
+  const int32_t* cell_peak = nullptr;
+  const uint32_t* pix_cell = nullptr;
+  uint32_t* near_state = nullptr;
+};
 
-template <typename T, int KA, bool WANT2>
-int launch_assign_mma_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                        const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                        uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min) {
-  // small inputs get short spans so that there are enough CTAs to fill the GPU
-  const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
-  // 16-byte gathers of whole 8-pixel groups need aligned planes and the long span
-  const int vec_gather = (span == cpe::kAmSpanMax) && ((uintptr_t)e % 16 == 0) && (HW % 8 == 0);
-  const int two_tiles = (vec_gather && sizeof(T) == 2 && KA == 16) ? 1 : 0;
-  // as many peaks resident in shared memory as leave room for two CTAs per SM
-  int peak_cap = (p->max_instances + 7) & ~7;
-  const int budget = 110 * 1024;
-  const int fixed = cpe::am_smem_layout(KA, 0, span, two_tiles).total;
-  peak_cap = std::max(8, std::min(peak_cap, ((budget - fixed) / ((2 * KA + 8) * 2)) & ~7));
-  const int smem = cpe::am_smem_layout(KA, peak_cap, span, two_tiles).total;
-  auto kern = cpe::assign_mma_kernel<T, KA, WANT2>;
-  static bool configured = false;   // per instantiation; the attribute is sticky for the process
-  if (!configured) {
-    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-    configured = true;
-  }
-  const int n_spans = (HW + span - 1) / span;
-  const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
-  dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
-  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) && (HW % 8 == 0);
-  const int need_exact = p->tau < INFINITY ? 1 : 0;
-  CPE_CUDA(launch_dependent(kern, grid, cpe::kAmThreads, smem, st, e, fg, HW, F, p->max_instances, peak_emb, count, p->tau,
-                            need_exact, peak_cap, span, vec_mask, vec_gather, labels, best, second, counters, status,
-                            votes_to_zero, cells, k_min));
-  CPE_CUDA(cudaGetLastError());
-  return CPE_OK;
-}
-
-// The filtered assignment for 16-byte aligned planes: one launch, the tcgen05 pipeline for the images whose peaks
-// fit one of its rounds, the mma.sync body for the others (the choice is made on the device, per image).
-template <typename T, int KA, bool WANT2>
-int launch_assign_filter_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                           const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                           uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, int k_min, uint32_t* acc) {
-  // tcgen05 body: as many peaks resident in shared memory as leave room for two CTAs per SM (each CTA holds half of
-  // the SM's tensor memory, so there must never be more than two)
-  const int budget = 104 * 1024;
-  int tc_cap = (p->max_instances + cpe::kTcRound - 1) / cpe::kTcRound * cpe::kTcRound;
-  const int tc_fixed = cpe::tc_smem_layout(KA, 0).total;
-  tc_cap = std::max(cpe::kTcRound, std::min(tc_cap, (budget - tc_fixed) / (2 * KA * 2) / cpe::kTcRound * cpe::kTcRound));
-  // up to 128 peaks fit the two tensor-memory stages at once; beyond that the mma.sync body is the faster one
-  // (CPE_ASSIGN_PATH=tc lifts the limit: tests, comparisons; CPE_ASSIGN_PATH=tc64 keeps it at one stage)
-  static const char* path = getenv("CPE_ASSIGN_PATH");
-  const int tc_k_max = (path && strcmp(path, "tc") == 0)     ? tc_cap
-                       : (path && strcmp(path, "tc64") == 0) ? std::min(tc_cap, cpe::kTcRound)
-                                                             : std::min(tc_cap, 2 * cpe::kTcRound);
-  const int tc_smem = cpe::tc_smem_layout(KA, tc_cap).total;
-  // mma.sync body
-  const int span = ((long long)B * HW >= (1 << 20)) ? cpe::kAmSpanMax : 512;
-  const int vec_gather = span == cpe::kAmSpanMax ? 1 : 0;
-  const int two_tiles = (vec_gather && sizeof(T) == 2 && KA == 16) ? 1 : 0;
-  int mma_cap = (p->max_instances + 7) & ~7;
-  const int mma_fixed = cpe::am_smem_layout(KA, 0, span, two_tiles).total;
-  mma_cap = std::max(8, std::min(mma_cap, ((110 * 1024 - mma_fixed) / ((2 * KA + 8) * 2)) & ~7));
-  const int mma_smem = cpe::am_smem_layout(KA, mma_cap, span, two_tiles).total;
-  const int smem = std::max(std::max(tc_smem, mma_smem), 78 * 1024);
-  auto kern = cpe::assign_filter_kernel<T, KA, WANT2>;
-  static bool configured = false;   // per instantiation; the attribute is sticky for the process
-  if (!configured) {
-    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-    configured = true;
-  }
-  const int n_spans = (HW + cpe::kTcSpan - 1) / cpe::kTcSpan;
-  const int per_image = std::max(1, (2 * sm_count() + B - 1) / B);
-  dim3 grid((unsigned)std::min(n_spans, per_image), (unsigned)B);
-  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
-  const int need_exact = p->tau < INFINITY ? 1 : 0;
-  CPE_CUDA(launch_dependent(kern, grid, cpe::kTcThreads, smem, st, e, fg, HW, F, p->max_instances, peak_emb, count, p->tau,
-                            need_exact, tc_cap, tc_k_max, vec_mask, mma_cap, span, vec_mask, vec_gather, labels, best, second,
-                            counters, status, votes_to_zero, cells, k_min, acc));
-  CPE_CUDA(cudaGetLastError());
-  return CPE_OK;
-}
-
+// Stage 4+5.  The number of peaks is only known on the device, so several kernels are enqueued and every image is
+// done by exactly one of them; the CTAs of the others exit at once:
+//   - all pairs on the plain ALUs when an image has few peaks (the fixed costs of the others do not pay);
+//   - else, with pruning enabled, the kernel that walks per-peak candidate lists (after the kernel that makes them);
+//   - else (pruning disabled, or that kernel handed the image on) the tensor-core filtered kernel.
+// `ev_lists`: an event recorded between the list kernel and the assignment kernels (per-stage timing).
 template <typename T>
 int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                   const float* peak_emb, const int32_t* count, int32_t* labels, float* best, float* second,
-                  uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, uint32_t* acc) {
-  if (p->flags & CPE_FLAG_EXACT_ASSIGN)
+                  uint32_t* counters, uint32_t* status, uint32_t* votes_to_zero, int cells, uint32_t* acc,
+                  const PruneArgs* pr, cudaEvent_t ev_lists) {
+  if (p->flags & CPE_FLAG_EXACT_ASSIGN) {
+    if (ev_lists) CPE_CUDA(cudaEventRecord(ev_lists, st));
     return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
                                   votes_to_zero, cells, 0x7fffffff);
-  // The number of peaks is only known on the device.  Two kernels are enqueued and every image is done by
-  // exactly one of them: all pairs on the plain ALUs when an image has few peaks (the fixed cost of the
-  // tensor-core filter does not pay), the filtered kernel otherwise.  The other kernel's CTAs exit at once.
-  const int k_limit = (p->flags & CPE_FLAG_FILTER_ASSIGN) ? 0 : (F <= 8 ? 32 : 16);
+  }
+  const int k_limit = cpe::all_pairs_limit(F, p);
   // A caller whose max_instances already is within the all-pairs range needs no second kernel: no image can have
-  // more peaks than that (the list is truncated to max_instances), so the chain is one launch shorter.
-  if (p->max_instances <= k_limit)
+  // more peaks than that (the list is truncated to max_instances), so the chain is shorter.
+  if (p->max_instances <= k_limit) {
+    if (ev_lists) CPE_CUDA(cudaEventRecord(ev_lists, st));
     return launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
                                   votes_to_zero, cells, 0x7fffffff);
-  int rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
-                                  cells, k_limit);
-  if (rc) return rc;
-  const T* e = static_cast<const T*>(emb);
-  const bool want2 = best != nullptr;
-  const int k_min = k_limit + 1;
-  // CPE_ASSIGN_PATH=mma in the environment keeps the mma.sync kernel everywhere (comparisons)
-  static const char* path = getenv("CPE_ASSIGN_PATH");
-  const bool aligned = (uintptr_t)e % 16 == 0 && HW % 8 == 0;
-  if (aligned && !(path && strcmp(path, "mma") == 0)) {
-    if (F <= 8)
-      return want2 ? launch_assign_filter_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                         counters, status, votes_to_zero, cells, k_min, acc)
-                   : launch_assign_filter_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                          counters, status, votes_to_zero, cells, k_min, acc);
-    return want2 ? launch_assign_filter_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                       counters, status, votes_to_zero, cells, k_min, acc)
-                 : launch_assign_filter_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                        counters, status, votes_to_zero, cells, k_min, acc);
   }
-  if (F <= 8) {
-    return want2 ? launch_assign_mma_t<T, 16, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
-                                                    status, votes_to_zero, cells, k_min)
-                 : launch_assign_mma_t<T, 16, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                     counters, status, votes_to_zero, cells, k_min);
+  int rc = CPE_OK;
+  if (pr) {
+    rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->nbr);
+    if (rc) return rc;
   }
-  return want2 ? launch_assign_mma_t<T, 32, true>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
-                                                  status, votes_to_zero, cells, k_min)
-               : launch_assign_mma_t<T, 32, false>(st, e, fg, B, HW, F, p, peak_emb, count, labels, best, second,
-                                                   counters, status, votes_to_zero, cells, k_min);
+  if (ev_lists) CPE_CUDA(cudaEventRecord(ev_lists, st));
+  if (pr) {
+    rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref2, pr->cand2, pr->nbr, pr->cell_peak, pr->pix_cell,
+                                       cells, count, labels, best, second, pr->near_state, k_limit + 1);
+    if (rc) return rc;
+  }
+  if (k_limit > 0) {
+    rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
+                                cells, k_limit);
+    if (rc) return rc;
+  }
+  return cpe::host::launch_assign_filtered(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                           status, votes_to_zero, cells, k_limit + 1, acc, pr ? pr->near_state : nullptr);
 }
 
-// CPE_DEBUG_SYNC=1 in the environment: wait after every stage and name the stage whose kernel failed
-// (never inside stream capture).
+// Debug builds only (-DCPE_DEBUG_SYNC): wait after every stage and name the stage whose kernel failed (never
+// inside stream capture).  The product build compiles this to nothing.
 int debug_stage_check(cudaStream_t st, const char* stage) {
-  static const bool on = getenv("CPE_DEBUG_SYNC") != nullptr;
-  if (!on) return CPE_OK;
+#ifndef CPE_DEBUG_SYNC
+  (void)st;
+  (void)stage;
+  return CPE_OK;
+#else
   cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone) return CPE_OK;
   cudaError_t e = cudaStreamSynchronize(st);
@@ -312,6 +170,7 @@ int debug_stage_check(cudaStream_t st, const char* stage) {
     return cuda_fail(e);
   }
   return CPE_OK;
+#endif
 }
 
 // The chain.  `ev`, when given, holds CPE_STAGE_N + 1 events recorded around the stages.
@@ -346,14 +205,25 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (keep_votes) CPE_CUDA(cudaMemsetAsync(ws + L.votes, 0, L.votes_end - L.votes, st));
   // The per-bin sums of the refinement: a small map, which one CTA of the peak kernel handles per image, is cleared
   // by that CTA after its last read; otherwise (or when the intermediates are to stay readable) they are cleared here.
-  long long* sums = (p->flags & CPE_FLAG_REFINE) ? reinterpret_cast<long long*>(ws + L.sums) : nullptr;
+  const bool refine = (p->flags & CPE_FLAG_REFINE) != 0;
+  long long* sums = (refine || L.prune) ? reinterpret_cast<long long*>(ws + L.sums) : nullptr;
+  PruneArgs pr;
+  if (L.prune) {
+    pr.ref_emb = reinterpret_cast<const float*>(ws + L.ref_emb);
+    pr.ref2 = reinterpret_cast<float*>(ws + L.ref2);
+    pr.cand2 = reinterpret_cast<float*>(ws + L.cand2);
+    pr.nbr = reinterpret_cast<uint32_t*>(ws + L.nbr);
+    pr.cell_peak = reinterpret_cast<const int32_t*>(ws + L.cell_peak);
+    pr.pix_cell = reinterpret_cast<const uint32_t*>(ws + L.pix_cell);
+    pr.near_state = reinterpret_cast<uint32_t*>(ws + L.near_state);
+  }
   const bool one_peak_cta = L.words <= cpe::kPeakStageWords;
   const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes;
   if (sums && !sums_cleared_by_peaks) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
-  rc = p->dtype == CPE_F32 ? launch_decode_vote<float>(st, emb, fg, B, HW, F, p, votes, acc, sums)
-                           : launch_decode_vote<__half>(st, emb, fg, B, HW, F, p, votes, acc, sums);
+  rc = cpe::host::launch_decode_vote(st, emb, fg, B, HW, F, p, votes, acc, sums,
+                                     L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
@@ -365,21 +235,23 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     dim3 grid((unsigned)ctas, (unsigned)B);
     // one CTA per image: it works on a copy of the vote map in shared memory (at most 32 KB)
     const size_t map_smem = one_peak_cta ? 4 * (size_t)L.cells : 0;
-    CPE_CUDA(launch_dependent(cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes, p->bins_w, p->bins_h, L.words,
+    CPE_CUDA(launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes, p->bins_w, p->bins_h, L.words,
                               (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W, pal_w, pal_h, peak_cell,
                               peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums,
-                              sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0));
+                              sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0, refine ? 1 : 0,
+                              L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
+                              L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr, pr.near_state));
     CPE_CUDA(cudaGetLastError());
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
-  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_COMPACT], st));
-
-  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_ASSIGN], st));
+  if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_LISTS], st));
   uint32_t* votes_to_zero = keep_votes ? nullptr : votes;
+  const PruneArgs* prp = L.prune ? &pr : nullptr;
+  cudaEvent_t ev_lists = ev ? ev[CPE_STAGE_ASSIGN] : nullptr;
   rc = p->dtype == CPE_F32 ? launch_assign<float>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best, second,
-                                                  counters, status, votes_to_zero, L.cells, acc)
+                                                  counters, status, votes_to_zero, L.cells, acc, prp, ev_lists)
                            : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best,
-                                                   second, counters, status, votes_to_zero, L.cells, acc);
+                                                   second, counters, status, votes_to_zero, L.cells, acc, prp, ev_lists);
   if (rc) return rc;
   if ((rc = debug_stage_check(st, "assign"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
@@ -487,6 +359,11 @@ int cpe_get_intermediate(const cpe_params* params, int which, int B, int H, int 
       if (!(params->flags & CPE_FLAG_REFINE) || !(params->flags & CPE_FLAG_KEEP_VOTES)) return CPE_ERR_WHICH;
       off = L.sums;
       sz = 16 * (size_t)L.cells * B;
+      break;
+    case CPE_INT_PRUNE_STATE:
+      if (!L.prune) return CPE_ERR_WHICH;
+      off = L.near_state;
+      sz = 4 * (size_t)cpe::kNearStride * B;
       break;
     default: return CPE_ERR_WHICH;
   }
@@ -735,6 +612,7 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   cpe_params p = *params;
   if (p.flags & CPE_FLAG_WRITE_SCORES) return CPE_ERR_STATIC_LIMIT;
   p.flags |= CPE_FLAG_KEEP_VOTES;   // the vote map is cleared at the start of every call instead of at the end
+  p.flags |= CPE_FLAG_NO_PRUNE;     // the pruned assignment keeps per-pixel scratch, which the built-in array has no room for
   p.workspace = nullptr;
   p.workspace_bytes = 0;
   const cpe::Layout L = cpe::make_layout(B, H, W, F, &p);
@@ -786,30 +664,6 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
 }
 
-namespace {
-template <typename T, int KA>
-int launch_soft_votes_t(cudaStream_t st, const T* e, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                        const float* pal_w, const float* pal_h, float* hist, uint32_t* status) {
-  const int smem = cpe::sv_smem_layout(KA).total;
-  auto kern = cpe::soft_vote_kernel<T, KA>;
-  static bool configured = false;   // per instantiation; the attribute is sticky for the process
-  if (!configured) {
-    CPE_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    configured = true;
-  }
-  // one CTA per SM (it holds all of the SM's tensor memory): the SMs are shared among the images and the
-  // 128 x 128 blocks of bins, the CTAs of one block split the pixels
-  const int n_blocks = ((p->bins_w + cpe::kSvBins - 1) / cpe::kSvBins) * ((p->bins_h + cpe::kSvBins - 1) / cpe::kSvBins);
-  const int n_spans = (HW + cpe::kTcSpan - 1) / cpe::kTcSpan;
-  const int split = std::max(1, std::min(n_spans, sm_count() / std::max(1, n_blocks * B)));
-  dim3 grid((unsigned)split, (unsigned)n_blocks, (unsigned)B);
-  const int vec_mask = fg && ((uintptr_t)fg % 8 == 0) ? 1 : 0;
-  kern<<<grid, cpe::kSvThreads, smem, st>>>(e, fg, HW, F, p->bins_w, p->bins_h, pal_w, pal_h, vec_mask, hist, status);
-  CPE_CUDA(cudaGetLastError());
-  return CPE_OK;
-}
-}  // namespace
-
 extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
                    const cpe_params* params, float* out_hist) {
   if (!emb || !out_hist) return CPE_ERR_NULL;
@@ -824,15 +678,7 @@ extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_
   const float* pal_h = reinterpret_cast<const float*>(ws + L.pal_h);
   uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.status);
   CPE_CUDA(cudaMemsetAsync(out_hist, 0, sizeof(float) * (size_t)B * params->bins_w * params->bins_h, st));
-  if (params->dtype == CPE_F32)
-    return F <= 8 ? launch_soft_votes_t<float, 16>(st, static_cast<const float*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
-                                                   pal_h, out_hist, status)
-                  : launch_soft_votes_t<float, 32>(st, static_cast<const float*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
-                                                   pal_h, out_hist, status);
-  return F <= 8 ? launch_soft_votes_t<__half, 16>(st, static_cast<const __half*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
-                                                  pal_h, out_hist, status)
-                : launch_soft_votes_t<__half, 32>(st, static_cast<const __half*>(emb), fg_mask, B, (int)HW, F, params, pal_w,
-                                                  pal_h, out_hist, status);
+  return cpe::host::launch_soft_votes(st, emb, fg_mask, B, (int)HW, F, params, pal_w, pal_h, out_hist, status);
 }
 
 extern "C" int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, int B, int H, int W, int n_planes,

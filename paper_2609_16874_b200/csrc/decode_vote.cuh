@@ -44,6 +44,11 @@ __device__ __forceinline__ void vote_cache_add(uint32_t* keys, uint32_t* cnts, u
 // reductions).  Called by all 32 lanes; cell < 0 = this lane has no vote.
 constexpr float kRefineScale = 16777216.0f;  // 2^24
 
+// What a voting kernel records besides the vote map (template parameter MODE, a bit set):
+constexpr int kVoteSums = 1;    // the per-bin fixed-point sums of the estimates
+constexpr int kVoteCells = 2;   // every participating pixel's bin (uint32 [B][H*W]; 0xffffffff: it did not vote), which the
+                                // pruned assignment looks its candidate list up with
+
 __device__ __forceinline__ void vote_sums_add(long long* __restrict__ sums_img, int cell, float px, float py,
                                               bool one_bin, uint32_t voters) {
   const int lane = threadIdx.x & 31;
@@ -122,11 +127,13 @@ __device__ __forceinline__ int compact_span(const uint8_t* __restrict__ fg_img, 
 }
 
 // Scalar-load variant: any F, any alignment, any H*W.  FT > 0 fixes F at compile time.
-template <typename T, int FT, bool REFINE>
+template <typename T, int FT, int MODE>
 __global__ void __launch_bounds__(kVoteThreads)
 decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
                    int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
-                   uint32_t* __restrict__ acc, long long* __restrict__ sums) {
+                   uint32_t* __restrict__ acc, long long* __restrict__ sums, uint32_t* __restrict__ pix_cell) {
+  constexpr bool REFINE = (MODE & kVoteSums) != 0;
+  constexpr bool CELLS = (MODE & kVoteCells) != 0;
   grid_dependency_sync();
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
@@ -209,6 +216,8 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
         } else {
           ++nonfinite;
         }
+        if constexpr (CELLS)
+          pix_cell[(size_t)b * plane + (size_t)(src[q] - e)] = (uint32_t)cell;   // 0xffffffff: no vote
       }
       // warp-aggregated insertion; fast path: every voting lane of the warp names the same bin
       const uint32_t voters = __ballot_sync(0xffffffffu, cell >= 0);
@@ -258,11 +267,13 @@ constexpr int kVecGroupsMax = 256;   // groups per CTA: 256, 128 or 64 (template
                                      // and want many short CTAs, large ones want fewer fixed costs)
 constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight together (2 loads each)
 
-template <typename T, int FT, bool REFINE, int GROUPS>
+template <typename T, int FT, int MODE, int GROUPS>
 __global__ void __launch_bounds__(kVoteThreads, 3)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
                        int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
-                       long long* __restrict__ sums) {
+                       long long* __restrict__ sums, uint32_t* __restrict__ pix_cell) {
+  constexpr bool REFINE = (MODE & kVoteSums) != 0;
+  constexpr bool CELLS = (MODE & kVoteCells) != 0;
   grid_dependency_sync();
   constexpr int VEC = Elem<T>::kVec;
   constexpr int F = FT;
@@ -390,6 +401,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
     float other[VEC];
 #pragma unroll
     for (int j = 0; j < VEC; ++j) other[j] = __shfl_xor_sync(0xffffffffu, p[j], 1);
+    uint32_t my_cells[VEC / 2];
 #pragma unroll
     for (int jj = 0; jj < VEC / 2; ++jj) {
       const int j = axis * (VEC / 2) + jj;       // axis-0 lane finishes the first half, axis-1 lane the second
@@ -408,6 +420,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
           ++nonfinite;
         }
       }
+      my_cells[jj] = (uint32_t)cell;
       const uint32_t voters = __ballot_sync(0xffffffffu, cell >= 0);
       if (voters) {
         const int leader = __ffs(voters) - 1;
@@ -421,6 +434,16 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
           if (cell >= 0 && lane == __ffs(same) - 1)
             vote_cache_add(s_keys, s_cnts, (uint32_t)cell, (uint32_t)__popc(same), votes_img);
         }
+      }
+    }
+    if constexpr (CELLS) {
+      // this lane's half of the group: VEC/2 consecutive pixels, one 16-byte (fp16) or 8-byte (fp32) store
+      if (have) {
+        uint32_t* dst = pix_cell + (size_t)b * plane + (size_t)span0 + (size_t)(ent & 0xffu) * VEC + (size_t)axis * (VEC / 2);
+        if constexpr (VEC == 8)
+          *reinterpret_cast<uint4*>(dst) = make_uint4(my_cells[0], my_cells[1], my_cells[2], my_cells[3]);
+        else
+          *reinterpret_cast<uint2*>(dst) = make_uint2(my_cells[0], my_cells[1]);
       }
     }
   }

@@ -28,6 +28,11 @@ constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared me
 // and rounded once, the way the palette rows are made.  `zero_sums` (only with one CTA per image): the sums are cleared
 // at the end, so that the decode needs no clearing pass for them.
 //
+// `refine_out` = 0 with `sums` (the pruned assignment of the unrefined decode): the peaks stay on their bin positions
+// and keep their palette rows, and gamma(mean) goes to `ref_emb` instead, where the assignment uses it as the point
+// its distance bounds are taken around.  `cell_peak` (with the pruned assignment): bin -> index of the peak whose 3x3
+// window holds it, -1 where there is none; `near_state`: that kernel's per-image words, zeroed here.
+//
 // `staged` (only with one CTA per image; needs 4 * bins_w * bins_h bytes of dynamic shared memory): the CTA first
 // copies the whole vote map into shared memory with independent loads -- one round trip to L2 instead of one or two
 // per 32-bin word and warp iteration -- and keeps the bitmap and the head of the peak list there as well, so that
@@ -38,7 +43,8 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
              uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
-             long long* __restrict__ sums, int zero_sums, int staged) {
+             long long* __restrict__ sums, int zero_sums, int staged, int refine_out,
+             float* __restrict__ ref_emb, int32_t* __restrict__ cell_peak, uint32_t* __restrict__ near_state) {
   extern __shared__ uint32_t s_map[];                 // [cells] when staged
   __shared__ uint32_t s_bm[kPeakStageWords];
   __shared__ int s_pc[kPeakListStage];
@@ -85,6 +91,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
         }
       }
     }
+    if (cell_peak && lin < cells) cell_peak[(size_t)b * cells + lin] = -1;
     const uint32_t word = __ballot_sync(0xffffffffu, peak);
     if (lane == 0) {
       bm[warp] = word;
@@ -172,6 +179,8 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     cnt[CPE_CNT_FILTER_PAIRS] = 0u;
     cnt[CPE_CNT_RESCORED] = 0u;
     cnt[CPE_CNT_FULL_SCORED] = 0u;
+    if (near_state)
+      for (int i = 0; i < kNearStride; ++i) near_state[b * kNearStride + i] = 0u;
     status[b] = (nonfinite ? (uint32_t)CPE_STATUS_NONFINITE : 0u) |
                 (total > K_max ? (uint32_t)CPE_STATUS_PEAK_OVERFLOW : 0u);
   }
@@ -179,7 +188,26 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
 
   const int D = 4 * F;
   float* pe = peak_emb + (size_t)b * K_max * D;
+  if (cell_peak) {
+    // every bin of a peak's 3x3 window names that peak (two peaks are never neighbours, so a peak's own bin is in no
+    // other window; a bin between two peaks gets either)
+    int32_t* cp = cell_peak + (size_t)b * cells;
+    for (int k = tid; k < count; k += kPeakThreads) {
+      const int lin = cell_of(pc, k);
+      const int cy = lin / bins_w, cx = lin - cy * bins_w;
+#pragma unroll
+      for (int dy = -1; dy <= 1; ++dy) {
+#pragma unroll
+        for (int dx = -1; dx <= 1; ++dx) {
+          const int ny = cy + dy, nx = cx + dx;
+          if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+          cp[ny * bins_w + nx] = k;
+        }
+      }
+    }
+  }
   if (sums) {
+    float* gm = refine_out ? pe : ref_emb + (size_t)b * K_max * D;   // where gamma(mean) goes
     __shared__ double s_mean[2 * kRefineChunk];
     long long* S = sums + (size_t)b * cells * 2;
     for (int k0 = 0; k0 < count; k0 += kRefineChunk) {
@@ -203,8 +231,9 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
         const double m = __ddiv_rn((double)s, __dmul_rn((double)n, 16777216.0));
         s_mean[i] = m;
         // pixel centres sit at x = -1 + (2 col + 1)/W
-        out_centroids[((size_t)b * K_max + k) * 2 + axis] =
-            (float)__dmul_rn(__dadd_rn(__dmul_rn(__dadd_rn(m, 1.0), (double)(axis ? H : W)), -1.0), 0.5);
+        if (refine_out)
+          out_centroids[((size_t)b * K_max + k) * 2 + axis] =
+              (float)__dmul_rn(__dadd_rn(__dmul_rn(__dadd_rn(m, 1.0), (double)(axis ? H : W)), -1.0), 0.5);
       }
       __syncthreads();
       for (int i = tid; i < 2 * F * nk; i += kPeakThreads) {   // (peak, axis, harmonic): sin and cos of pi 2^l mean
@@ -212,7 +241,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
         const int axis = r / F, l = r - axis * F;
         double sn, cs;
         sincospi(scalbn(s_mean[2 * kk + axis], l), &sn, &cs);
-        float* o = pe + (size_t)(k0 + kk) * D + axis * 2 * F + 2 * l;
+        float* o = gm + (size_t)(k0 + kk) * D + axis * 2 * F + 2 * l;
         o[0] = (float)sn;
         o[1] = (float)cs;
       }
@@ -221,7 +250,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     // small maps (this CTA does the whole image): the sums have no reader left and are left zero for the next decode
     if (zero_sums)
       for (int i = tid; i < 2 * cells; i += kPeakThreads) S[i] = 0;
-    return;
+    if (refine_out) return;
   }
   for (int i = tid; i < count * D; i += kPeakThreads) {
     const int k = i / D, c = i - k * D;

@@ -9,13 +9,14 @@ REL = 1e-4         # relative tolerance of float scores and centroids
 
 
 def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, scores=True, mode="direct",
-            exact_assign=False, keep_votes=True, filter_assign=False):
+            exact_assign=False, keep_votes=True, filter_assign=False, refine=False, flags=0):
     import torch
     B, D, H, W = emb.shape
     F = D // 4
     dtype = "f32" if emb.dtype == np.float32 else "f16"
     dec = cb.Decoder(B, H, W, F, dtype, bins_w, bins_h, T_v, float(tau), K_max, levels, write_scores=scores,
-                     exact_assign=exact_assign, keep_votes=keep_votes, filter_assign=filter_assign)
+                     exact_assign=exact_assign, keep_votes=keep_votes, filter_assign=filter_assign, refine=refine,
+                     flags=flags)
     d_emb = torch.from_numpy(emb).cuda()
     d_fg = None if fg is None else torch.from_numpy(np.ascontiguousarray(fg, np.uint8)).cuda()
     if mode == "direct":
@@ -42,6 +43,9 @@ def run_gpu(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, levels=0, sc
         "status": int(np.bitwise_or.reduce(dec.intermediate(cb.CPE_INT_STATUS).cpu().numpy())),
         "counters": dec.intermediate(cb.CPE_INT_COUNTERS).cpu().numpy().astype(np.int64),
     }
+    rc, _, _ = cb.cpe_get_intermediate(dec.params, cb.CPE_INT_PRUNE_STATE, B, H, W, F)
+    out["prune_state"] = (dec.intermediate(cb.CPE_INT_PRUNE_STATE).cpu().numpy().astype(np.int64)
+                          if rc == cb.CPE_OK else None)
     if scores:
         out["best"] = dec.intermediate(cb.CPE_INT_BEST_SCORE).cpu().numpy()
         out["second"] = dec.intermediate(cb.CPE_INT_SECOND_SCORE).cpu().numpy()

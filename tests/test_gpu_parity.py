@@ -303,37 +303,27 @@ def test_full_size_configs(name):
 
 
 def test_tensor_memory_path_with_several_rounds_of_peaks():
-    """The tcgen05 assignment serves up to 64 peaks by default; with CPE_ASSIGN_PATH=tc (read once per process, hence
-    the child process) it takes every image whose peaks fit its shared-memory operand, in rounds of 64.  Labels and
-    scores must be those of the all-pairs kernel, bit for bit."""
-    import os
-    import subprocess
-    import sys
-    code = r"""
-import sys, numpy as np
-sys.path.insert(0, sys.argv[1]); sys.path.insert(0, sys.argv[1] + "/tests")
-from paper_2609_16874_b200 import workloads as wl
-from gpu_util import run_gpu
-for name, over in (("c4", dict(B=2, H=320, W=384, K=100)), ("c5", dict(H=512, W=512, K=200, bins_w=256, bins_h=256))):
-    cfg = wl.scaled(wl.CONFIGS[name], **over)
-    fr = wl.make_frame(cfg, 0)
-    for scores in (False, True):
-        a = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=scores, keep_votes=False)
-        b = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=scores, keep_votes=False,
-                    exact_assign=True)
-        assert a["count"].min() > 64, a["count"]
-        assert a["status"] == 0, hex(a["status"])
-        assert np.array_equal(a["labels"], b["labels"])
-        assert a["counters"][:, 5].min() > 0          # the filter ran (pairs were counted)
-        if scores:
-            assert np.array_equal(a["best"].view(np.uint32), b["best"].view(np.uint32))
-            assert np.array_equal(a["second"].view(np.uint32), b["second"].view(np.uint32))
-print("ok")
-"""
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    env = dict(os.environ, CPE_ASSIGN_PATH="tc")
-    out = subprocess.run([sys.executable, "-c", code, root], env=env, capture_output=True, text=True, timeout=600)
-    assert out.returncode == 0 and "ok" in out.stdout, out.stdout[-2000:] + out.stderr[-4000:]
+    """The tcgen05 assignment serves up to 128 peaks by default; with CPE_FLAG_TC_ALL_ROUNDS it takes every image whose
+    peaks fit its shared-memory operand, in rounds of 64, and with CPE_FLAG_TC_ONE_STAGE only those with at most 64.
+    Labels and scores must be those of the all-pairs kernel, bit for bit.  (CPE_FLAG_NO_PRUNE: these images would
+    otherwise go to the pruned assignment first.)"""
+    for name, over in (("c4", dict(B=2, H=320, W=384, K=100)), ("c5", dict(H=512, W=512, K=200, bins_w=256, bins_h=256))):
+        cfg = wl.scaled(wl.CONFIGS[name], **over)
+        fr = wl.make_frame(cfg, 0)
+        for scores in (False, True):
+            b = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=scores,
+                        keep_votes=False, exact_assign=True)
+            for path in (cb.CPE_FLAG_TC_ALL_ROUNDS, cb.CPE_FLAG_TC_ONE_STAGE, cb.CPE_FLAG_MMA_ASSIGN, 0):
+                a = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, scores=scores,
+                            keep_votes=False, flags=path | cb.CPE_FLAG_NO_PRUNE)
+                assert a["count"].min() > 64, a["count"]
+                assert a["status"] == 0, hex(a["status"])
+                assert a["prune_state"] is None
+                assert np.array_equal(a["labels"], b["labels"]), path
+                assert a["counters"][:, cb.CPE_CNT_FILTER_PAIRS].min() > 0          # the filter ran (pairs were counted)
+                if scores:
+                    assert np.array_equal(a["best"].view(np.uint32), b["best"].view(np.uint32))
+                    assert np.array_equal(a["second"].view(np.uint32), b["second"].view(np.uint32))
 
 
 @pytest.mark.parametrize("name,over", [("c2", dict(H=384, W=384, K=90, bins_w=96, bins_h=96)),              # fp32, F = 8

@@ -125,8 +125,9 @@ def test_refined_centroids_are_closer_to_the_truth_than_bin_centres():
 
 
 def test_refine_intermediate_needs_the_flag_and_workspace_grows_by_the_sums():
-    p0 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, 0)
-    p1 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, cb.CPE_FLAG_REFINE)
+    # (without the pruned assignment, which keeps the sums for its own use in either mode)
+    p0 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, cb.CPE_FLAG_NO_PRUNE)
+    p1 = cb.make_params(cb.CPE_F32, 64, 48, 0, 8, float("inf"), 128, cb.CPE_FLAG_REFINE | cb.CPE_FLAG_NO_PRUNE)
     n0, n1 = cb.cpe_workspace_size(2, 96, 128, 4, p0), cb.cpe_workspace_size(2, 96, 128, 4, p1)
     assert n1 - n0 == 16 * 64 * 48 * 2
     import torch
