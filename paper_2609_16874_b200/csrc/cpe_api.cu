@@ -145,11 +145,10 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
                                        cells, count, labels, best, second, pr->near_state, k_limit + 1);
     if (rc) return rc;
   }
-  if (k_limit > 0) {
-    rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
-                                cells, k_limit);
-    if (rc) return rc;
-  }
+  // (also with a limit of 0: an image without any peak still gets its all-zero label map from this kernel)
+  rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
+                              cells, k_limit);
+  if (rc) return rc;
   return cpe::host::launch_assign_filtered(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
                                            status, votes_to_zero, cells, k_limit + 1, acc, pr ? pr->near_state : nullptr);
 }

@@ -339,8 +339,8 @@ def test_between_65_and_128_peaks_both_tensor_memory_stages_serve_one_tile(name,
 
 
 def test_small_max_instances_takes_the_three_kernel_chain():
-    """With max_instances inside the all-pairs range no image can need the filtered kernel, so it is not enqueued:
-    the captured graph has three kernel nodes instead of four, results are the oracle's, and replays repeat them
+    """With max_instances inside the all-pairs range no image can need the pruned or the filtered assignment, so neither
+    is enqueued: the captured graph has three kernel nodes, results are the oracle's, and replays repeat them
     (the all-pairs kernel then is the one that leaves the vote map zero for the next decode)."""
     import torch
     cfg = wl.scaled(wl.CONFIGS["c2"], H=192, W=256, K=12, bins_w=48, bins_h=32)
@@ -366,4 +366,4 @@ def test_small_max_instances_takes_the_three_kernel_chain():
                 near_tie = (ora["second"] - ora["best"]) < 1e-5
             assert ((lab == ora["labels"]) | near_tie).all()
         dec.close()
-    assert nodes[32] == nodes[33] - 1, nodes
+    assert nodes[32] == 3 and nodes[33] > nodes[32], nodes

@@ -46,8 +46,10 @@ def check_pruned(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, refine=
             out = gpu
         # the tau-rejected counter is exact whichever kernel finished the image
         assert np.array_equal(gpu["counters"][:, cb.CPE_CNT_TAU_REJECTED], exact["counters"][:, cb.CPE_CNT_TAU_REJECTED])
+        # (checked without scores: when the runner-up's distance is wanted as well, a walk can only end at
+        # G > second-best + t, which heavy noise puts beyond every candidate)
         handed = gpu["prune_state"][:, 2] != 0
-        if expect_handed_on is not None:
+        if expect_handed_on is not None and not scores:
             assert handed.tolist() == list(expect_handed_on), gpu["prune_state"].tolist()
     return out, ora
 
@@ -83,9 +85,10 @@ def test_refined_candidates_leave_about_one_candidate_per_pixel():
     gpu, ora = check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=True, flags=0,
                             expect_handed_on=[False, False])
     assert ora["count"].min() > 64                                   # more peaks than a list has entries
-    pairs = gpu["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum()        # scores wanted: the runner-up is scored as well
+    # scores wanted: the walk goes on until the runner-up is settled too, i.e. up to G = (second-best distance) + t
+    pairs = gpu["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum()
     voting = gpu["counters"][:, cb.CPE_CNT_VOTING].sum()
-    assert pairs <= 4 * voting, (pairs, voting)
+    assert pairs <= 12 * voting, (pairs, voting)
     fast = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, keep_votes=False,
                    refine=True)
     pairs = fast["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum()
