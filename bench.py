@@ -131,7 +131,7 @@ def algorithmic_bytes(cfg, fg_pixels: int):
         "clear": 4 * cells,
         "decode_vote": fg_pixels * D * esz + P,
         "peaks": 4 * cells + cells // 8,
-        "compact": cells // 8,
+        "lists": 0,
         "assign": fg_pixels * D * esz + P + 4 * P,
     }
 
@@ -229,7 +229,7 @@ def run_ours(args, cfg):
         flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
 
     dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max,
-                     device=dev)
+                     device=dev, refine=args.refine, flags=args.flags)
     stream = torch.cuda.Stream(device=dev)
     sampler = ClockSampler(dev.index)
     sampler.start()
@@ -294,8 +294,10 @@ def run_ours(args, cfg):
     # ---- end to end through the host-buffer entry point (rank-local wall clock, max over ranks)
     if args.quick:
         cnt = dec.intermediate(cb.CPE_INT_COUNTERS).cpu().numpy().sum(0).tolist()
-        print(json.dumps({"quick": True, "name": cfg.name, "p50_ms": p50, "value": value, "stage_ms": stage_ms,
-                          "counters": cnt}))
+        st = dec.intermediate(cb.CPE_INT_PRUNE_STATE).cpu().numpy().tolist() if dec.params.flags & 0 == 0 and cb.cpe_get_intermediate(dec.params, cb.CPE_INT_PRUNE_STATE, cfg.B, cfg.H, cfg.W, cfg.F)[0] == 0 else None
+        print(json.dumps({"quick": True, "name": cfg.name, "refine": args.refine, "flags": args.flags, "p50_ms": p50,
+                          "value": value, "stage_ms": stage_ms, "counters": cnt, "prune_state": st,
+                          "kernel_nodes": kernel_nodes}))
         dec.close()
         dist_util.shutdown()
         return
@@ -640,6 +642,8 @@ def main():
     ap.add_argument("--only-default", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--quick", action="store_true",
                     help="profiling runs: no clock pre-heat, no host-buffer leg, no CPU baseline (few launches)")
+    ap.add_argument("--refine", action="store_true", help="sub-cell refined centroids (CPE_FLAG_REFINE)")
+    ap.add_argument("--flags", type=int, default=0, help="extra cpe_params.flags bits (A/B runs)")
     ap.add_argument("--soft-votes", action="store_true",
                     help="profiling runs: only the second vote mode (cpe_soft_votes) on the chosen workload")
     args = ap.parse_args()

@@ -75,6 +75,11 @@ enum {
   CPE_FLAG_NO_PRUNE = 512u,       /* do not prune the candidates of Eq. 7 (see cpe_decode): every image with more peaks
                                      than the all-pairs range goes to the tensor-core filtered kernels; same results  */
   CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment for every image, however few peaks it has; same results    */
+  CPE_FLAG_PRUNE_WALK_ONLY = 2048u, /* pruned assignment: the one-thread-per-pixel kernel also where the streaming kernel
+                                       would run (tests, comparisons; same results)                                   */
+  CPE_FLAG_TEST_STALL = 4096u,    /* tests of the time-out path only: the pruned assignment's copy pipeline withholds
+                                     its first tile and waits briefly, so that a bounded wait runs out, the kernel
+                                     winds down and CPE_STATUS_TIMEOUT is set (the label map is then incomplete)      */
   CPE_FLAG_REFINE = 16u       /* sub-cell refined centroids (an extension: the paper's candidates of Eq. 7 are the
                                  bin positions of Eq. 9, up to half a bin off the voted centroid).  Next to its
                                  count every bin keeps the sum of the estimates that fell into it, as integers
@@ -92,8 +97,11 @@ enum {
 enum {
   CPE_STATUS_PEAK_OVERFLOW = 1u, /* an image had more local maxima than max_instances            */
   CPE_STATUS_NONFINITE = 2u,     /* at least one participating pixel had a non-finite channel    */
-  CPE_STATUS_INTERNAL = 4u       /* an index self-check failed (site code in bits 8..15); the access was
+  CPE_STATUS_INTERNAL = 4u,      /* an index self-check failed (site code in bits 8..15); the access was
                                     skipped.  Never set by a correct build: please report it.      */
+  CPE_STATUS_TIMEOUT = 8u        /* a bounded device-side wait (on an mbarrier of a copy or tensor-core pipeline)
+                                    ran out; the kernel wound down and returned, the image's outputs are
+                                    incomplete.  Never set by a correct build on a healthy GPU.    */
 };
 
 /* per-image counters, uint32 [B][CPE_CNT_N] */

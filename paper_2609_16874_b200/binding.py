@@ -34,7 +34,9 @@ CPE_FLAG_TC_ONE_STAGE = 128
 CPE_FLAG_MMA_ASSIGN = 256
 CPE_FLAG_NO_PRUNE = 512
 CPE_FLAG_PRUNE_ALL = 1024
-CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL = 1, 2, 4
+CPE_FLAG_PRUNE_WALK_ONLY = 2048
+CPE_FLAG_TEST_STALL = 4096
+CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL, CPE_STATUS_TIMEOUT = 1, 2, 4, 8
 CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
 CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8
 (CPE_INT_VOTES, CPE_INT_PEAK_CELLS, CPE_INT_PEAK_VOTES, CPE_INT_PEAK_EMB, CPE_INT_PALETTE_W, CPE_INT_PALETTE_H,

@@ -14,6 +14,13 @@
 // separates: a vote map too coarse for the harmonics, heavy noise), the image is handed to the tensor-core filtered
 // kernel launched after this one (`near_state[kNearGiveUp]`), which then redoes it as a whole; both kernels compute
 // the same bits, so pixels already written are simply written again.
+//
+// Three kernels.  assign_near_stream_kernel (16-byte aligned planes, no scores wanted) streams the embedding the way
+// the voting kernel does -- a thread takes (8-pixel group, axis), 128-bit plane loads, background never fetched --
+// and only certifies, from cheap upper bounds of t and of the distance to the first candidate of k0's list, that the
+// second list entry is already out of reach (nearly every pixel when the candidates sit on the voted centroids):
+// the label is then final.  The other pixels go to a queue in global memory, which assign_near_walk_kernel decides
+// exactly, one thread per pixel.  assign_near_kernel is that walk for every pixel: any alignment, and scores.
 #pragma once
 
 #include "assign.cuh"
@@ -24,6 +31,123 @@ namespace cpe {
 
 constexpr int kNearThreads = 256;
 constexpr float kNearSlack = 1.00002f;
+
+// The walk of one pixel, given its 4F values as (x channel c, y channel c) pairs.
+template <int D, bool WANT2>
+__device__ __forceinline__ void near_walk(const float2 (&e2)[D / 2], int k0, int K, bool same_rows,
+                                          const float* __restrict__ ref_img, const float* __restrict__ cand_img,
+                                          const uint32_t* __restrict__ nbr_img, float& d1, float& d2, int& k1, bool& hard,
+                                          uint32_t& scored) {
+  const float inf = __int_as_float(0x7f800000);
+  const float t = score_direct<D>(e2, reinterpret_cast<const float2*>(ref_img + (size_t)k0 * D), inf);
+  const uint32_t* list = nbr_img + (size_t)k0 * kNbrCap;
+  float bound2 = inf;
+  int j = 0;
+  for (; j < kNbrCap; ++j) {
+    const uint32_t ent = __ldg(list + j);
+    if (ent == kNbrEnd) break;                                   // every candidate of the image has been seen
+    const float G = (float)(ent >> 12) * (1.0f / 65536.0f);
+    const float U = WANT2 ? d2 : d1;
+    if (G > (U + t) * kNearSlack) break;                         // this one and all later ones: d >= G - t > U
+    const int k = (int)(ent & 0xfffu);
+    const float d = (same_rows && k == k0)
+                        ? t
+                        : score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
+    ++scored;
+    if (d < d1 || (d == d1 && k < k1)) { d2 = d1; d1 = d; k1 = k; }   // the lowest k keeps an exact tie
+    else if (d < d2) { d2 = d; }
+    const float bound = WANT2 ? d2 : d1;
+    bound2 = bound * bound * (1.0f + 1e-6f);
+  }
+  hard = (j == kNbrCap) && K > kNbrCap;                          // the list ran out before the bound closed it
+}
+
+// Every peak, in ascending k (a hard pixel).
+template <int D, bool WANT2>
+__device__ __forceinline__ void near_full_scan(const float2 (&e2)[D / 2], int K, const float* __restrict__ cand_img,
+                                               float& d1, float& d2, int& k1) {
+  const float inf = __int_as_float(0x7f800000);
+  d1 = d2 = inf;
+  k1 = -1;
+  float bound2 = inf;
+  for (int k = 0; k < K; ++k) {
+    const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
+    if (d < d1) { d2 = d1; d1 = d; k1 = k; }
+    else if (d < d2) { d2 = d; }
+    const float bound = WANT2 ? d2 : d1;
+    bound2 = bound * bound * (1.0f + 1e-6f);
+  }
+}
+
+// The same for one pixel by a whole warp (every lane passes the same pixel): lane l scores the peaks l, l + 32, ...
+// with the pixel's values fetched by every lane (the same addresses: one transaction per load), then the lanes' results
+// are merged -- smaller distance first, lower k on equal distances, which is what the serial scan in ascending k gives.
+// A single thread scanning hundreds of peaks is a chain of dependent row fetches that takes as long as the rest of the
+// kernel; 32 lanes share it.
+template <typename T, int D, bool WANT2>
+__device__ __forceinline__ void near_full_scan_warp(const T* __restrict__ p, size_t plane, int K,
+                                                    const float* __restrict__ cand_img, float& d1, float& d2, int& k1) {
+  const float inf = __int_as_float(0x7f800000);
+  const int lane = threadIdx.x & 31;
+  float2 e2[D / 2];
+#pragma unroll
+  for (int c = 0; c < D / 2; ++c) {
+    e2[c].x = Elem<T>::load1(p + (size_t)c * plane);
+    e2[c].y = Elem<T>::load1(p + (size_t)(D / 2 + c) * plane);
+  }
+  d1 = d2 = inf;
+  k1 = 0x7fffffff;
+  float bound2 = inf;
+  for (int k = lane; k < K; k += 32) {
+    const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
+    if (d < d1) { d2 = d1; d1 = d; k1 = k; }
+    else if (d < d2) { d2 = d; }
+    const float bound = WANT2 ? d2 : d1;
+    bound2 = bound * bound * (1.0f + 1e-6f);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float od1 = __shfl_xor_sync(0xffffffffu, d1, off), od2 = __shfl_xor_sync(0xffffffffu, d2, off);
+    const int ok1 = __shfl_xor_sync(0xffffffffu, k1, off);
+    const bool other_wins = od1 < d1 || (od1 == d1 && ok1 < k1);
+    const float loser = other_wins ? d1 : od1;       // the larger of the two best distances is a runner-up candidate
+    if (other_wins) { d1 = od1; k1 = ok1; }
+    d2 = fminf(fminf(d2, od2), loser);
+  }
+  if (k1 == 0x7fffffff) k1 = -1;
+}
+
+// Called by one thread of a CTA with the hard pixels it has just found among `visited` pixels: updates the image's
+// totals and decides whether the image is handed on.  Returns the stop flag.
+// (Hard pixels come in clusters -- an instance whose peak a stronger neighbour suppressed --, so the ratio is only
+// looked at once an eighth of the image has been visited.)
+__device__ __forceinline__ uint32_t near_account(uint32_t* state, uint32_t visited, uint32_t n_hard, uint32_t min_proc) {
+  const uint32_t proc = atomicAdd(&state[kNearProcessed], visited) + visited;
+  if (!n_hard) return *reinterpret_cast<volatile uint32_t*>(&state[kNearGiveUp]);
+  const uint32_t hd = atomicAdd(&state[kNearHard], n_hard) + n_hard;
+  uint32_t stop = *reinterpret_cast<volatile uint32_t*>(&state[kNearGiveUp]);
+  if (!stop && proc >= min_proc && hd > proc / 8u) {
+    atomicExch(&state[kNearGiveUp], 1u);
+    stop = 1u;
+  }
+  return stop;
+}
+
+__device__ __forceinline__ void near_flush_counters(uint32_t* state, uint32_t n_rejected, uint32_t n_pairs,
+                                                    uint32_t n_multi, uint32_t n_full) {
+  // one atomic per warp and counter, into this kernel's own words; the last kernel of the chain folds them into the
+  // image's counters unless the image was handed on (a CTA that returned early has dropped its share)
+  const uint32_t rej = __reduce_add_sync(0xffffffffu, n_rejected), prs = __reduce_add_sync(0xffffffffu, n_pairs),
+                 mul = __reduce_add_sync(0xffffffffu, n_multi), ful = __reduce_add_sync(0xffffffffu, n_full);
+  if ((threadIdx.x & 31) == 0) {
+    if (rej) atomicAdd(&state[kNearCnt + 0], rej);
+    if (prs) atomicAdd(&state[kNearCnt + 1], prs);
+    if (mul) atomicAdd(&state[kNearCnt + 2], mul);
+    if (ful) atomicAdd(&state[kNearCnt + 3], ful);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ one thread per pixel
 
 template <typename T, int FT, bool WANT2>
 __global__ void __launch_bounds__(kNearThreads, FT == 16 ? 2 : 3)
@@ -78,59 +202,31 @@ assign_near_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, in
     int k1 = -1;
     bool hard = act && (k0 < 0 || k0 >= K);
     uint32_t scored = 0;
-    if (act && !hard) {
-      const float t = score_direct<D>(e2, reinterpret_cast<const float2*>(ref_img + (size_t)k0 * D), inf);
-      const uint32_t* list = nbr_img + (size_t)k0 * kNbrCap;
-      float bound2 = inf;
-      int j = 0;
-      for (; j < kNbrCap; ++j) {
-        const uint32_t ent = __ldg(list + j);
-        if (ent == kNbrEnd) break;                                   // every candidate of the image has been seen
-        const float G = (float)(ent >> 12) * (1.0f / 65536.0f);
-        const float U = WANT2 ? d2 : d1;
-        if (G > (U + t) * kNearSlack) break;                         // this one and all later ones: d >= G - t > U
-        const int k = (int)(ent & 0xfffu);
-        const float d = (same_rows && k == k0)
-                            ? t
-                            : score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
-        ++scored;
-        if (d < d1 || (d == d1 && k < k1)) { d2 = d1; d1 = d; k1 = k; }   // the lowest k keeps an exact tie
-        else if (d < d2) { d2 = d; }
-        const float bound = WANT2 ? d2 : d1;
-        bound2 = bound * bound * (1.0f + 1e-6f);
-      }
-      hard = (j == kNbrCap) && K > kNbrCap;                          // the list ran out before the bound closed it
-    }
+    if (act && !hard) near_walk<D, WANT2>(e2, k0, K, same_rows, ref_img, cand_img, nbr_img, d1, d2, k1, hard, scored);
 
     // hard pixels: count them, let the image go to the filtered kernel if there are too many, else score every peak
     // (the ratio is taken over all pixels visited, participating or not)
     const int n_hard = __syncthreads_count(hard);
     if (n_hard) {
-      if (tid == 0) {
-        const uint32_t proc = atomicAdd(&state[kNearProcessed], (uint32_t)kNearThreads) + (uint32_t)kNearThreads;
-        const uint32_t hd = atomicAdd(&state[kNearHard], (uint32_t)n_hard) + (uint32_t)n_hard;
-        uint32_t stop = *reinterpret_cast<volatile uint32_t*>(&state[kNearGiveUp]);
-        if (!stop && proc >= 8192u && hd > proc / 8u) {
-          atomicExch(&state[kNearGiveUp], 1u);
-          stop = 1u;
-        }
-        s_stop = stop;
-      }
+      if (tid == 0) s_stop = near_account(state, (uint32_t)kNearThreads, (uint32_t)n_hard, max(8192u, (uint32_t)HW / 8u));
       __syncthreads();
       if (s_stop) return;                                            // the filtered kernel redoes the whole image
-      if (hard) {
-        d1 = d2 = inf;
-        k1 = -1;
-        float bound2 = inf;
-        for (int k = 0; k < K; ++k) {
-          const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
-          if (d < d1) { d2 = d1; d1 = d; k1 = k; }
-          else if (d < d2) { d2 = d; }
-          const float bound = WANT2 ? d2 : d1;
-          bound2 = bound * bound * (1.0f + 1e-6f);
+      // every peak, by the whole warp, one hard pixel after the other
+      uint32_t hm = __ballot_sync(0xffffffffu, hard);
+      while (hm) {
+        const int src_lane = __ffs(hm) - 1;
+        hm &= hm - 1;
+        const long long nn = __shfl_sync(0xffffffffu, n, src_lane);
+        float w1, w2;
+        int wk;
+        near_full_scan_warp<T, D, WANT2>(emb + (size_t)b * D * plane + nn, plane, K, cand_img, w1, w2, wk);
+        if ((tid & 31) == src_lane) {
+          d1 = w1;
+          d2 = w2;
+          k1 = wk;
+          scored = (uint32_t)K;
+          ++n_full;
         }
-        scored = (uint32_t)K;
-        ++n_full;
       }
     } else if (tid == 0) {
       atomicAdd(&state[kNearProcessed], (uint32_t)kNearThreads);
@@ -152,16 +248,434 @@ assign_near_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, in
       }
     }
   }
-  // counters: one atomic per warp and counter, into this kernel's own words; the last kernel of the chain folds them
-  // into the image's counters unless the image was handed on (a CTA that returned above has dropped its share)
-  const uint32_t rej = __reduce_add_sync(0xffffffffu, n_rejected), prs = __reduce_add_sync(0xffffffffu, n_pairs),
-                 mul = __reduce_add_sync(0xffffffffu, n_multi), ful = __reduce_add_sync(0xffffffffu, n_full);
-  if ((tid & 31) == 0) {
-    if (rej) atomicAdd(&state[kNearCnt + 0], rej);
-    if (prs) atomicAdd(&state[kNearCnt + 1], prs);
-    if (mul) atomicAdd(&state[kNearCnt + 2], mul);
-    if (ful) atomicAdd(&state[kNearCnt + 3], ful);
+  near_flush_counters(state, n_rejected, n_pairs, n_multi, n_full);
+}
+
+// ------------------------------------------------------------------------------------------------ the streaming kernel
+
+// Square root to within 2^-21 relative (the special-function unit's), for bounds that carry their own slack.
+__device__ __forceinline__ float fast_sqrt(float x) {
+  float r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+constexpr int kStreamThreads = 256;
+// What turns a distance accumulated in packed binary16 into an upper bound of the true one.  Per axis the sum has at
+// most 32 non-negative terms: each rounding (difference, fused multiply-add) is within 2^-11 relative, so the sum is
+// within 34 * 2^-11 < 1.7 %, its root within 0.85 %; the candidate rows are rounded to binary16 (2^-12 per component,
+// |r| <= 1: at most sqrt(32) * 2^-12 = 0.0014 on the norm); binary32 pixels are rounded to binary16 first (2^-11
+// relative per component: at most 0.0005 ||v||, with ||v|| <= 8 for anything that is not far from every row anyway).
+// Non-finite sums (overflow) fail every comparison and send the pixel to the exact walk.
+constexpr float kHalfRel = 1.01f, kHalfAbs = 0.008f;
+
+// Warps stream the embedding with 128-bit plane loads, a thread per (8-pixel group, axis) -- the access pattern of the
+// voting kernel -- and only have to CERTIFY, per pixel, that the second entry of its peak's list is out of reach:
+//     G_2 > (d_ub + t_ub) * slack,   t_ub >= t (distance to the reference point),  d_ub >= d (to the first candidate).
+// Upper bounds need no exact arithmetic: the sums of squares are accumulated in packed binary16 (two pixels per
+// instruction, no widening of the loaded values) and inflated by their worst-case error.  A certified pixel gets the
+// first candidate's label; every other pixel -- not certified, no peak for its bin, tau finite (the exact distance is
+// then needed) -- is appended to the image's queue in global memory (`slow_q`, capacity q_cap; its fill is
+// near_state[kNearQueue]) and decided exactly by assign_near_walk_kernel afterwards.  A queue that overflows hands the
+// image to the filtered kernel, like too many hard pixels do.
+//
+// Dynamic shared memory (`smem_rows_bytes`): binary16 copies of the reference rows [K][D] and, unless SAME, of the
+// candidate rows; an image whose rows do not fit reads them from global memory (`ref_h` / `cand_h`, [K][D] binary16,
+// written by peak_graph_kernel).  Needs 16-byte aligned planes, mask and labels, and H*W a multiple of the group size.
+template <typename T, int FT, bool SAME>
+__global__ void __launch_bounds__(kStreamThreads, 3)
+assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int K_max,
+                          const __half* __restrict__ ref_h, const __half* __restrict__ cand_h,
+                          const uint32_t* __restrict__ nbr, const int32_t* __restrict__ cell_peak,
+                          const uint32_t* __restrict__ pix_cell, int cells, const int32_t* __restrict__ count_ptr, float tau,
+                          int32_t* __restrict__ labels, uint32_t* __restrict__ near_state, uint32_t* __restrict__ slow_q,
+                          int q_cap, int k_min, int smem_rows_bytes) {
+  extern __shared__ __align__(16) unsigned char near_smem[];
+  grid_dependency_sync();
+  constexpr int VEC = Elem<T>::kVec;           // pixels per 128-bit load
+  constexpr int H2 = VEC / 2;
+  constexpr int F = FT, D = 4 * FT, D2 = 2 * FT;
+  const int b = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const size_t plane = (size_t)HW;
+  const int K = count_ptr[b];
+  if (K < k_min) return;                       // few peaks: the all-pairs kernel's image
+  uint32_t* state = near_state + b * kNearStride;
+  if (K > kNearMaxPeaks) {                      // no lists were made: the filtered kernel's image
+    if (tid == 0 && blockIdx.x == 0) state[kNearGiveUp] = 1u;
+    return;
   }
+  const T* e_img = emb + (size_t)b * D * plane;
+  const uint32_t* nbr_img = nbr + (size_t)b * K_max * kNbrCap;
+  const int32_t* cp_img = cell_peak + (size_t)b * cells;
+  const uint32_t* pc_img = pix_cell + (size_t)b * plane;
+  int32_t* lab_img = labels + (size_t)b * plane;
+  uint32_t* q_img = slow_q + (size_t)b * q_cap;
+
+  // the rows this CTA bounds against (binary16): in shared memory if this image's peaks fit
+  const bool rows_in_smem = (size_t)K * D * sizeof(__half) * (SAME ? 1 : 2) <= (size_t)smem_rows_bytes;
+  const __half* rows_ref = rows_in_smem ? reinterpret_cast<const __half*>(near_smem) : ref_h + (size_t)b * K_max * D;
+  const __half* rows_cand = SAME ? rows_ref
+                                 : (rows_in_smem ? reinterpret_cast<const __half*>(near_smem) + (size_t)K * D
+                                                 : cand_h + (size_t)b * K_max * D);
+  if (rows_in_smem) {
+    const uint4* g_ref = reinterpret_cast<const uint4*>(ref_h + (size_t)b * K_max * D);
+    const uint4* g_cand = reinterpret_cast<const uint4*>(cand_h + (size_t)b * K_max * D);
+    uint4* dst = reinterpret_cast<uint4*>(near_smem);
+    const int n16 = K * D * (int)sizeof(__half) / 16;
+    for (int i = tid; i < n16; i += kStreamThreads) {
+      dst[i] = __ldg(g_ref + i);
+      if (!SAME) dst[n16 + i] = __ldg(g_cand + i);
+    }
+    __syncthreads();
+  }
+
+  const bool certify = !(tau < __int_as_float(0x7f800000));   // with a finite tau every pixel needs its exact distance
+  const uint32_t min_proc = max(8192u, (uint32_t)HW / 8u);
+  uint32_t n_pairs = 0;
+  uint32_t visited = 0, hard_acc = 0;          // lane 0: not yet added to the image's totals
+  const int axis = lane & 1;                    // lanes 2j and 2j+1 share a group
+  const long long n_groups = (long long)HW / VEC;
+  const long long n_steps = (n_groups + 15) / 16;
+  const long long warp0 = (long long)blockIdx.x * (kStreamThreads / 32) + wid, n_warps = (long long)gridDim.x * (kStreamThreads / 32);
+
+  auto load_take = [&](long long step) -> uint32_t {      // participation bits of this lane's group in that step
+    const long long grp = step * 16 + (lane >> 1);
+    if (step < 0 || grp >= n_groups) return 0u;
+    if (!fg) return (1u << VEC) - 1u;
+    const uint8_t* m = fg + (size_t)b * plane + (size_t)grp * VEC;
+    uint32_t take = 0;
+    if constexpr (VEC == 8) {
+      const uint2 w = __ldg(reinterpret_cast<const uint2*>(m));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        take |= (((w.x >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+        take |= (((w.y >> (8 * j)) & 0xffu) ? 1u : 0u) << (4 + j);
+      }
+    } else {
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(m));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) take |= (((w >> (8 * j)) & 0xffu) ? 1u : 0u) << j;
+    }
+    return take;
+  };
+
+  // from the end of the image backwards: what the voting kernel read last may still be in L2
+  long long step = n_steps - 1 - warp0;
+  uint32_t take_next = load_take(step);
+  for (; step >= 0; step -= n_warps) {
+    const long long grp = step * 16 + (lane >> 1);
+    const bool in_range = grp < n_groups;
+    const size_t pix0 = (size_t)(in_range ? grp : 0) * VEC;
+    const uint32_t take = take_next;
+    take_next = load_take(step - n_warps);      // the next step's mask is on its way while this step runs
+    const bool have = take != 0;
+    const T* src = e_img + pix0 + (size_t)axis * D2 * plane;
+
+    // the first plane loads and the bins go out together
+    constexpr int LB = F < 4 ? F : 4;          // harmonics whose plane loads are in flight together (2 loads each)
+    uint4 raw[2 * LB];
+    uint32_t cell[VEC];
+    if (have) {
+#pragma unroll
+      for (int q = 0; q < 2 * LB; ++q) raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)q * plane));
+#pragma unroll
+      for (int j = 0; j < VEC; j += 4) {
+        const uint4 c4 = __ldg(reinterpret_cast<const uint4*>(pc_img + pix0 + j));
+        cell[j] = c4.x; cell[j + 1] = c4.y; cell[j + 2] = c4.z; cell[j + 3] = c4.w;
+      }
+    }
+    // bins -> peaks.  Pixels of one group nearly always share their peak; a group with several peaks keeps them per pixel.
+    int kpix[VEC];
+    uint32_t voted = 0;                         // participating pixels that voted
+    bool uniform = true;
+    int ku = -1;
+    if (have) {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        int k = -1;
+        if (((take >> j) & 1u) && cell[j] != 0xffffffffu && (int)cell[j] < cells) {
+          voted |= 1u << j;
+          k = (j > 0 && cell[j] == cell[j - 1] && ((voted >> (j - 1)) & 1u)) ? kpix[j - 1] : __ldg(cp_img + cell[j]);
+          if (k >= K) k = -1;
+          if (k >= 0) {
+            if (ku < 0) ku = k;
+            else if (k != ku) uniform = false;
+          }
+        }
+        kpix[j] = k;
+      }
+    }
+    // the first two entries of the peaks' lists (one lookup for a uniform group)
+    uint2 e01u = make_uint2(0u, kNbrEnd);
+    if (ku >= 0) e01u = __ldg(reinterpret_cast<const uint2*>(nbr_img + (size_t)ku * kNbrCap));
+    const int kfu = (int)(e01u.x & 0xfffu);
+
+    __half2 s[H2], sc[H2];                      // sums of squares so far, two pixels each: reference rows, candidates
+#pragma unroll
+    for (int j = 0; j < H2; ++j) s[j] = sc[j] = __float2half2_rn(0.0f);
+    // widening-free view of one 128-bit load as pixel pairs
+    auto pairs_of = [](const uint4& r, __half2 (&v)[H2]) {
+      if constexpr (sizeof(T) == 2) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < H2; ++j) v[j] = *reinterpret_cast<const __half2*>(&w[j]);
+      } else {
+        v[0] = __floats2half2_rn(__uint_as_float(r.x), __uint_as_float(r.y));
+        v[1] = __floats2half2_rn(__uint_as_float(r.z), __uint_as_float(r.w));
+      }
+    };
+    if (ku >= 0 && uniform) {
+      // ---- the common case: one peak for the whole group, its row values splat over the pixel pairs
+      const __half* rr = rows_ref + (size_t)ku * D + axis * D2;
+      const __half* rc = rows_cand + (size_t)kfu * D + axis * D2;
+#pragma unroll
+      for (int l0 = 0; l0 < F; l0 += LB) {
+        if (l0 > 0) {
+#pragma unroll
+          for (int q = 0; q < 2 * LB; ++q)
+            raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + q) * plane));
+        }
+#pragma unroll
+        for (int q = 0; q < 2 * LB; q += 2) {
+          const int c = 2 * l0 + q;                // channels c and c + 1: one 32-bit row load serves both
+          const __half2 r2 = *reinterpret_cast<const __half2*>(rr + c);
+          const __half2 r_lo = __low2half2(r2), r_hi = __high2half2(r2);
+          __half2 v0[H2], v1[H2];
+          pairs_of(raw[q], v0);
+          pairs_of(raw[q + 1], v1);
+#pragma unroll
+          for (int j = 0; j < H2; ++j) {
+            const __half2 d = __hsub2(v0[j], r_lo);
+            s[j] = __hfma2(d, d, s[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < H2; ++j) {
+            const __half2 d = __hsub2(v1[j], r_hi);
+            s[j] = __hfma2(d, d, s[j]);
+          }
+          if constexpr (!SAME) {
+            const __half2 q2 = *reinterpret_cast<const __half2*>(rc + c);
+            const __half2 q_lo = __low2half2(q2), q_hi = __high2half2(q2);
+#pragma unroll
+            for (int j = 0; j < H2; ++j) {
+              const __half2 d = __hsub2(v0[j], q_lo);
+              sc[j] = __hfma2(d, d, sc[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < H2; ++j) {
+              const __half2 d = __hsub2(v1[j], q_hi);
+              sc[j] = __hfma2(d, d, sc[j]);
+            }
+          }
+        }
+      }
+    } else if (ku >= 0) {
+      // ---- a group with several peaks: every pixel against its own rows (rare: instance borders)
+      int kr[VEC], kc[VEC];
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        kr[j] = kpix[j] >= 0 ? kpix[j] : ku;
+        kc[j] = SAME ? kr[j] : (int)(__ldg(nbr_img + (size_t)kr[j] * kNbrCap) & 0xfffu);
+      }
+#pragma unroll 1
+      for (int l0 = 0; l0 < F; l0 += LB) {
+        if (l0 > 0) {
+#pragma unroll
+          for (int q = 0; q < 2 * LB; ++q)
+            raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + q) * plane));
+        }
+#pragma unroll
+        for (int q = 0; q < 2 * LB; ++q) {
+          const int c = axis * D2 + 2 * l0 + q;
+          __half2 v[H2];
+          pairs_of(raw[q], v);
+#pragma unroll
+          for (int j = 0; j < H2; ++j) {
+            const __half2 r = __halves2half2(rows_ref[(size_t)kr[2 * j] * D + c], rows_ref[(size_t)kr[2 * j + 1] * D + c]);
+            const __half2 d = __hsub2(v[j], r);
+            s[j] = __hfma2(d, d, s[j]);
+            if constexpr (!SAME) {
+              const __half2 qq = __halves2half2(rows_cand[(size_t)kc[2 * j] * D + c], rows_cand[(size_t)kc[2 * j + 1] * D + c]);
+              const __half2 dc = __hsub2(v[j], qq);
+              sc[j] = __hfma2(dc, dc, sc[j]);
+            }
+          }
+        }
+      }
+    }
+    // swap with the partner lane: afterwards every lane has both axes' sums of its half of the pixels
+    // (all register-array indices below are compile-time constants: the axis picks between two of them)
+    __half2 so[H2], sco[H2];
+#pragma unroll
+    for (int j = 0; j < H2; ++j) {
+      uint32_t w = *reinterpret_cast<uint32_t*>(&s[j]);
+      w = __shfl_xor_sync(0xffffffffu, w, 1);
+      so[j] = *reinterpret_cast<__half2*>(&w);
+      if constexpr (!SAME) {
+        uint32_t wc = *reinterpret_cast<uint32_t*>(&sc[j]);
+        wc = __shfl_xor_sync(0xffffffffu, wc, 1);
+        sco[j] = *reinterpret_cast<__half2*>(&wc);
+      } else {
+        sco[j] = so[j];
+      }
+    }
+    int my_label[H2];
+    uint32_t n_likely_hard = 0;
+    constexpr int Q2 = H2 / 2;                  // half2 registers per half of the group (2 for binary16, 1 for binary32)
+#pragma unroll
+    for (int jj = 0; jj < H2; ++jj) {
+      const int j = axis * H2 + jj;              // the axis-0 lane finishes the first half, the axis-1 lane the second
+      // own sums of pixel jj (first half) and of pixel H2 + jj (second half), and the partner's
+      const float2 own_lo = __half22float2(s[jj / 2]), own_hi = __half22float2(s[Q2 + jj / 2]);
+      const float2 oth_lo = __half22float2(so[jj / 2]), oth_hi = __half22float2(so[Q2 + jj / 2]);
+      const float2 cwn_lo = __half22float2(sc[jj / 2]), cwn_hi = __half22float2(sc[Q2 + jj / 2]);
+      const float2 cth_lo = __half22float2(sco[jj / 2]), cth_hi = __half22float2(sco[Q2 + jj / 2]);
+      const float sx = axis == 0 ? ((jj & 1) ? own_lo.y : own_lo.x) : ((jj & 1) ? oth_hi.y : oth_hi.x);
+      const float sy = axis == 0 ? ((jj & 1) ? oth_lo.y : oth_lo.x) : ((jj & 1) ? own_hi.y : own_hi.x);
+      const float cx = axis == 0 ? ((jj & 1) ? cwn_lo.y : cwn_lo.x) : ((jj & 1) ? cth_hi.y : cth_hi.x);
+      const float cy = axis == 0 ? ((jj & 1) ? cth_lo.y : cth_lo.x) : ((jj & 1) ? cwn_hi.y : cwn_hi.x);
+      const int k0j = axis == 0 ? kpix[jj] : kpix[H2 + jj];
+      int label = 0;
+      bool slow = false;
+      if ((voted >> j) & 1u) {
+        slow = true;
+        bool likely_hard = k0j < 0;
+        if (k0j >= 0) {
+          const uint2 e01 = uniform ? e01u : __ldg(reinterpret_cast<const uint2*>(nbr_img + (size_t)k0j * kNbrCap));
+          const int kfj = (int)(e01.x & 0xfffu);
+          const float t = (fast_sqrt(sx) + fast_sqrt(sy)) * kHalfRel + kHalfAbs;
+          const float dub = SAME ? t : (fast_sqrt(cx) + fast_sqrt(cy)) * kHalfRel + kHalfAbs;
+          const float reach = (dub + t) * kNearSlack;
+          // the list's first entry is the candidate bounded above (with refined candidates that must be k0 itself:
+          // an identical row with a lower index may precede it); the second entry decides whether the walk is over
+          const bool first_ok = !SAME || kfj == k0j;
+          const bool closed = e01.y == kNbrEnd || (float)(e01.y >> 12) * (1.0f / 65536.0f) > reach;
+          if (certify && first_ok && closed) {
+            label = kfj + 1;
+            slow = false;
+            ++n_pairs;
+          } else if (K > kNbrCap) {
+            const uint32_t el = __ldg(nbr_img + (size_t)k0j * kNbrCap + kNbrCap - 1);
+            // (a comparison that a non-finite bound fails counts as likely hard)
+            likely_hard = el != kNbrEnd && !((float)(el >> 12) * (1.0f / 65536.0f) > reach);
+          }
+        }
+        if (likely_hard) ++n_likely_hard;
+      }
+      my_label[jj] = label;
+      // queue the pixel: one atomic per warp and round
+      const uint32_t sm = __ballot_sync(0xffffffffu, slow);
+      if (sm) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&state[kNearQueue], (uint32_t)__popc(sm));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (slow) {
+          const uint32_t at = base + (uint32_t)__popc(sm & ((1u << lane) - 1u));
+          if (at < (uint32_t)q_cap) q_img[at] = (uint32_t)(pix0 + j);
+        }
+        if (lane == 0 && base + (uint32_t)__popc(sm) > (uint32_t)q_cap) atomicExch(&state[kNearGiveUp], 1u);
+      }
+    }
+    if (in_range) {
+      int32_t* dst = lab_img + pix0 + (size_t)axis * H2;
+      if constexpr (VEC == 8)
+        *reinterpret_cast<int4*>(dst) = make_int4(my_label[0], my_label[1], my_label[2], my_label[3]);
+      else
+        *reinterpret_cast<int2*>(dst) = make_int2(my_label[0], my_label[1]);
+    }
+    // ---- hand the image on if too many pixels cannot be closed by the bounds (before the walks are paid for)
+    const uint32_t nh = __reduce_add_sync(0xffffffffu, n_likely_hard);
+    visited += 16u * VEC;
+    hard_acc += nh;
+    uint32_t stop = 0;
+    if (lane == 0 && (hard_acc || visited >= 4096u)) {
+      stop = near_account(state, visited, hard_acc, min_proc);
+      visited = hard_acc = 0;
+    }
+    if (__shfl_sync(0xffffffffu, stop, 0)) return;     // the filtered kernel redoes the whole image
+  }
+  if (lane == 0 && visited) near_account(state, visited, hard_acc, min_proc);
+  near_flush_counters(state, 0u, n_pairs, 0u, 0u);
+}
+
+// The walk of the pixels that the streaming kernel queued, one thread per pixel.
+template <typename T, int FT>
+__global__ void __launch_bounds__(kNearThreads, FT == 16 ? 2 : 3)
+assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const float* __restrict__ ref2,
+                        const float* __restrict__ cand2, const uint32_t* __restrict__ nbr,
+                        const int32_t* __restrict__ cell_peak, const uint32_t* __restrict__ pix_cell, int cells,
+                        const int32_t* __restrict__ count_ptr, float tau, int32_t* __restrict__ labels,
+                        uint32_t* __restrict__ near_state, const uint32_t* __restrict__ slow_q, int q_cap, int k_min) {
+  grid_dependency_sync();
+  constexpr int D = 4 * FT;
+  const int b = blockIdx.y;
+  const size_t plane = (size_t)HW;
+  const int K = count_ptr[b];
+  if (K < k_min || K > kNearMaxPeaks) return;
+  uint32_t* state = near_state + b * kNearStride;
+  if (state[kNearGiveUp]) return;                // the filtered kernel redoes the whole image
+  const int n_q = (int)min(state[kNearQueue], (uint32_t)q_cap);
+  const bool same_rows = ref2 == cand2;
+  const float* ref_img = ref2 + (size_t)b * K_max * D;
+  const float* cand_img = cand2 + (size_t)b * K_max * D;
+  const uint32_t* nbr_img = nbr + (size_t)b * K_max * kNbrCap;
+  const int32_t* cp_img = cell_peak + (size_t)b * cells;
+  const float inf = __int_as_float(0x7f800000);
+  uint32_t n_rejected = 0, n_pairs = 0, n_multi = 0, n_full = 0;
+  const int lane = threadIdx.x & 31;
+  for (int base = blockIdx.x * kNearThreads; base < n_q; base += gridDim.x * kNearThreads) {   // uniform per CTA
+    const int i = base + threadIdx.x;
+    const bool have = i < n_q;
+    const size_t n = have ? slow_q[(size_t)b * q_cap + i] : 0;
+    const T* p = emb + (size_t)b * D * plane + n;
+    float d1 = inf, d2 = inf;
+    int k1 = -1;
+    bool hard = false;
+    uint32_t scored = 0;
+    if (have) {
+      const uint32_t cell = __ldg(pix_cell + (size_t)b * plane + n);
+      int k0 = (cell != 0xffffffffu && (int)cell < cells) ? __ldg(cp_img + cell) : -1;
+      if (k0 >= K) k0 = -1;
+      hard = k0 < 0;
+      if (!hard) {
+        float2 e2[D / 2];
+#pragma unroll
+        for (int c = 0; c < D / 2; ++c) {
+          e2[c].x = Elem<T>::load1(p + (size_t)c * plane);
+          e2[c].y = Elem<T>::load1(p + (size_t)(D / 2 + c) * plane);
+        }
+        near_walk<D, false>(e2, k0, K, same_rows, ref_img, cand_img, nbr_img, d1, d2, k1, hard, scored);
+      }
+    }
+    // hard pixels: every peak, by the whole warp, one pixel after the other
+    uint32_t hm = __ballot_sync(0xffffffffu, hard);
+    while (hm) {
+      const int src_lane = __ffs(hm) - 1;
+      hm &= hm - 1;
+      const unsigned long long pp = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)p, src_lane);
+      float w1, w2;
+      int wk;
+      near_full_scan_warp<T, D, false>(reinterpret_cast<const T*>((uintptr_t)pp), plane, K, cand_img, w1, w2, wk);
+      if (lane == src_lane) {
+        d1 = w1;
+        k1 = wk;
+        scored = (uint32_t)K;
+        ++n_full;
+      }
+    }
+    if (have) {
+      if (!hard && scored > 1) ++n_multi;
+      n_pairs += scored;
+      int label = 0;
+      if (k1 >= 0) {
+        if (d1 < tau) label = k1 + 1;
+        else ++n_rejected;
+      }
+      labels[(size_t)b * plane + n] = label;
+    }
+  }
+  near_flush_counters(state, n_rejected, n_pairs, n_multi, n_full);
 }
 
 }  // namespace cpe

@@ -108,6 +108,10 @@ struct PruneArgs {
   const int32_t* cell_peak = nullptr;
   const uint32_t* pix_cell = nullptr;
   uint32_t* near_state = nullptr;
+  uint32_t* slow_q = nullptr;
+  int q_cap = 0;
+  void* ref_h = nullptr;
+  void* cand_h = nullptr;
 };
 
 // Stage 4+5.  The number of peaks is only known on the device, so several kernels are enqueued and every image is
@@ -136,13 +140,15 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   }
   int rc = CPE_OK;
   if (pr) {
-    rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->nbr);
+    rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->ref_h,
+                                      pr->cand_h, pr->nbr);
     if (rc) return rc;
   }
   if (ev_lists) CPE_CUDA(cudaEventRecord(ev_lists, st));
   if (pr) {
-    rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref2, pr->cand2, pr->nbr, pr->cell_peak, pr->pix_cell,
-                                       cells, count, labels, best, second, pr->near_state, k_limit + 1);
+    rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref_emb, peak_emb, pr->ref2, pr->cand2, pr->nbr,
+                                       pr->cell_peak, pr->pix_cell, cells, count, labels, best, second, pr->near_state,
+                                       k_limit + 1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h);
     if (rc) return rc;
   }
   // (also with a limit of 0: an image without any peak still gets its all-zero label map from this kernel)
@@ -215,6 +221,10 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     pr.cell_peak = reinterpret_cast<const int32_t*>(ws + L.cell_peak);
     pr.pix_cell = reinterpret_cast<const uint32_t*>(ws + L.pix_cell);
     pr.near_state = reinterpret_cast<uint32_t*>(ws + L.near_state);
+    pr.slow_q = reinterpret_cast<uint32_t*>(ws + L.slow_q);
+    pr.q_cap = L.q_cap;
+    pr.ref_h = ws + L.ref_h;
+    pr.cand_h = ws + L.cand_h;
   }
   const bool one_peak_cta = L.words <= cpe::kPeakStageWords;
   const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes;

@@ -12,80 +12,100 @@
 // A list entry is (Gq << 12) | k with Gq = floor(G * 2^16 * (1 - 2^-15)), i.e. G rounded DOWN by more than its own
 // rounding error (at most (2F + 3) units in the last place), as the bound needs; entries ascend as plain integers.
 // Unused entries are 0xffffffff.  Also written: the reference and candidate rows with their x and y halves
-// interleaved, row[2c] = x channel c, row[2c + 1] = y channel c, the operand layout of score_direct.
+// interleaved, row[2c] = x channel c, row[2c + 1] = y channel c, the operand layout of score_direct, and binary16
+// copies of the rows in plain order for the streaming kernel's bounds.
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "cpe_common.cuh"
 
 namespace cpe {
 
-constexpr int kGraphThreads = 256;
+constexpr int kGraphThreads = 128;
 constexpr uint32_t kNbrEnd = 0xffffffffu;
 
-// One warp per peak k0; lanes share the candidates.  Dynamic shared memory: (8 warps) x K_cap keys.
+// One CTA per peak k0 (the grid strides over the peaks); its threads share the candidates.
+template <int FT>
 __global__ void __launch_bounds__(kGraphThreads)
 peak_graph_kernel(const float* __restrict__ ref_emb, const float* __restrict__ cand_emb,
-                  const int32_t* __restrict__ count_ptr, int K_max, int F, int k_min, float* __restrict__ ref2,
-                  float* __restrict__ cand2, uint32_t* __restrict__ nbr) {
-  extern __shared__ uint32_t s_keys_all[];
-  __shared__ float s_ref[kGraphThreads / 32][64];
+                  const int32_t* __restrict__ count_ptr, int K_max, int k_min, float* __restrict__ ref2,
+                  float* __restrict__ cand2, __half* __restrict__ ref_h, __half* __restrict__ cand_h,
+                  uint32_t* __restrict__ nbr) {
+  constexpr int D = 4 * FT, D2 = 2 * FT;
+  __shared__ __align__(16) float s_ref[D];                    // plain order: x half, y half
+  __shared__ __align__(16) uint32_t s_keys[kNearMaxPeaks];
   grid_dependency_sync();
   const int b = blockIdx.y;
   const int K = count_ptr[b];
   if (K < k_min || K > kNearMaxPeaks) return;
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int D = 4 * F, D2 = 2 * F;
+  const int tid = threadIdx.x;
   const float* ref_img = ref_emb + (size_t)b * K_max * D;
   const float* cand_img = cand_emb + (size_t)b * K_max * D;
-  uint32_t* keys = s_keys_all + (size_t)wid * kNearMaxPeaks;
   const bool same = ref2 == cand2;
+  const int Kpad = (K + 3) & ~3;
 
-  for (int k0 = blockIdx.x * (kGraphThreads / 32) + wid; k0 < K; k0 += gridDim.x * (kGraphThreads / 32)) {
-    // this peak's rows, interleaved
-    for (int c = lane; c < D; c += 32) {
-      const int src = (c & 1) ? D2 + (c >> 1) : (c >> 1);
-      const float r = ref_img[(size_t)k0 * D + src];
-      s_ref[wid][c] = r;
-      ref2[((size_t)b * K_max + k0) * D + c] = r;
-      if (!same) cand2[((size_t)b * K_max + k0) * D + c] = cand_img[(size_t)k0 * D + src];
-    }
-    __syncwarp();
-    // G(k0, k) for the lane's candidates
-    for (int k = lane; k < K; k += 32) {
-      const float* e = cand_img + (size_t)k * D;
-      float sx = 0.0f, sy = 0.0f;
-      for (int c = 0; c < D2; ++c) {
-        const float tx = s_ref[wid][2 * c] - e[c];
-        const float ty = s_ref[wid][2 * c + 1] - e[D2 + c];
-        sx = fmaf(tx, tx, sx);
-        sy = fmaf(ty, ty, sy);
+  for (int k0 = blockIdx.x; k0 < K; k0 += gridDim.x) {
+    // this peak's rows: a plain copy for the distances below, interleaved copies for the assignment
+    for (int c = tid; c < D; c += kGraphThreads) {
+      const float r = ref_img[(size_t)k0 * D + c];
+      s_ref[c] = r;
+      const int dst = c < D2 ? 2 * c : 2 * (c - D2) + 1;
+      ref2[((size_t)b * K_max + k0) * D + dst] = r;
+      ref_h[((size_t)b * K_max + k0) * D + c] = __float2half_rn(r);
+      if (!same) {
+        const float e = cand_img[(size_t)k0 * D + c];
+        cand2[((size_t)b * K_max + k0) * D + dst] = e;
+        cand_h[((size_t)b * K_max + k0) * D + c] = __float2half_rn(e);
       }
-      const float G = sqrtf(sx) + sqrtf(sy);
-      const float q = floorf(G * (65536.0f * (1.0f - 1.0f / 32768.0f)));
-      const uint32_t Gq = (uint32_t)fminf(q, 1048575.0f);
-      keys[k] = (Gq << 12) | (uint32_t)k;
     }
-    __syncwarp();
-    // the kNbrCap smallest keys in ascending order (keys are distinct: k is part of them)
+    __syncthreads();
+    // G(k0, k) for this thread's candidates: a row is fetched with independent 128-bit loads
+    for (int k = tid; k < Kpad; k += kGraphThreads) {
+      uint32_t key = kNbrEnd;                                  // padding up to a multiple of four
+      if (k < K) {
+        const float4* e = reinterpret_cast<const float4*>(cand_img + (size_t)k * D);
+        float4 row[D / 4];
+#pragma unroll
+        for (int q = 0; q < D / 4; ++q) row[q] = __ldg(e + q);
+        float sx = 0.0f, sy = 0.0f;
+#pragma unroll
+        for (int q = 0; q < D2 / 4; ++q) {
+          const float4 gx = *reinterpret_cast<const float4*>(&s_ref[4 * q]);
+          const float4 gy = *reinterpret_cast<const float4*>(&s_ref[D2 + 4 * q]);
+          const float4 ex = row[q], ey = row[D2 / 4 + q];
+          float t;
+          t = gx.x - ex.x; sx = fmaf(t, t, sx);
+          t = gx.y - ex.y; sx = fmaf(t, t, sx);
+          t = gx.z - ex.z; sx = fmaf(t, t, sx);
+          t = gx.w - ex.w; sx = fmaf(t, t, sx);
+          t = gy.x - ey.x; sy = fmaf(t, t, sy);
+          t = gy.y - ey.y; sy = fmaf(t, t, sy);
+          t = gy.z - ey.z; sy = fmaf(t, t, sy);
+          t = gy.w - ey.w; sy = fmaf(t, t, sy);
+        }
+        const float G = sqrtf(sx) + sqrtf(sy);
+        const float q = floorf(G * (65536.0f * (1.0f - 1.0f / 32768.0f)));
+        const uint32_t Gq = (uint32_t)fminf(q, 1048575.0f);
+        key = (Gq << 12) | (uint32_t)k;
+      }
+      s_keys[k] = key;
+    }
+    __syncthreads();
+    // the kNbrCap smallest keys in ascending order: a key's slot is the number of smaller keys (keys are distinct: k
+    // is part of them)
     uint32_t* out = nbr + ((size_t)b * K_max + k0) * kNbrCap;
-    uint32_t last = 0;
-    bool first = true;
-    for (int j = 0; j < kNbrCap; ++j) {
-      uint32_t m = kNbrEnd;
-      for (int k = lane; k < K; k += 32) {
-        const uint32_t v = keys[k];
-        if ((first || v > last) && v < m) m = v;
+    for (int k = tid; k < K; k += kGraphThreads) {
+      const uint32_t mine = s_keys[k];
+      int rank = 0;
+      for (int i = 0; i < Kpad; i += 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(&s_keys[i]);
+        rank += (v.x < mine) + (v.y < mine) + (v.z < mine) + (v.w < mine);
       }
-      m = __reduce_min_sync(0xffffffffu, m);
-      if (lane == 0) out[j] = m;
-      if (m == kNbrEnd) {          // fewer candidates than entries: the rest are end markers
-        for (int jj = j + 1 + lane; jj < kNbrCap; jj += 32) out[jj] = kNbrEnd;
-        break;
-      }
-      last = m;
-      first = false;
+      if (rank < kNbrCap) out[rank] = mine;
     }
-    __syncwarp();
+    for (int j = K + tid; j < kNbrCap; j += kGraphThreads) out[j] = kNbrEnd;   // fewer candidates than entries
+    __syncthreads();
   }
 }
 
