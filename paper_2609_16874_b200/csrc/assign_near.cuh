@@ -385,11 +385,12 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
         cell[j] = c4.x; cell[j + 1] = c4.y; cell[j + 2] = c4.z; cell[j + 3] = c4.w;
       }
     }
-    // bins -> peaks.  Pixels of one group nearly always share their peak; a group with several peaks keeps them per pixel.
+    // bins -> peaks.  Pixels of one group nearly always share their peak (ku); at an instance border there is a second
+    // one (kv); with more than two the group's pixels are left to the exact walk.
     int kpix[VEC];
     uint32_t voted = 0;                         // participating pixels that voted
-    bool uniform = true;
-    int ku = -1;
+    bool many = false;
+    int ku = -1, kv = -1;
     if (have) {
 #pragma unroll
       for (int j = 0; j < VEC; ++j) {
@@ -400,20 +401,26 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
           if (k >= K) k = -1;
           if (k >= 0) {
             if (ku < 0) ku = k;
-            else if (k != ku) uniform = false;
+            else if (k != ku) {
+              if (kv < 0) kv = k;
+              else if (k != kv) many = true;
+            }
           }
         }
         kpix[j] = k;
       }
     }
-    // the first two entries of the peaks' lists (one lookup for a uniform group)
-    uint2 e01u = make_uint2(0u, kNbrEnd);
+    if (many) ku = kv = -1;
+    // the first two entries of the peaks' lists
+    uint2 e01u = make_uint2(0u, kNbrEnd), e01v = make_uint2(0u, kNbrEnd);
     if (ku >= 0) e01u = __ldg(reinterpret_cast<const uint2*>(nbr_img + (size_t)ku * kNbrCap));
-    const int kfu = (int)(e01u.x & 0xfffu);
+    if (kv >= 0) e01v = __ldg(reinterpret_cast<const uint2*>(nbr_img + (size_t)kv * kNbrCap));
+    const int kfu = (int)(e01u.x & 0xfffu), kfv = (int)(e01v.x & 0xfffu);
 
-    __half2 s[H2], sc[H2];                      // sums of squares so far, two pixels each: reference rows, candidates
+    // sums of squares, two pixels per register: against the reference row and the first candidate of ku, and of kv
+    __half2 s[H2], sc[H2], sv[H2], scv[H2];
 #pragma unroll
-    for (int j = 0; j < H2; ++j) s[j] = sc[j] = __float2half2_rn(0.0f);
+    for (int j = 0; j < H2; ++j) s[j] = sc[j] = sv[j] = scv[j] = __float2half2_rn(0.0f);
     // widening-free view of one 128-bit load as pixel pairs
     auto pairs_of = [](const uint4& r, __half2 (&v)[H2]) {
       if constexpr (sizeof(T) == 2) {
@@ -425,13 +432,14 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
         v[1] = __floats2half2_rn(__uint_as_float(r.z), __uint_as_float(r.w));
       }
     };
-    if (ku >= 0 && uniform) {
-      // ---- the common case: one peak for the whole group, its row values splat over the pixel pairs
-      const __half* rr = rows_ref + (size_t)ku * D + axis * D2;
-      const __half* rc = rows_cand + (size_t)kfu * D + axis * D2;
+    // all pixels of the group against the rows of one peak (row values splat over the pixel pairs); `first`: the first
+    // batch of plane loads is already in `raw`
+    auto accumulate = [&](int kref, int kcand, __half2 (&acc)[H2], __half2 (&accc)[H2], bool first) {
+      const __half* rr = rows_ref + (size_t)kref * D + axis * D2;
+      const __half* rc = rows_cand + (size_t)kcand * D + axis * D2;
 #pragma unroll
       for (int l0 = 0; l0 < F; l0 += LB) {
-        if (l0 > 0) {
+        if (l0 > 0 || !first) {
 #pragma unroll
           for (int q = 0; q < 2 * LB; ++q)
             raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + q) * plane));
@@ -447,12 +455,12 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 #pragma unroll
           for (int j = 0; j < H2; ++j) {
             const __half2 d = __hsub2(v0[j], r_lo);
-            s[j] = __hfma2(d, d, s[j]);
+            acc[j] = __hfma2(d, d, acc[j]);
           }
 #pragma unroll
           for (int j = 0; j < H2; ++j) {
             const __half2 d = __hsub2(v1[j], r_hi);
-            s[j] = __hfma2(d, d, s[j]);
+            acc[j] = __hfma2(d, d, acc[j]);
           }
           if constexpr (!SAME) {
             const __half2 q2 = *reinterpret_cast<const __half2*>(rc + c);
@@ -460,52 +468,37 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 #pragma unroll
             for (int j = 0; j < H2; ++j) {
               const __half2 d = __hsub2(v0[j], q_lo);
-              sc[j] = __hfma2(d, d, sc[j]);
+              accc[j] = __hfma2(d, d, accc[j]);
             }
 #pragma unroll
             for (int j = 0; j < H2; ++j) {
               const __half2 d = __hsub2(v1[j], q_hi);
-              sc[j] = __hfma2(d, d, sc[j]);
+              accc[j] = __hfma2(d, d, accc[j]);
             }
           }
         }
       }
-    } else if (ku >= 0) {
-      // ---- a group with several peaks: every pixel against its own rows (rare: instance borders)
-      int kr[VEC], kc[VEC];
+    };
+    if (ku >= 0) accumulate(ku, kfu, s, sc, true);
+    if (kv >= 0) accumulate(kv, kfv, sv, scv, false);   // an instance border: the planes come from L1 this time
+    // swap with the partner lane: afterwards every lane has both axes' sums of its half of the pixels
+    // (all register-array indices below are compile-time constants: the axis picks between two of them)
+    // per pixel, pick the sums of its own peak first (register pairs hold two pixels: blend the halves)
+    {
+      uint32_t use_v = 0;
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) {
-        kr[j] = kpix[j] >= 0 ? kpix[j] : ku;
-        kc[j] = SAME ? kr[j] : (int)(__ldg(nbr_img + (size_t)kr[j] * kNbrCap) & 0xfffu);
-      }
-#pragma unroll 1
-      for (int l0 = 0; l0 < F; l0 += LB) {
-        if (l0 > 0) {
+      for (int j = 0; j < VEC; ++j)
+        if (kv >= 0 && kpix[j] == kv) use_v |= 1u << j;
+      if (use_v) {
 #pragma unroll
-          for (int q = 0; q < 2 * LB; ++q)
-            raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + q) * plane));
-        }
-#pragma unroll
-        for (int q = 0; q < 2 * LB; ++q) {
-          const int c = axis * D2 + 2 * l0 + q;
-          __half2 v[H2];
-          pairs_of(raw[q], v);
-#pragma unroll
-          for (int j = 0; j < H2; ++j) {
-            const __half2 r = __halves2half2(rows_ref[(size_t)kr[2 * j] * D + c], rows_ref[(size_t)kr[2 * j + 1] * D + c]);
-            const __half2 d = __hsub2(v[j], r);
-            s[j] = __hfma2(d, d, s[j]);
-            if constexpr (!SAME) {
-              const __half2 qq = __halves2half2(rows_cand[(size_t)kc[2 * j] * D + c], rows_cand[(size_t)kc[2 * j + 1] * D + c]);
-              const __half2 dc = __hsub2(v[j], qq);
-              sc[j] = __hfma2(dc, dc, sc[j]);
-            }
-          }
+        for (int j = 0; j < H2; ++j) {
+          const bool lo = (use_v >> (2 * j)) & 1u, hi = (use_v >> (2 * j + 1)) & 1u;
+          s[j] = __halves2half2(lo ? __low2half(sv[j]) : __low2half(s[j]), hi ? __high2half(sv[j]) : __high2half(s[j]));
+          if constexpr (!SAME)
+            sc[j] = __halves2half2(lo ? __low2half(scv[j]) : __low2half(sc[j]), hi ? __high2half(scv[j]) : __high2half(sc[j]));
         }
       }
     }
-    // swap with the partner lane: afterwards every lane has both axes' sums of its half of the pixels
-    // (all register-array indices below are compile-time constants: the axis picks between two of them)
     __half2 so[H2], sco[H2];
 #pragma unroll
     for (int j = 0; j < H2; ++j) {
@@ -541,8 +534,8 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
       if ((voted >> j) & 1u) {
         slow = true;
         bool likely_hard = k0j < 0;
-        if (k0j >= 0) {
-          const uint2 e01 = uniform ? e01u : __ldg(reinterpret_cast<const uint2*>(nbr_img + (size_t)k0j * kNbrCap));
+        if (k0j >= 0 && !many) {
+          const uint2 e01 = k0j == ku ? e01u : e01v;
           const int kfj = (int)(e01.x & 0xfffu);
           const float t = (fast_sqrt(sx) + fast_sqrt(sy)) * kHalfRel + kHalfAbs;
           const float dub = SAME ? t : (fast_sqrt(cx) + fast_sqrt(cy)) * kHalfRel + kHalfAbs;
