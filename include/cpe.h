@@ -74,12 +74,16 @@ enum {
   CPE_FLAG_MMA_ASSIGN = 256u,     /* filtered assignment: the mma.sync kernel for every image (comparisons)          */
   CPE_FLAG_NO_PRUNE = 512u,       /* do not prune the candidates of Eq. 7 (see cpe_decode): every image with more peaks
                                      than the all-pairs range goes to the tensor-core filtered kernels; same results  */
-  CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment for every image, however few peaks it has; same results    */
+  CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment for every image, however few peaks it has and however small
+                                     the input is; same results                                                       */
+  CPE_FLAG_PRUNE_ANY_SIZE = 8192u,/* the pruned assignment also for inputs of fewer than 2^19 pixels (by default those
+                                     go without it: its extra launches cost more than it saves there); same results    */
   CPE_FLAG_PRUNE_WALK_ONLY = 2048u, /* pruned assignment: the one-thread-per-pixel kernel also where the streaming kernel
                                        would run (tests, comparisons; same results)                                   */
-  CPE_FLAG_TEST_STALL = 4096u,    /* tests of the time-out path only: the pruned assignment's copy pipeline withholds
-                                     its first tile and waits briefly, so that a bounded wait runs out, the kernel
-                                     winds down and CPE_STATUS_TIMEOUT is set (the label map is then incomplete)      */
+  CPE_FLAG_TEST_STALL = 4096u,    /* tests of the time-out path only: the tensor-memory assignment's producer warps
+                                     withhold the arrival of each CTA's first tile, so that the consumers' bounded wait
+                                     runs out, the kernel winds down and returns, and CPE_STATUS_TIMEOUT is set (the
+                                     label map of that decode is incomplete)                                          */
   CPE_FLAG_REFINE = 16u       /* sub-cell refined centroids (an extension: the paper's candidates of Eq. 7 are the
                                  bin positions of Eq. 9, up to half a bin off the voted centroid).  Next to its
                                  count every bin keeps the sum of the estimates that fell into it, as integers
@@ -99,8 +103,8 @@ enum {
   CPE_STATUS_NONFINITE = 2u,     /* at least one participating pixel had a non-finite channel    */
   CPE_STATUS_INTERNAL = 4u,      /* an index self-check failed (site code in bits 8..15); the access was
                                     skipped.  Never set by a correct build: please report it.      */
-  CPE_STATUS_TIMEOUT = 8u        /* a bounded device-side wait (on an mbarrier of a copy or tensor-core pipeline)
-                                    ran out; the kernel wound down and returned, the image's outputs are
+  CPE_STATUS_TIMEOUT = 8u        /* a bounded device-side wait (on an mbarrier of the tensor-core pipeline) ran
+                                    out; the kernel wound down and returned, the image's label map is
                                     incomplete.  Never set by a correct build on a healthy GPU.    */
 };
 
@@ -293,7 +297,9 @@ void cpe_host_ctx_destroy(cpe_host_ctx* ctx);
  *     call returns CPE_ERR_STATIC_LIMIT and enqueues nothing.
  *   - The first call on a device, and any call whose sizes or parameters (B, F, bins, max_instances) differ
  *     from the previous call on that device, also sets the scratch up: it looks up the array's device address, uploads the palettes
- *     and waits for the stream.  Make such a call before starting a stream capture, not inside one.
+ *     and waits for the stream.  Make such a call before starting a stream capture: inside one it is refused with
+ *     CPE_ERR_PARAM and enqueues nothing (a call that needs no set-up only enqueues).  The device that owns
+ *     `stream` must be the current device.
  *   - All calls on a device share the one array, which keeps what the last call left in it; every call
  *     clears the parts that must start at zero.  Two calls that overlap on the GPU (different streams)
  *     would race on it: keep them on one stream, or order them yourself.

@@ -143,6 +143,9 @@ __device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
   asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" ::"r"(mbar) : "memory");
 }
+// A bounded wait ran out: reported in the image's status word; the caller winds its CTA down (abort flag) and returns.
+__device__ __forceinline__ void tc_timed_out(uint32_t* status) { atomicOr(status, (uint32_t)CPE_STATUS_TIMEOUT); }
+
 // Bounded wait for the phase of the given parity; gives up early once the CTA's abort flag is up.  False: gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, const volatile int* abort_flag) {
   for (int it = 0; it < kTcWaitLimit; ++it) {
@@ -382,7 +385,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
                  const float* __restrict__ peak_emb, const int32_t* __restrict__ count_ptr, float tau, int need_exact,
                  int peak_cap, int vec_mask, int32_t* __restrict__ labels, float* __restrict__ best,
                  float* __restrict__ second, uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all,
-                 uint32_t* __restrict__ votes, int cells, int k_min, int k_max, uint32_t* __restrict__ acc) {
+                 uint32_t* __restrict__ votes, int cells, int k_min, int k_max, uint32_t* __restrict__ acc, int test_stall) {
   constexpr int KS = KA / 16;                       // k-steps per axis
   constexpr int kTiles = tc_tiles(KA);              // tile buffers
   constexpr int kAhead = kTiles - 2;                // tiles whose copies are in flight while one is being completed
@@ -617,7 +620,9 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
       s_rcd[us * kTcRows + ptid] = cD;
       s_rflags[us * kTcRows + ptid] = flags;
       __syncwarp();
-      if (lane == 0) mbar_arrive(mb_meta + 8 * us);
+      // (`test_stall`, tests of the time-out path only: the first tile's arrival is withheld, so that the consumers'
+      // bounded wait for it runs out and the CTA winds down)
+      if (lane == 0 && !(test_stall && u == 0)) mbar_arrive(mb_meta + 8 * us);
     };
     // a new tile's copies go out, then the oldest tile in flight is completed once kAhead newer ones are on their way
     auto emit = [&](int ng) {
@@ -741,7 +746,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
     }
     if (bad || my_bad) {
       *s_abort = 1;
-      am_ok(false, 8u, status);
+      tc_timed_out(status);
     }
     asm volatile("cp.async.wait_all;\n" ::: "memory");
   } else {
@@ -812,7 +817,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
         const uint32_t old = atomicAdd(&s_relcnt[as], 1u);
         if ((old & 3u) == 3u && !issue_round(q + (both ? 1u : 2u))) {
           *s_abort = 1;
-          am_ok(false, 11u, status);
+          tc_timed_out(status);
         }
       }
       __syncwarp();
@@ -821,7 +826,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
     if (tid == 0) {
       if (!issue_round(0) || (!both && !issue_round(1))) {
         *s_abort = 1;
-        am_ok(false, 11u, status);
+        tc_timed_out(status);
       }
     }
     __syncwarp();
@@ -1037,7 +1042,7 @@ assign_tc_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW
     }
     if (bad) {
       *s_abort = 1;
-      am_ok(false, 10u, status);
+      tc_timed_out(status);
     }
     __syncwarp();
     if (lane == 0) {
@@ -1080,7 +1085,7 @@ assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, 
                      int tc_peak_cap, int tc_k_max, int tc_vec_mask, int mma_peak_cap, int mma_span, int mma_vec_mask,
                      int mma_vec_gather, int32_t* __restrict__ labels, float* __restrict__ best, float* __restrict__ second,
                      uint32_t* __restrict__ counters, uint32_t* __restrict__ status_all, uint32_t* __restrict__ votes, int cells,
-                     int k_min, uint32_t* __restrict__ acc, const uint32_t* __restrict__ near_state) {
+                     int k_min, uint32_t* __restrict__ acc, const uint32_t* __restrict__ near_state, int test_stall) {
   static_assert(kTcThreads == kAmThreads, "both bodies run with the same block size");
   grid_dependency_sync();
   // after the pruned assignment (near_state given) this kernel only takes the images which that one handed on
@@ -1090,7 +1095,7 @@ assign_filter_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, 
   }
   if (count_ptr[blockIdx.y] <= tc_k_max)
     assign_tc_body<T, KA, WANT2>(emb, fg, HW, F, K_max, peak_emb, count_ptr, tau, need_exact, tc_peak_cap, tc_vec_mask, labels,
-                                 best, second, counters, status_all, votes, cells, k_min, tc_k_max, acc);
+                                 best, second, counters, status_all, votes, cells, k_min, tc_k_max, acc, test_stall);
   else {
     // This kernel is one that uses tensor memory: a CTA that takes the other path gives up its right to allocate at
     // once, or the SM would not take a second CTA while this one runs.

@@ -231,9 +231,15 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
   if (sums && !sums_cleared_by_peaks) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
+  // From here on the vote map and the accumulators may hold this decode's votes.  If a later enqueue fails, the
+  // kernel that would have left them zero for the next decode never runs: clear them here instead.
+  auto fail_after_votes = [&](int code) {
+    cudaMemsetAsync(ws + L.acc, 0, L.votes_end - L.acc, st);
+    return code;
+  };
   rc = cpe::host::launch_decode_vote(st, emb, fg, B, HW, F, p, votes, acc, sums,
                                      L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr);
-  if (rc) return rc;
+  if (rc) return fail_after_votes(rc);
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_PEAKS], st));
@@ -244,13 +250,14 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     dim3 grid((unsigned)ctas, (unsigned)B);
     // one CTA per image: it works on a copy of the vote map in shared memory (at most 32 KB)
     const size_t map_smem = one_peak_cta ? 4 * (size_t)L.cells : 0;
-    CPE_CUDA(launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes, p->bins_w, p->bins_h, L.words,
-                              (uint32_t)p->vote_threshold, bitmap, p->max_instances, F, H, W, pal_w, pal_h, peak_cell,
-                              peak_votes, peak_emb, out_centroids, out_count, acc, counters, status, sums,
-                              sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0, refine ? 1 : 0,
-                              L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
-                              L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr, pr.near_state));
-    CPE_CUDA(cudaGetLastError());
+    cudaError_t e = launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes,
+                                     p->bins_w, p->bins_h, L.words, (uint32_t)p->vote_threshold, bitmap, p->max_instances, F,
+                                     H, W, pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids, out_count, acc,
+                                     counters, status, sums, sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0,
+                                     refine ? 1 : 0, L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
+                                     L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr, pr.near_state);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return fail_after_votes(cuda_fail(e));
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_LISTS], st));
@@ -261,7 +268,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
                                                   counters, status, votes_to_zero, L.cells, acc, prp, ev_lists)
                            : launch_assign<__half>(st, emb, fg, B, HW, F, p, peak_emb, out_count, out_labels, best,
                                                    second, counters, status, votes_to_zero, L.cells, acc, prp, ev_lists);
-  if (rc) return rc;
+  if (rc) return fail_after_votes(rc);
   if ((rc = debug_stage_check(st, "assign"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_N], st));
   return CPE_OK;
@@ -643,6 +650,11 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   char* ws = static_cast<char*>(slot.ptr);
   if (slot.F != F || slot.bins_w != p.bins_w || slot.bins_h != p.bins_h || slot.off_w != L.pal_w ||
       slot.off_h != L.pal_h) {
+    // the set-up copies from a host staging buffer and waits for the stream: impossible while the stream is being
+    // captured (the wait would invalidate the capture), so such a call is refused and enqueues nothing
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    CPE_CUDA(cudaStreamIsCapturing(st, &cs));
+    if (cs != cudaStreamCaptureStatusNone) return CPE_ERR_PARAM;
     // Eq. 9 positions through Eq. 2, in double, rounded once to binary32 (as cpe_init_workspace does)
     const double pi = 3.14159265358979323846;
     for (int axis = 0; axis < 2; ++axis) {

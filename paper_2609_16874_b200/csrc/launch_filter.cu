@@ -83,7 +83,7 @@ int launch_assign_filter_t(cudaStream_t st, const T* e, const uint8_t* fg, int B
   CPE_CUDA(launch_dependent(plain_launch(p), kern, grid, cpe::kTcThreads, smem, st, e, fg, HW, F, p->max_instances,
                             peak_emb, count, p->tau, need_exact, tc_cap, tc_k_max, vec_mask, mma_cap, span, vec_mask,
                             vec_gather, labels, best, second, counters, status, votes_to_zero, cells, k_min, acc,
-                            near_state));
+                            near_state, (p->flags & CPE_FLAG_TEST_STALL) ? 1 : 0));
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }

@@ -41,7 +41,8 @@ def test_params_struct_and_workspace_size():
     pp = cb.make_params(cb.CPE_F16, 256, 128)
     n_pruned = cb.cpe_workspace_size(1, 1024, 2048, 8, pp)
     assert n + 5 * 1024 * 2048 <= n_pruned < n + 5 * 1024 * 2048 + 4 * 1024 * 1024
-    # ... but not when no image can have more peaks than the all-pairs kernel takes
+    # ... but not when no image can have more peaks than the all-pairs kernel takes, nor on small inputs
+    assert cb.cpe_workspace_size(1, 512, 512, 8, pp) < 4 * 512 * 512
     assert cb.cpe_workspace_size(1, 1024, 2048, 8, cb.make_params(cb.CPE_F16, 256, 128, max_instances=32)) < n
     p2 = cb.make_params(cb.CPE_F16, 256, 128, flags=cb.CPE_FLAG_WRITE_SCORES | cb.CPE_FLAG_NO_PRUNE)
     assert cb.cpe_workspace_size(1, 1024, 2048, 8, p2) >= n + 2 * 4 * 1024 * 2048

@@ -73,6 +73,12 @@ def test_nonfinite_pixels_are_skipped_and_counted():
         pick = rng.choice(ys.size, 40, replace=False)
         for i, j in enumerate(pick):
             emb[0, rng.integers(0, cfg.D), ys[j], xs[j]] = [np.nan, np.inf, -np.inf][i % 3]
+        if dtype == "f32":
+            # a FINITE (sin, cos) pair whose |s| + |c| overflows binary32 counts as non-finite too (binary16 cannot hold one)
+            j = pick[0]
+            emb[0, :, ys[j], xs[j]] = fr["emb"][0, :, ys[j], xs[j]]
+            emb[0, 4, ys[j], xs[j]] = 2.5e38
+            emb[0, 5, ys[j], xs[j]] = -2.5e38
         gpu, ora, _ = check_case(emb, fr["fg"], cfg.bins_w, cfg.bins_h)
         assert gpu["counters"][0, cb.CPE_CNT_NONFINITE] == 40
         assert gpu["status"] & cb.CPE_STATUS_NONFINITE
@@ -300,6 +306,23 @@ def test_full_size_configs(name):
         assert lab.max() <= n and lab.min() >= 0
     assert gpu["status"] == 0
     print(f"{name}: peaks {ora['count'].tolist()}, sampled near-tie pixels {near}, excused label differences {excused}")
+    # the configuration the benchmark times -- no score output, vote map re-zeroed by the last kernel, graph replay --
+    # against the oracle's assignment of EVERY pixel (all host threads; a few seconds for c5)
+    fast = run_gpu(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, "graph", keep_votes=False)
+    compare_front(fast, ora, cfg.F, cfg.bins_w, cfg.bins_h)
+    assert fast["status"] == 0
+    oracle.set_threads(oracle.max_threads())
+    near = excused = 0
+    for b in range(cfg.B):
+        n = int(ora["count"][b])
+        res = oracle.assign_image(emb[b], fg[b], cfg.bins_w, cfg.bins_h, ora["peak_cell"][b, :n], cfg.tau)
+        rep = compare_labels(fast["labels"][b], None, None, res["labels"], res["best"], res["second"])
+        near += rep["near_tie_pixels"]
+        excused += rep["excused_mismatches"]
+    handed = None if fast["prune_state"] is None else fast["prune_state"][:, 2].tolist()
+    pairs = fast["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum() / max(1, fast["counters"][:, cb.CPE_CNT_VOTING].sum())
+    print(f"{name} (no scores, every pixel): near-tie pixels {near}, excused {excused}, handed on {handed}, "
+          f"scored pairs per voting pixel {pairs:.2f}")
 
 
 def test_tensor_memory_path_with_several_rounds_of_peaks():
@@ -324,6 +347,25 @@ def test_tensor_memory_path_with_several_rounds_of_peaks():
                 if scores:
                     assert np.array_equal(a["best"].view(np.uint32), b["best"].view(np.uint32))
                     assert np.array_equal(a["second"].view(np.uint32), b["second"].view(np.uint32))
+
+
+def test_mma_sync_body_as_the_c5_benchmark_instantiates_it():
+    """F = 16 binary16, more than 128 peaks, at least 2^20 pixels, no scores: the mma.sync body with 32 k-values per
+    axis, 16-byte gathers over the long span and the peak operand re-loaded in chunks (c5's 300 peaks do not fit the
+    resident operand) -- against the oracle's assignment of every pixel."""
+    cfg = wl.scaled(wl.CONFIGS["c5"], H=1024, W=1024, K=300, bins_w=512, bins_h=512)
+    fr = wl.make_frame(cfg, 0)
+    emb, fg = fr["emb"], fr["fg"]
+    ora = oracle.decode(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    assert ora["count"][0] > 246                                   # beyond the resident peak operand
+    for mode in ("direct", "graph"):
+        gpu = run_gpu(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, mode, keep_votes=False,
+                      flags=cb.CPE_FLAG_NO_PRUNE)
+        compare_front(gpu, ora, cfg.F, cfg.bins_w, cfg.bins_h)
+        assert gpu["status"] == 0
+        rep = compare_labels(gpu["labels"], None, None, ora["labels"], ora["best"], ora["second"])
+        assert gpu["counters"][0, cb.CPE_CNT_FILTER_PAIRS] > 0
+    print("c5-like, mma.sync body:", ora["count"].tolist(), rep)
 
 
 @pytest.mark.parametrize("name,over", [("c2", dict(H=384, W=384, K=90, bins_w=96, bins_h=96)),              # fp32, F = 8

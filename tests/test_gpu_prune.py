@@ -17,6 +17,7 @@ from gpu_util import compare_front, compare_labels, run_gpu
 pytestmark = pytest.mark.gpu
 
 PRUNE_ALL = cb.CPE_FLAG_PRUNE_ALL
+ANY_SIZE = cb.CPE_FLAG_PRUNE_ANY_SIZE     # the pruned assignment as the library chooses it, also on these small inputs
 
 
 def check_pruned(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, refine=False, flags=PRUNE_ALL, mode="direct",
@@ -30,9 +31,11 @@ def check_pruned(emb, fg, bins_w, bins_h, T_v=8, tau=np.inf, K_max=1024, refine=
     exact = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, 0, True, mode, exact_assign=True, refine=refine,
                     keep_votes=False)
     out = None
-    for scores in (True, False):
+    # with scores (the one-thread-per-pixel kernel), without (the streaming kernel where the shapes allow it, then the
+    # queue walk), and without scores on the one-thread-per-pixel kernel
+    for scores, extra in ((True, 0), (False, 0), (False, cb.CPE_FLAG_PRUNE_WALK_ONLY)):
         gpu = run_gpu(emb, fg, bins_w, bins_h, T_v, tau, K_max, 0, scores, mode, keep_votes=False, refine=refine,
-                      flags=flags)
+                      flags=flags | extra)
         assert not (gpu["status"] & cb.CPE_STATUS_INTERNAL), hex(gpu["status"])
         assert gpu["prune_state"] is not None, "the pruned assignment was not enabled"
         assert np.array_equal(gpu["count"], ora["count"])
@@ -82,7 +85,7 @@ def test_refined_candidates_leave_about_one_candidate_per_pixel():
     # other peak is excluded without being scored
     cfg = wl.scaled(wl.CONFIGS["c4"], B=2, H=320, W=384, K=100)
     fr = wl.make_frame(cfg, 0)
-    gpu, ora = check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=True, flags=0,
+    gpu, ora = check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=True, flags=ANY_SIZE,
                             expect_handed_on=[False, False])
     assert ora["count"].min() > 64                                   # more peaks than a list has entries
     # scores wanted: the walk goes on until the runner-up is settled too, i.e. up to G = (second-best distance) + t
@@ -90,7 +93,7 @@ def test_refined_candidates_leave_about_one_candidate_per_pixel():
     voting = gpu["counters"][:, cb.CPE_CNT_VOTING].sum()
     assert pairs <= 12 * voting, (pairs, voting)
     fast = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, keep_votes=False,
-                   refine=True)
+                   refine=True, flags=ANY_SIZE)
     pairs = fast["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum()
     assert pairs <= 2 * voting, (pairs, voting)
 
@@ -101,11 +104,11 @@ def test_aliased_grid_is_handed_to_the_filtered_kernel():
     # the same results
     cfg = wl.scaled(wl.CONFIGS["c5"], H=512, W=512, K=200, bins_w=256, bins_h=256)
     fr = wl.make_frame(cfg, 0)
-    gpu, ora = check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=False, flags=0,
+    gpu, ora = check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=False, flags=ANY_SIZE,
                             expect_handed_on=[True])
     assert ora["count"][0] > 64
     # ... and with refined candidates the same input stays with the pruned kernel
-    check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=True, flags=0,
+    check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, refine=True, flags=ANY_SIZE,
                  expect_handed_on=[False])
 
 
@@ -122,11 +125,11 @@ def _grid_instances(H, W, F, bw, bh, K, run, sigma, dtype, seed):
 def test_more_peaks_than_list_entries_and_more_than_the_lists_cover():
     # 600 peaks: lists hold the 64 nearest, alias-free grid (F = 4, 64 x 48 bins), so the bounds close every pixel
     emb, fg = _grid_instances(96, 128, 4, 64, 48, 600, 20, 0.02, np.float32, 5)
-    gpu, ora = check_pruned(emb, fg, 64, 48, T_v=8, K_max=1024, flags=0, expect_handed_on=[False])
+    gpu, ora = check_pruned(emb, fg, 64, 48, T_v=8, K_max=1024, flags=ANY_SIZE, expect_handed_on=[False])
     assert ora["count"][0] == 600
     # 1100 peaks: beyond what the list kernel serves, the image goes to the filtered kernel untouched
     emb, fg = _grid_instances(160, 160, 4, 96, 64, 1100, 20, 0.02, np.float16, 6)
-    gpu, ora = check_pruned(emb, fg, 96, 64, T_v=8, K_max=2048, flags=0, expect_handed_on=[True])
+    gpu, ora = check_pruned(emb, fg, 96, 64, T_v=8, K_max=2048, flags=ANY_SIZE, expect_handed_on=[True])
     assert ora["count"][0] == 1100
 
 
@@ -162,6 +165,6 @@ def test_pruned_assignment_edge_cases():
         e, _ = _grid_instances(H, W, F, bw, bh, K, 40, 0.03, np.float16, 20 + b)
         emb[b] = e[0]
         fg[b] = 1
-    gpu, ora = check_pruned(emb, fg, bw, bh, flags=0, expect_handed_on=[False, False, False])
+    gpu, ora = check_pruned(emb, fg, bw, bh, flags=ANY_SIZE, expect_handed_on=[False, False, False])
     assert ora["count"].tolist() == [0, 5, 60]
     assert gpu["prune_state"][2, 0] > 0 and gpu["prune_state"][1, 0] == 0      # only the third image was walked

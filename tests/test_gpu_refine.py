@@ -12,7 +12,7 @@ import oracle
 from paper_2609_16874_b200 import binding as cb
 from paper_2609_16874_b200 import workloads as wl
 
-from gpu_util import REL, compare_labels
+from gpu_util import REL, compare_labels, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -137,7 +137,7 @@ def test_refine_intermediate_needs_the_flag_and_workspace_grows_by_the_sums():
     assert rc == cb.CPE_ERR_WHICH
 
 
-@pytest.mark.parametrize("name", ["c2", "c3", "c5"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
 def test_refined_full_size_configs(name):
     """Full-size inputs, graph replay as the benchmark runs it: votes, per-bin sums, peak list, refined centroids and
     candidate embeddings against the full oracle; labels and scores on sampled pixels; label-map properties on all."""
@@ -150,7 +150,7 @@ def test_refined_full_size_configs(name):
     assert np.array_equal(gpu["votes"], ov["votes"])
     assert np.array_equal(gpu["sums"], sums)
     rng = np.random.default_rng(7)
-    n_sample = {"c2": 60000, "c3": 40000, "c5": 12000}[name]
+    n_sample = {"c2": 60000, "c3": 40000, "c4": 8000, "c5": 12000}[name]
     for b in range(cfg.B):
         cells, _, raw = oracle.peaks(ov["votes"][b], cfg.T_v, cfg.K_max)
         n = len(cells)
@@ -166,6 +166,20 @@ def test_refined_full_size_configs(name):
         assert ((lab > 0) == (fg[b] > 0)).all() and lab.max() <= n
         print(name, "peaks", n, rep)
     assert gpu["status"] == 0
+    # the configuration the benchmark times (no scores, vote map and sums re-zeroed on the device, graph replay) against
+    # the oracle's assignment of EVERY pixel
+    fast = run_gpu(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, "graph", keep_votes=False,
+                   refine=True)
+    assert fast["status"] == 0 and np.array_equal(fast["count"], gpu["count"])
+    oracle.set_threads(oracle.max_threads())
+    for b in range(cfg.B):
+        cells, _, raw = oracle.peaks(ov["votes"][b], cfg.T_v, cfg.K_max)
+        r = oracle.refined_peaks(ov["votes"][b], sums[b], cells, cfg.F, cfg.H, cfg.W)
+        res = oracle.assign_image(emb[b], fg[b], cfg.bins_w, cfg.bins_h, cells, cfg.tau, peak_emb=r["peak_emb"])
+        rep = compare_labels(fast["labels"][b], None, None, res["labels"], res["best"], res["second"])
+    handed = None if fast["prune_state"] is None else fast["prune_state"][:, 2].tolist()
+    pairs = fast["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum() / max(1, fast["counters"][:, cb.CPE_CNT_VOTING].sum())
+    print(f"{name} refined (no scores, every pixel): {rep}, handed on {handed}, scored pairs per voting pixel {pairs:.2f}")
 
 
 def test_refined_edge_cases_empty_truncated_nonfinite_and_border_peaks():

@@ -264,6 +264,30 @@ def test_votes_sum_mask_and_nonfinite_rules():
     assert res_all["votes"].sum() == cfg.H * cfg.W
 
 
+def test_a_finite_pair_whose_magnitudes_overflow_when_added_counts_as_non_finite():
+    """The usability rule of a (sin, cos) pair is "fl32(|s| + |c|) is finite": two finite binary32 values whose sum of
+    magnitudes overflows make the pixel unusable -- no vote, label 0, counted -- while either value alone (sum still
+    finite) is fine.  Pinned here against the rule's own statement: numpy's binary32 addition decides which is which."""
+    cfg = wl.scaled(wl.CONFIGS["c1"], H=40, W=56)
+    fr = wl.make_frame(cfg, 3)
+    emb, fg = fr["emb"].copy(), fr["fg"]
+    ys, xs = np.nonzero(fg[0])
+    big = np.float32(2.5e38)
+    with np.errstate(over="ignore"):
+        assert np.isfinite(big) and np.isinf(np.float32(big) + np.float32(big)) and np.isfinite(big + np.float32(1.0))
+    emb[0, 4, ys[0], xs[0]], emb[0, 5, ys[0], xs[0]] = big, -big      # harmonic 2 of x: |s| + |c| overflows
+    emb[0, 4, ys[1], xs[1]] = big                                     # the same magnitude alone: still usable
+    emb[0, 9, ys[2], xs[2]], emb[0, 10, ys[2], xs[2]] = big, big      # cos of one harmonic, sin of the next: different pairs
+    res = oracle.votes(emb, fg, cfg.bins_w, cfg.bins_h, want_cell=True)
+    assert res["counters"][0, oracle.CNT_NONFINITE] == 1
+    assert res["votes"].sum() == fg.sum() - 1
+    assert res["cell"][0, ys[0], xs[0]] == -1
+    assert res["cell"][0, ys[1], xs[1]] >= 0 and res["cell"][0, ys[2], xs[2]] >= 0
+    dec = oracle.decode(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    assert dec["labels"][0, ys[0], xs[0]] == 0 and np.isinf(dec["best"][0, ys[0], xs[0]])
+    assert dec["labels"][0, ys[1], xs[1]] > 0 and dec["labels"][0, ys[2], xs[2]] > 0
+
+
 def test_votes_fp16_equals_fp32_of_widened_values():
     cfg = wl.scaled(wl.CONFIGS["c3"], H=32, W=48, K=4, bins_w=32, bins_h=16)
     fr = wl.make_frame(cfg, 0)
