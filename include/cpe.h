@@ -137,10 +137,11 @@ enum {
   CPE_INT_VOTE_SUMS = 10,   /* int64  [B][bins_h][bins_w][2]    fixed-point (2^-24) sums of the x and y
                                                                 estimates per bin (CPE_FLAG_REFINE and
                                                                 CPE_FLAG_KEEP_VOTES)                 */
-  CPE_INT_PRUNE_STATE = 11, /* uint32 [B][8]  the pruned assignment's words of each image (only when it is enabled):
+  CPE_INT_PRUNE_STATE = 11, /* uint32 [B][12] the pruned assignment's words of each image (only when it is enabled):
                                                 [0] pixels visited, [1] pixels whose candidate list did not settle them,
                                                 [2] non-zero: the image was handed to the tensor-core filtered kernel,
-                                                [4..7] that kernel's own counters (folded into CPE_INT_COUNTERS)  */
+                                                [3] pixels queued for the exact walk, [4..7] its own counters (folded
+                                                into CPE_INT_COUNTERS), [8] pixels queued for the scan of every peak */
   CPE_INT_N = 12
 };
 

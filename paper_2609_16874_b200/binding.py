@@ -372,7 +372,7 @@ class Decoder:
             CPE_INT_STATUS: (torch.int32, (self.B,)),
             CPE_INT_COUNTERS: (torch.int32, (self.B, CPE_CNT_N)),
             CPE_INT_VOTE_SUMS: (torch.int64, (self.B, bh, bw, 2)),
-            CPE_INT_PRUNE_STATE: (torch.int32, (self.B, 8)),
+            CPE_INT_PRUNE_STATE: (torch.int32, (self.B, 12)),
         }
         dt, shape = shapes[which]
         return raw.view(dt).view(shape)

@@ -31,6 +31,7 @@ namespace cpe {
 
 constexpr int kNearThreads = 256;
 constexpr float kNearSlack = 1.00002f;
+constexpr int kNearWalkMax = 12;     // list entries one thread walks before the pixel goes to the warp-wide scan
 
 // The walk of one pixel, given its 4F values as (x channel c, y channel c) pairs.
 template <int D, bool WANT2>
@@ -43,7 +44,8 @@ __device__ __forceinline__ void near_walk(const float2 (&e2)[D / 2], int k0, int
   const uint32_t* list = nbr_img + (size_t)k0 * kNbrCap;
   float bound2 = inf;
   int j = 0;
-  for (; j < kNbrCap; ++j) {
+  constexpr int kWalkMax = WANT2 ? kNbrCap : kNearWalkMax;       // (the runner-up alone needs a longer walk)
+  for (; j < kNbrCap && j < kWalkMax; ++j) {
     const uint32_t ent = __ldg(list + j);
     if (ent == kNbrEnd) break;                                   // every candidate of the image has been seen
     const float G = (float)(ent >> 12) * (1.0f / 65536.0f);
@@ -59,7 +61,10 @@ __device__ __forceinline__ void near_walk(const float2 (&e2)[D / 2], int k0, int
     const float bound = WANT2 ? d2 : d1;
     bound2 = bound * bound * (1.0f + 1e-6f);
   }
-  hard = (j == kNbrCap) && K > kNbrCap;                          // the list ran out before the bound closed it
+  // the list ran out before the bound closed it, or the walk is getting long: a thread's walk is a chain of dependent
+  // row fetches, and a pixel far from its reference point (large t) would go through most of the list that way -- it
+  // is handed to the warp-wide scan instead
+  hard = (j == kNbrCap && K > kNbrCap) || (!WANT2 && j == kWalkMax);
 }
 
 // Every peak, in ascending k (a hard pixel).
@@ -599,7 +604,8 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
                         const float* __restrict__ cand2, const uint32_t* __restrict__ nbr,
                         const int32_t* __restrict__ cell_peak, const uint32_t* __restrict__ pix_cell, int cells,
                         const int32_t* __restrict__ count_ptr, float tau, int32_t* __restrict__ labels,
-                        uint32_t* __restrict__ near_state, const uint32_t* __restrict__ slow_q, int q_cap, int k_min) {
+                        uint32_t* __restrict__ near_state, const uint32_t* __restrict__ slow_q,
+                        uint32_t* __restrict__ hard_q, int q_cap, int k_min) {
   grid_dependency_sync();
   constexpr int D = 4 * FT;
   const int b = blockIdx.y;
@@ -641,24 +647,18 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
         near_walk<D, false>(e2, k0, K, same_rows, ref_img, cand_img, nbr_img, d1, d2, k1, hard, scored);
       }
     }
-    // hard pixels: every peak, by the whole warp, one pixel after the other
-    uint32_t hm = __ballot_sync(0xffffffffu, hard);
-    while (hm) {
-      const int src_lane = __ffs(hm) - 1;
-      hm &= hm - 1;
-      const unsigned long long pp = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)p, src_lane);
-      float w1, w2;
-      int wk;
-      near_full_scan_warp<T, D, false>(reinterpret_cast<const T*>((uintptr_t)pp), plane, K, cand_img, w1, w2, wk);
-      if (lane == src_lane) {
-        d1 = w1;
-        k1 = wk;
-        scored = (uint32_t)K;
-        ++n_full;
-      }
+    // hard pixels (no peak for the bin, list run out, long walk): every peak has to be scored, which a warp does
+    // together.  They come in runs (an instance without a peak of its own), so they go to a second queue from which
+    // assign_near_hard_kernel deals them out one per warp, instead of being done here, a run at a time by one warp.
+    const uint32_t hm = __ballot_sync(0xffffffffu, hard);
+    if (hm) {
+      uint32_t hbase = 0;
+      if (lane == 0) hbase = atomicAdd(&state[kNearHardQueue], (uint32_t)__popc(hm));
+      hbase = __shfl_sync(0xffffffffu, hbase, 0);
+      if (hard) hard_q[(size_t)b * q_cap + hbase + (uint32_t)__popc(hm & ((1u << lane) - 1u))] = (uint32_t)n;
     }
-    if (have) {
-      if (!hard && scored > 1) ++n_multi;
+    if (have && !hard) {
+      if (scored > 1) ++n_multi;
       n_pairs += scored;
       int label = 0;
       if (k1 >= 0) {
@@ -669,6 +669,44 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
     }
   }
   near_flush_counters(state, n_rejected, n_pairs, n_multi, n_full);
+}
+
+// The pixels that the walk left over: every peak, one warp per pixel (near_full_scan_warp), the queue dealt out
+// warp by warp so that a run of such pixels spreads over the whole grid.
+template <typename T, int FT>
+__global__ void __launch_bounds__(kNearThreads)
+assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const float* __restrict__ cand2,
+                        const int32_t* __restrict__ count_ptr, float tau, int32_t* __restrict__ labels,
+                        uint32_t* __restrict__ near_state, const uint32_t* __restrict__ hard_q, int q_cap, int k_min) {
+  grid_dependency_sync();
+  constexpr int D = 4 * FT;
+  const int b = blockIdx.y;
+  const size_t plane = (size_t)HW;
+  const int K = count_ptr[b];
+  if (K < k_min || K > kNearMaxPeaks) return;
+  uint32_t* state = near_state + b * kNearStride;
+  if (state[kNearGiveUp]) return;                // the filtered kernel redoes the whole image
+  const int n_h = (int)min(state[kNearHardQueue], (uint32_t)q_cap);
+  const float* cand_img = cand2 + (size_t)b * K_max * D;
+  const int lane = threadIdx.x & 31;
+  const int warp = blockIdx.x * (kNearThreads / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (kNearThreads / 32);
+  uint32_t n_rejected = 0, n_full = 0;
+  for (int i = warp; i < n_h; i += n_warps) {
+    const size_t n = hard_q[(size_t)b * q_cap + i];
+    float d1, d2;
+    int k1;
+    near_full_scan_warp<T, D, false>(emb + (size_t)b * D * plane + n, plane, K, cand_img, d1, d2, k1);
+    if (lane == 0) {
+      ++n_full;
+      int label = 0;
+      if (k1 >= 0) {
+        if (d1 < tau) label = k1 + 1;
+        else ++n_rejected;
+      }
+      labels[(size_t)b * plane + n] = label;
+    }
+  }
+  near_flush_counters(state, n_rejected, n_full * (uint32_t)K, 0u, n_full);
 }
 
 }  // namespace cpe

@@ -112,6 +112,7 @@ struct PruneArgs {
   int q_cap = 0;
   void* ref_h = nullptr;
   void* cand_h = nullptr;
+  uint32_t* hard_q = nullptr;
 };
 
 // Stage 4+5.  The number of peaks is only known on the device, so several kernels are enqueued and every image is
@@ -148,7 +149,8 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   if (pr) {
     rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref_emb, peak_emb, pr->ref2, pr->cand2, pr->nbr,
                                        pr->cell_peak, pr->pix_cell, cells, count, labels, best, second, pr->near_state,
-                                       k_limit + 1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h);
+                                       k_limit + 1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h,
+                                       pr->hard_q);
     if (rc) return rc;
   }
   // (also with a limit of 0: an image without any peak still gets its all-zero label map from this kernel)
@@ -223,6 +225,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     pr.near_state = reinterpret_cast<uint32_t*>(ws + L.near_state);
     pr.slow_q = reinterpret_cast<uint32_t*>(ws + L.slow_q);
     pr.q_cap = L.q_cap;
+    pr.hard_q = reinterpret_cast<uint32_t*>(ws + L.hard_q);
     pr.ref_h = ws + L.ref_h;
     pr.cand_h = ws + L.cand_h;
   }

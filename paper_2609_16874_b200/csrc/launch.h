@@ -76,7 +76,8 @@ int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                        const float* ref_emb, const float* cand_emb, const float* ref2, const float* cand2,
                        const uint32_t* nbr, const int32_t* cell_peak, const uint32_t* pix_cell, int cells,
                        const int32_t* count, int32_t* labels, float* best, float* second, uint32_t* near_state, int k_min,
-                       uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h);
+                       uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h,
+                       uint32_t* hard_q);
 
 // ---- second vote mode (launch_soft.cu)
 int launch_soft_votes(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,

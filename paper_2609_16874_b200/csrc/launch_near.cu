@@ -51,6 +51,7 @@ struct NearArgs {
   int q_cap;
   uint32_t* status;
   const void *ref_h, *cand_h;
+  uint32_t* hard_q;
 };
 
 template <typename T, int FT, bool WANT2>
@@ -90,11 +91,20 @@ int launch_stream_t(cudaStream_t st, const NearArgs& a) {
                             smem));
   CPE_CUDA(cudaGetLastError());
   // the pixels it queued
-  const long long walk_ctas = std::max(1, (2 * sm_count() + a.B - 1) / a.B);
+  const long long walk_ctas = std::max(1, ((FT == 16 ? 2 : 3) * sm_count() + a.B - 1) / a.B);
   dim3 wgrid((unsigned)std::min<long long>(walk_ctas, (a.q_cap + cpe::kNearThreads - 1) / cpe::kNearThreads), (unsigned)a.B);
   CPE_CUDA(launch_dependent(plain_launch(a.p), cpe::assign_near_walk_kernel<T, FT>, wgrid, cpe::kNearThreads, 0, st,
                             static_cast<const T*>(a.emb), a.HW, a.p->max_instances, a.ref2, a.cand2, a.nbr, a.cell_peak,
-                            a.pix_cell, a.cells, a.count, a.p->tau, a.labels, a.near_state, a.slow_q, a.q_cap, a.k_min));
+                            a.pix_cell, a.cells, a.count, a.p->tau, a.labels, a.near_state, a.slow_q, a.hard_q, a.q_cap,
+                            a.k_min));
+  CPE_CUDA(cudaGetLastError());
+  // ... and the pixels that the walk left to the scan of every peak, one warp each
+  // (a pixel keeps its warp for a few microseconds of dependent fetches: as many warps as the SMs hold)
+  const long long hard_ctas = std::max(1, (8 * sm_count() + a.B - 1) / a.B);
+  dim3 hgrid((unsigned)std::min<long long>(hard_ctas, (a.q_cap + 7) / 8), (unsigned)a.B);
+  CPE_CUDA(launch_dependent(plain_launch(a.p), cpe::assign_near_hard_kernel<T, FT>, hgrid, cpe::kNearThreads, 0, st,
+                            static_cast<const T*>(a.emb), a.HW, a.p->max_instances, a.cand2, a.count, a.p->tau, a.labels,
+                            a.near_state, a.hard_q, a.q_cap, a.k_min));
   CPE_CUDA(cudaGetLastError());
   return CPE_OK;
 }
@@ -127,9 +137,10 @@ int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                        const float* ref_emb, const float* cand_emb, const float* ref2, const float* cand2,
                        const uint32_t* nbr, const int32_t* cell_peak, const uint32_t* pix_cell, int cells,
                        const int32_t* count, int32_t* labels, float* best, float* second, uint32_t* near_state, int k_min,
-                       uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h) {
+                       uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h,
+                       uint32_t* hard_q) {
   const NearArgs a{emb, fg, B, HW, p, ref_emb, cand_emb, ref2, cand2, nbr, cell_peak, pix_cell, cells, count, labels, best,
-                   second, near_state, k_min, slow_q, q_cap, status, ref_h, cand_h};
+                   second, near_state, k_min, slow_q, q_cap, status, ref_h, cand_h, hard_q};
   return p->dtype == CPE_F32 ? launch_near_f<float>(st, F, a) : launch_near_f<__half>(st, F, a);
 }
 

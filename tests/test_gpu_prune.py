@@ -94,8 +94,10 @@ def test_refined_candidates_leave_about_one_candidate_per_pixel():
     assert pairs <= 12 * voting, (pairs, voting)
     fast = run_gpu(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, False, keep_votes=False,
                    refine=True, flags=ANY_SIZE)
+    # (every peak is scored for the few pixels whose instance has no peak of its own: they are far from any reference)
     pairs = fast["counters"][:, cb.CPE_CNT_FILTER_PAIRS].sum()
-    assert pairs <= 2 * voting, (pairs, voting)
+    full = fast["counters"][:, cb.CPE_CNT_FULL_SCORED].sum()
+    assert pairs - full * int(ora["count"].max()) <= 2 * voting, (pairs, full, voting)
 
 
 def test_aliased_grid_is_handed_to_the_filtered_kernel():
