@@ -64,6 +64,8 @@ def _load():
         lib.cpe_oracle_votes.restype = c_int
         lib.cpe_oracle_peaks.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp, vp]
         lib.cpe_oracle_peaks.restype = c_int
+        lib.cpe_oracle_real_peaks.argtypes = [vp, c_int, c_int, c_dbl, c_int, vp, vp]
+        lib.cpe_oracle_real_peaks.restype = c_int
         lib.cpe_oracle_centroid_px.argtypes = [c_int] * 6 + [vp]
         lib.cpe_oracle_centroid_px.restype = None
         lib.cpe_oracle_assign_image.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, vp, c_int, vp, c_int,
@@ -174,6 +176,41 @@ def peaks(V: np.ndarray, T_v: int, K_max: int):
     raw = np.zeros(1, np.int32)
     kept = _load().cpe_oracle_peaks(_ptr(V), bw, bh, T_v, K_max, _ptr(cells), _ptr(pv), _ptr(raw))
     return cells[:kept].copy(), pv[:kept].copy(), int(raw[0])
+
+
+def real_peaks(Hmap: np.ndarray, threshold: float, K_max: int):
+    """The paper's literal local-maxima search on ONE real-valued map ``[bins_h, bins_w]``: (cells ascending, raw count)."""
+    Hmap = np.ascontiguousarray(Hmap, np.float64)
+    bh, bw = Hmap.shape
+    cells = np.full(K_max, -1, np.int32)
+    raw = np.zeros(1, np.int32)
+    kept = _load().cpe_oracle_real_peaks(_ptr(Hmap), bw, bh, float(threshold), K_max, _ptr(cells), _ptr(raw))
+    return cells[:kept].copy(), int(raw[0])
+
+
+def decode_soft(emb: np.ndarray, fg, bins_w: int, bins_h: int, threshold: float, tau=np.inf, K_max: int = 1024):
+    """The paper's own chain: soft-vote histogram (Eq. 6), strict local maxima above ``threshold`` (Sec. 3.2),
+    assignment to the peaks' palette rows (Eq. 7-8).  Returns the histogram, the peak lists and the label maps."""
+    emb = np.ascontiguousarray(emb)
+    B, D, H, W = emb.shape
+    Hmap = soft_votes(emb, fg, bins_w, bins_h)
+    labels = np.empty((B, H, W), np.int32)
+    best = np.empty((B, H, W), np.float64)
+    second = np.empty((B, H, W), np.float64)
+    pc_all = np.full((B, K_max), -1, np.int32)
+    count = np.zeros(B, np.int32)
+    centroids = np.full((B, K_max, 2), np.nan, np.float32)
+    for b in range(B):
+        pc, raw = real_peaks(Hmap[b], threshold, K_max)
+        a = assign_image(emb[b], None if fg is None else fg[b], bins_w, bins_h, pc, tau)
+        k = pc.shape[0]
+        count[b] = k
+        pc_all[b, :k] = pc
+        for i, lin in enumerate(pc):
+            centroids[b, i] = centroid_px(lin % bins_w, lin // bins_w, bins_w, bins_h, H, W)
+        labels[b], best[b], second[b] = a["labels"], a["best"], a["second"]
+    return {"hist": Hmap, "labels": labels, "best": best, "second": second, "peak_cell": pc_all, "count": count,
+            "centroids": centroids}
 
 
 def centroid_px(cx: int, cy: int, bins_w: int, bins_h: int, H: int, W: int):

@@ -282,6 +282,37 @@ int cpe_oracle_peaks(const uint32_t* V, int bins_w, int bins_h, int T_v, int K_m
   return kept;
 }
 
+/*
+ * The local-maxima search as the paper prints it, on a real-valued map H (Sec. 3.2, "Local Maxima Search"): a bin
+ * is a candidate centroid iff its value exceeds the threshold and is a STRICT maximum of its 8-connected
+ * neighbourhood (neighbours outside the map do not exist).  Two equal neighbours are both rejected: the printed
+ * test has no tie rule and real-valued sums do not tie.  Peaks are listed by ascending linear index, at most K_max.
+ */
+int cpe_oracle_real_peaks(const double* Hmap, int bins_w, int bins_h, double threshold, int K_max, int32_t* peak_cell,
+                          int32_t* raw_count) {
+  int kept = 0, raw = 0;
+  for (int cy = 0; cy < bins_h; ++cy)
+    for (int cx = 0; cx < bins_w; ++cx) {
+      const int lin = cy * bins_w + cx;
+      const double v = Hmap[lin];
+      if (!(v > threshold)) continue;
+      int is_peak = 1;
+      for (int dy = -1; dy <= 1 && is_peak; ++dy)
+        for (int dx = -1; dx <= 1; ++dx) {
+          if (!dx && !dy) continue;
+          const int ny = cy + dy, nx = cx + dx;
+          if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+          if (!(v > Hmap[ny * bins_w + nx])) { is_peak = 0; break; }
+        }
+      if (!is_peak) continue;
+      if (kept < K_max && peak_cell) peak_cell[kept] = lin;
+      if (kept < K_max) ++kept;
+      ++raw;
+    }
+  if (raw_count) *raw_count = raw;
+  return kept;
+}
+
 /* O5: pixel-unit centre of bin (cx, cy): normalised x = -1 + (2 col + 1)/W  <=>  col = ((x+1) W - 1)/2. */
 void cpe_oracle_centroid_px(int cx, int cy, int bins_w, int bins_h, int H, int W, float* out_xy) {
   double x = bin_position(bins_w, cx + 1), y = bin_position(bins_h, cy + 1);

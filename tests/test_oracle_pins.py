@@ -721,3 +721,66 @@ def test_explicit_candidates_reduce_to_the_palette_case_and_to_brute_force():
          np.sqrt(((x[:, None, 2 * F:] - rows2[None, :, 2 * F:].astype(np.float64)) ** 2).sum(-1)))
     assert np.array_equal(a2["labels"].ravel(), d.argmin(1) + 1)
     np.testing.assert_allclose(a2["best"].ravel(), d.min(1), rtol=1e-12)
+
+
+# ---------------------------------------------------------------- the paper's literal local-maxima search on a real-valued map
+
+def test_real_peaks_equal_the_library_maximum_filter_and_a_brute_force():
+    """Strict 8-neighbour maxima above a threshold (Sec. 3.2): against scipy's maximum filter on maps of distinct values
+    (a bin is a strict maximum iff it equals the 3x3 maximum and no neighbour does), and against a differently written
+    brute force; border bins have fewer neighbours; equal neighbours are both rejected; truncation keeps the first K."""
+    from scipy import ndimage
+    rng = np.random.default_rng(21)
+    for shape in ((1, 1), (1, 7), (6, 1), (5, 8), (17, 13)):
+        Hm = rng.random(shape) * 10.0                           # distinct with probability 1
+        thr = 3.0
+        cells, raw = oracle.real_peaks(Hm, thr, 10_000)
+        mx = ndimage.maximum_filter(Hm, size=3, mode="constant", cval=-np.inf)
+        want = np.flatnonzero(((Hm == mx) & (Hm > thr)).ravel())
+        assert np.array_equal(cells, want) and raw == want.size, shape
+        brute = []
+        bh, bw = shape
+        for lin in range(bh * bw):
+            cy, cx = divmod(lin, bw)
+            nb = [Hm[y, x] for y in range(max(0, cy - 1), min(bh, cy + 2)) for x in range(max(0, cx - 1), min(bw, cx + 2))
+                  if (y, x) != (cy, cx)]
+            if Hm[cy, cx] > thr and all(Hm[cy, cx] > v for v in nb):
+                brute.append(lin)
+        assert cells.tolist() == brute
+        if len(brute) > 2:
+            first, raw2 = oracle.real_peaks(Hm, thr, 2)
+            assert first.tolist() == brute[:2] and raw2 == len(brute)
+    # hand cases: a plateau of two equal bins yields no peak (the literal test; the integer map's tie rule is an extension)
+    Hm = np.zeros((4, 5))
+    Hm[1, 1] = Hm[1, 2] = 5.0
+    Hm[3, 4] = 2.0                                               # a corner bin
+    cells, raw = oracle.real_peaks(Hm, 1.0, 16)
+    assert cells.tolist() == [3 * 5 + 4] and raw == 1
+    cells, _ = oracle.real_peaks(Hm, 2.0, 16)                    # the threshold is strict
+    assert cells.tolist() == []
+
+
+def test_soft_vote_chain_finds_the_instances_of_clean_encodings():
+    """Eq. 6 -> local maxima -> Eq. 7 on an alias-free grid (L = 4, 32 bins: the paper's setting) with noise-free
+    encodings of centroids on bin positions: the peaks are exactly the centroids' bins and the labels the instances."""
+    H, W, F, bw, bh = 48, 64, 4, 32, 32
+    inst = np.zeros((H, W), np.int32)
+    inst[2:20, 3:30] = 1
+    inst[24:46, 5:25] = 2
+    inst[10:40, 36:60] = 3
+    bins = [(6, 5), (9, 22), (25, 14)]
+    cents = np.array([[-1 + 2 * (cx + 1) / (bw + 1), -1 + 2 * (cy + 1) / (bh + 1)] for cx, cy in bins])
+    emb = wl.encode(inst, cents, F, 0.0, None, np.float32)[None]
+    fg = (inst > 0).astype(np.uint8)[None]
+    # side lobes of the sinusoidal kernel reach a quarter of a main lobe here (the largest is 121 against 451..725):
+    # the threshold separates them, as the paper's does
+    res = oracle.decode_soft(emb, fg, bw, bh, threshold=200.0)
+    assert res["count"][0] == 3
+    assert res["peak_cell"][0, :3].tolist() == sorted(cy * bw + cx for cx, cy in bins)
+    order = np.argsort([cy * bw + cx for cx, cy in bins])
+    relabel = np.zeros(4, np.int32)
+    relabel[1 + order] = 1 + np.arange(3)
+    assert np.array_equal(res["labels"][0], relabel[inst])
+    # the histogram's value at an instance's own bin: its pixels contribute exp(-0) = 1 each, the others less
+    for (cx, cy), area in zip(bins, [(inst == i).sum() for i in (1, 2, 3)]):
+        assert area <= res["hist"][0, cy, cx] < area + (fg.sum() - area) * np.exp(-0.3)
