@@ -84,6 +84,16 @@ enum {
                                      withhold the arrival of each CTA's first tile, so that the consumers' bounded wait
                                      runs out, the kernel winds down and returns, and CPE_STATUS_TIMEOUT is set (the
                                      label map of that decode is incomplete)                                          */
+  CPE_FLAG_SOFT_VOTE = 16384u,    /* vote as the paper prints it: the map is the real-valued histogram of Eq. 6,
+                                     H(a, b) = sum over the participating pixels of exp(-d) with d of Eq. 4 (the sum
+                                     that cpe_soft_votes computes, same accuracy), instead of the integer counts of the
+                                     hard vote.  A bin is a candidate centroid iff H > soft_threshold and H exceeds
+                                     each existing 8-neighbour STRICTLY (Sec. 3.2 as printed: no tie rule; equal
+                                     neighbours are both rejected).  Assignment, outputs and counters are as usual;
+                                     CPE_INT_VOTES and CPE_INT_PEAK_VOTES then hold binary32 values of H;
+                                     vote_threshold and levels are ignored.  Needs emb 16-byte aligned and H*W a
+                                     multiple of 8; not combinable with CPE_FLAG_REFINE (CPE_ERR_PARAM).  The candidates
+                                     are never pruned in this mode.                                                   */
   CPE_FLAG_REFINE = 16u       /* sub-cell refined centroids (an extension: the paper's candidates of Eq. 7 are the
                                  bin positions of Eq. 9, up to half a bin off the voted centroid).  Next to its
                                  count every bin keeps the sum of the estimates that fell into it, as integers
@@ -166,6 +176,8 @@ typedef struct cpe_params {
                               (16 when F > 8) the decode enqueues one kernel fewer: no image can
                               then need the tensor-core assignment.                            */
   uint32_t flags;          /* CPE_FLAG_*                                                       */
+  float soft_threshold;    /* with CPE_FLAG_SOFT_VOTE: a peak needs H > soft_threshold (finite, >= 0);
+                              ignored otherwise                                                 */
   void* workspace;         /* device memory, 256-byte aligned, owned by the caller             */
   size_t workspace_bytes;  /* >= cpe_workspace_size(...) for the same B, H, W, F and params    */
 } cpe_params;

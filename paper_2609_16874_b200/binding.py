@@ -37,6 +37,7 @@ CPE_FLAG_PRUNE_ALL = 1024
 CPE_FLAG_PRUNE_WALK_ONLY = 2048
 CPE_FLAG_TEST_STALL = 4096
 CPE_FLAG_PRUNE_ANY_SIZE = 8192
+CPE_FLAG_SOFT_VOTE = 16384
 CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL, CPE_STATUS_TIMEOUT = 1, 2, 4, 8
 CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
 CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8
@@ -66,6 +67,7 @@ class cpe_params(ctypes.Structure):
         ("tau", ctypes.c_float),
         ("max_instances", ctypes.c_int32),
         ("flags", ctypes.c_uint32),
+        ("soft_threshold", ctypes.c_float),
         ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t),
     ]
@@ -149,9 +151,10 @@ def load() -> ctypes.CDLL:
 
 
 def make_params(dtype: int, bins_w: int, bins_h: int, levels: int = 0, vote_threshold: int = 8, tau: float = math.inf,
-                max_instances: int = 1024, flags: int = 0, workspace: int = 0, workspace_bytes: int = 0) -> cpe_params:
+                max_instances: int = 1024, flags: int = 0, workspace: int = 0, workspace_bytes: int = 0,
+                soft_threshold: float = 0.0) -> cpe_params:
     return cpe_params(ctypes.sizeof(cpe_params), dtype, bins_w, bins_h, levels, vote_threshold, tau, max_instances,
-                      flags, workspace or None, workspace_bytes)
+                      flags, soft_threshold, workspace or None, workspace_bytes)
 
 
 # ---- the C entry points, same names, integer pointers
@@ -270,7 +273,7 @@ class Decoder:
 
     def __init__(self, B, H, W, F, dtype, bins_w, bins_h, vote_threshold=8, tau=math.inf, max_instances=1024,
                  levels=0, write_scores=False, device="cuda:0", exact_assign=False, keep_votes=False, filter_assign=False,
-                 refine=False, flags=0):
+                 refine=False, flags=0, soft_threshold=None):
         import torch
         self.torch = torch
         self.B, self.H, self.W, self.F = B, H, W, F
@@ -279,8 +282,10 @@ class Decoder:
         self.emb_dtype = torch.float32 if code == CPE_F32 else torch.float16
         flags = ((CPE_FLAG_WRITE_SCORES if write_scores else 0) | (CPE_FLAG_EXACT_ASSIGN if exact_assign else 0) |
                  (CPE_FLAG_KEEP_VOTES if keep_votes else 0) | (CPE_FLAG_FILTER_ASSIGN if filter_assign else 0) |
-                 (CPE_FLAG_REFINE if refine else 0) | int(flags))
-        self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances, flags)
+                 (CPE_FLAG_REFINE if refine else 0) | (CPE_FLAG_SOFT_VOTE if soft_threshold is not None else 0) |
+                 int(flags))
+        self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances, flags,
+                                  soft_threshold=float(soft_threshold or 0.0))
         n = cpe_workspace_size(B, H, W, F, self.params)
         if n == 0:
             raise CpeError(CPE_ERR_SIZE, "cpe_workspace_size")
@@ -393,10 +398,12 @@ class HostDecoder:
     """End-to-end front end for host buffers (``cpe_host_ctx_*``): numpy in, numpy out, copies included."""
 
     def __init__(self, B, H, W, F, dtype, bins_w, bins_h, vote_threshold=8, tau=math.inf, max_instances=1024,
-                 levels=0, has_mask=True, refine=False, flags=0):
+                 levels=0, has_mask=True, refine=False, flags=0, soft_threshold=None):
         code = {"f32": CPE_F32, "f16": CPE_F16}[dtype]
         self.params = make_params(code, bins_w, bins_h, levels, vote_threshold, tau, max_instances,
-                                  (CPE_FLAG_REFINE if refine else 0) | int(flags))
+                                  (CPE_FLAG_REFINE if refine else 0) |
+                                  (CPE_FLAG_SOFT_VOTE if soft_threshold is not None else 0) | int(flags),
+                                  soft_threshold=float(soft_threshold or 0.0))
         self.shape = (B, H, W, F)
         self.max_instances = max_instances
         rc, self.ctx = cpe_host_ctx_create(B, H, W, F, self.params, has_mask)

@@ -64,6 +64,10 @@ int check_shape(int B, int H, int W, int F, const cpe_params* p) {
   if (p->vote_threshold < 0 || p->max_instances < 1 || p->max_instances > (1 << 20)) return CPE_ERR_PARAM;
   if (p->levels < 0) return CPE_ERR_PARAM;
   if (p->tau != p->tau) return CPE_ERR_PARAM;  // NaN
+  if (p->flags & CPE_FLAG_SOFT_VOTE) {
+    if (p->flags & CPE_FLAG_REFINE) return CPE_ERR_PARAM;
+    if (!(p->soft_threshold >= 0.0f) || !(p->soft_threshold < INFINITY)) return CPE_ERR_PARAM;
+  }
   return CPE_OK;
 }
 
@@ -240,8 +244,21 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     cudaMemsetAsync(ws + L.acc, 0, L.votes_end - L.acc, st);
     return code;
   };
-  rc = cpe::host::launch_decode_vote(st, emb, fg, B, HW, F, p, votes, acc, sums,
-                                     L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr);
+  // Vote: by default the hard vote (each pixel's centroid estimate, one count).  With CPE_FLAG_SOFT_VOTE the map holds
+  // the binary32 histogram of Eq. 6 instead: non-negative binary32 values order like their bit patterns and 0.0f is
+  // all-zero bits, so the zeroing conventions and the peak kernel's comparisons carry over to it unchanged.
+  const bool soft = (p->flags & CPE_FLAG_SOFT_VOTE) != 0;
+  uint32_t t_v = (uint32_t)p->vote_threshold;
+  if (soft) {
+    if ((uintptr_t)emb % 16 || HW % 8) return CPE_ERR_ALIGN;
+    memcpy(&t_v, &p->soft_threshold, sizeof t_v);
+    // the soft-vote kernel only ever ORs into the status words; the peak kernel then ORs too
+    CPE_CUDA(cudaMemsetAsync(status, 0, sizeof(uint32_t) * (size_t)B, st));
+    rc = cpe::host::launch_soft_votes(st, emb, fg, B, HW, F, p, pal_w, pal_h, reinterpret_cast<float*>(votes), status, acc);
+  } else {
+    rc = cpe::host::launch_decode_vote(st, emb, fg, B, HW, F, p, votes, acc, sums,
+                                       L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr);
+  }
   if (rc) return fail_after_votes(rc);
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
@@ -254,7 +271,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     // one CTA per image: it works on a copy of the vote map in shared memory (at most 32 KB)
     const size_t map_smem = one_peak_cta ? 4 * (size_t)L.cells : 0;
     cudaError_t e = launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes,
-                                     p->bins_w, p->bins_h, L.words, (uint32_t)p->vote_threshold, bitmap, p->max_instances, F,
+                                     p->bins_w, p->bins_h, L.words, t_v, soft ? 1 : 0, bitmap, p->max_instances, F,
                                      H, W, pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids, out_count, acc,
                                      counters, status, sums, sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0,
                                      refine ? 1 : 0, L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
@@ -702,7 +719,7 @@ extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_
   const float* pal_h = reinterpret_cast<const float*>(ws + L.pal_h);
   uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.status);
   CPE_CUDA(cudaMemsetAsync(out_hist, 0, sizeof(float) * (size_t)B * params->bins_w * params->bins_h, st));
-  return cpe::host::launch_soft_votes(st, emb, fg_mask, B, (int)HW, F, params, pal_w, pal_h, out_hist, status);
+  return cpe::host::launch_soft_votes(st, emb, fg_mask, B, (int)HW, F, params, pal_w, pal_h, out_hist, status, nullptr);
 }
 
 extern "C" int cpe_instance_masks(cpe_stream_t stream, const int32_t* labels, int B, int H, int W, int n_planes,

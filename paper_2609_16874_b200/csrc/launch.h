@@ -79,9 +79,10 @@ int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                        uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h,
                        uint32_t* hard_q);
 
-// ---- second vote mode (launch_soft.cu)
+// ---- second vote mode (launch_soft.cu).  acc: the per-image accumulators that the peak kernel folds into the
+// counters (participating / non-finite pixels), or NULL.
 int launch_soft_votes(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                      const float* pal_w, const float* pal_h, float* hist, uint32_t* status);
+                      const float* pal_w, const float* pal_h, float* hist, uint32_t* status, uint32_t* acc);
 
 }  // namespace host
 }  // namespace cpe

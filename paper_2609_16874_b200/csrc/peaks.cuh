@@ -15,6 +15,10 @@ constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared me
 // of the peak indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it
 // beats each existing 8-neighbour: larger count, or equal count and lower linear index.
 //
+// `strict` (the soft vote's real-valued map, whose non-negative binary32 values are compared through their bit
+// patterns): the test as the paper prints it, a bin must exceed every existing neighbour; equal neighbours are both
+// rejected.  The image's status word is then OR-ed into (the soft-vote kernel may have set bits) instead of written.
+//
 // Phase 2 (the last CTA of each image to finish phase 1; found with a ticket counter, no waiting): ordered
 // compaction without atomics or sorting.  Every thread counts the set bits of its contiguous slice of the
 // bitmap, an exclusive block scan gives each slice its first output slot, and the slices are written out in
@@ -38,7 +42,7 @@ constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared me
 // per 32-bin word and warp iteration -- and keeps the bitmap and the head of the peak list there as well, so that
 // the dependent steps of this latency-bound kernel stay on the SM.
 __global__ void __launch_bounds__(kPeakThreads)
-peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v,
+peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v, int strict,
              uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
@@ -86,7 +90,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
             if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
             const int nlin = ny * bins_w + nx;
             const uint32_t nv = vote_at(nlin);
-            if (nv > v || (nv == v && nlin < lin)) peak = false;
+            if (nv > v || (nv == v && (strict || nlin < lin))) peak = false;
           }
         }
       }
@@ -181,8 +185,10 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     cnt[CPE_CNT_FULL_SCORED] = 0u;
     if (near_state)
       for (int i = 0; i < kNearStride; ++i) near_state[b * kNearStride + i] = 0u;
-    status[b] = (nonfinite ? (uint32_t)CPE_STATUS_NONFINITE : 0u) |
-                (total > K_max ? (uint32_t)CPE_STATUS_PEAK_OVERFLOW : 0u);
+    const uint32_t st_bits = (nonfinite ? (uint32_t)CPE_STATUS_NONFINITE : 0u) |
+                             (total > K_max ? (uint32_t)CPE_STATUS_PEAK_OVERFLOW : 0u);
+    if (strict) atomicOr(&status[b], st_bits);
+    else status[b] = st_bits;
   }
   __syncthreads();  // the list written above is read below by other threads of this CTA
 

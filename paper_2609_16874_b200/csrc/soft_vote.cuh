@@ -61,7 +61,7 @@ template <typename T, int KA>
 __global__ void __launch_bounds__(kSvThreads, 1)
 soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F, int bins_w, int bins_h,
                  const float* __restrict__ pal_w, const float* __restrict__ pal_h, int vec_mask, float* __restrict__ hist,
-                 uint32_t* __restrict__ status_all) {
+                 uint32_t* __restrict__ status_all, uint32_t* __restrict__ acc) {
   constexpr int KS = KA / 16;                       // k-steps per axis
   constexpr int kPartHalves = 2 * KA * kTcRows;     // one tile part (high or low)
   constexpr uint32_t kTileLbo = kTcRows * 16;       // bytes between core matrices along K in a pixel tile
@@ -245,6 +245,17 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       s_rnx[us * kTcRows + ptid] = nx;
       s_rny[us * kTcRows + ptid] = ny;
       s_rflags[us * kTcRows + ptid] = (present && finite) ? kRfLive : 0u;
+      if (acc && blockIdx.y == 0) {
+        // the decode's counters (the CTAs of the first block of bins see every pixel once): pixels that take part, and
+        // participating pixels with a channel that is not finite
+        const bool any_nonfinite = !((nx + ny) < inf);
+        const uint32_t bv = __ballot_sync(0xffffffffu, present && !any_nonfinite);
+        const uint32_t bn = __ballot_sync(0xffffffffu, present && any_nonfinite);
+        if (lane == 0) {
+          if (bv) atomicAdd(&acc[img * kAccStride + kAccVoting], (uint32_t)__popc(bv));
+          if (bn) atomicAdd(&acc[img * kAccStride + kAccNonfinite], (uint32_t)__popc(bn));
+        }
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(mb_meta + 8 * us);
       ring_head += (uint32_t)ng;
