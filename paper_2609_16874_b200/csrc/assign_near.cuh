@@ -265,7 +265,25 @@ __device__ __forceinline__ float fast_sqrt(float x) {
   return r;
 }
 
+// Shuffles of packed binary16 pairs as plain 32-bit words.
+__device__ __forceinline__ uint32_t h2_bits(__half2 v) {
+  return (uint32_t)__half_as_ushort(__low2half(v)) | ((uint32_t)__half_as_ushort(__high2half(v)) << 16);
+}
+__device__ __forceinline__ __half2 bits_h2(uint32_t w) {
+  return __halves2half2(__ushort_as_half((unsigned short)(w & 0xffffu)), __ushort_as_half((unsigned short)(w >> 16)));
+}
+__device__ __forceinline__ __half2 shfl_xor_h2(__half2 v, int off) {
+  return bits_h2(__shfl_xor_sync(0xffffffffu, h2_bits(v), off));
+}
+__device__ __forceinline__ __half2 shfl_h2(__half2 v, int src) {
+  return bits_h2(__shfl_sync(0xffffffffu, h2_bits(v), src));
+}
+
 constexpr int kStreamThreads = 256;
+// Two CTAs per SM (the step's working set needs more than the 85 registers that three would leave: it spilled), and
+// the plane loads of this many harmonics in flight per thread.
+__host__ __device__ constexpr int stream_ctas_per_sm(int) { return 2; }
+__host__ __device__ constexpr int stream_level_batch(int ft) { return ft >= 4 ? 4 : ft; }
 // What turns a distance accumulated in packed binary16 into an upper bound of the true one.  Per axis the sum has at
 // most 32 non-negative terms: each rounding (difference, fused multiply-add) is within 2^-11 relative, so the sum is
 // within 34 * 2^-11 < 1.7 %, its root within 0.85 %; the candidate rows are rounded to binary16 (2^-12 per component,
@@ -288,7 +306,7 @@ constexpr float kHalfRel = 1.01f, kHalfAbs = 0.008f;
 // candidate rows; an image whose rows do not fit reads them from global memory (`ref_h` / `cand_h`, [K][D] binary16,
 // written by peak_graph_kernel).  Needs 16-byte aligned planes, mask and labels, and H*W a multiple of the group size.
 template <typename T, int FT, bool SAME>
-__global__ void __launch_bounds__(kStreamThreads, 3)
+__global__ void __launch_bounds__(kStreamThreads, stream_ctas_per_sm(FT))
 assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int K_max,
                           const __half* __restrict__ ref_h, const __half* __restrict__ cand_h,
                           const uint32_t* __restrict__ nbr, const int32_t* __restrict__ cell_peak,
@@ -378,42 +396,59 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
     const T* src = e_img + pix0 + (size_t)axis * D2 * plane;
 
     // the first plane loads and the bins go out together
-    constexpr int LB = F < 4 ? F : 4;          // harmonics whose plane loads are in flight together (2 loads each)
+    constexpr int LB = F < stream_level_batch(FT) ? F : stream_level_batch(FT);   // harmonics whose plane loads are in flight together (2 loads each)
     uint4 raw[2 * LB];
-    uint32_t cell[VEC];
+    // a lane looks up, and later finishes, its half of the group's pixels: the axis-0 lane the first half
+    uint32_t cell[H2];
     if (have) {
 #pragma unroll
       for (int q = 0; q < 2 * LB; ++q) raw[q] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)q * plane));
-#pragma unroll
-      for (int j = 0; j < VEC; j += 4) {
-        const uint4 c4 = __ldg(reinterpret_cast<const uint4*>(pc_img + pix0 + j));
-        cell[j] = c4.x; cell[j + 1] = c4.y; cell[j + 2] = c4.z; cell[j + 3] = c4.w;
+      if constexpr (H2 == 4) {
+        const uint4 c4 = __ldg(reinterpret_cast<const uint4*>(pc_img + pix0 + axis * H2));
+        cell[0] = c4.x; cell[1] = c4.y; cell[2] = c4.z; cell[3] = c4.w;
+      } else {
+        const uint2 c2 = __ldg(reinterpret_cast<const uint2*>(pc_img + pix0 + axis * H2));
+        cell[0] = c2.x; cell[1] = c2.y;
       }
     }
     // bins -> peaks.  Pixels of one group nearly always share their peak (ku); at an instance border there is a second
     // one (kv); with more than two the group's pixels are left to the exact walk.
-    int kpix[VEC];
-    uint32_t voted = 0;                         // participating pixels that voted
+    int kpix[H2];
+    uint32_t voted = 0;                         // bit jj: pixel jj of this lane's half participates and voted
     bool many = false;
     int ku = -1, kv = -1;
-    if (have) {
-#pragma unroll
-      for (int j = 0; j < VEC; ++j) {
-        int k = -1;
-        if (((take >> j) & 1u) && cell[j] != 0xffffffffu && (int)cell[j] < cells) {
-          voted |= 1u << j;
-          k = (j > 0 && cell[j] == cell[j - 1] && ((voted >> (j - 1)) & 1u)) ? kpix[j - 1] : __ldg(cp_img + cell[j]);
-          if (k >= K) k = -1;
-          if (k >= 0) {
-            if (ku < 0) ku = k;
-            else if (k != ku) {
-              if (kv < 0) kv = k;
-              else if (k != kv) many = true;
-            }
-          }
+    auto add_peak = [&](int k) {
+      if (k >= 0) {
+        if (ku < 0) ku = k;
+        else if (k != ku) {
+          if (kv < 0) kv = k;
+          else if (k != kv) many = true;
         }
-        kpix[j] = k;
       }
+    };
+    {
+      const uint32_t take_h = (take >> (axis * H2)) & ((1u << H2) - 1u);
+#pragma unroll
+      for (int jj = 0; jj < H2; ++jj) {
+        int k = -1;
+        if (((take_h >> jj) & 1u) && cell[jj] != 0xffffffffu && (int)cell[jj] < cells) {
+          voted |= 1u << jj;
+          k = (jj > 0 && cell[jj] == cell[jj - 1] && ((voted >> (jj - 1)) & 1u)) ? kpix[jj - 1] : __ldg(cp_img + cell[jj]);
+          if (k >= K) k = -1;
+          add_peak(k);
+        }
+        kpix[jj] = k;
+      }
+      // the two halves' peaks become the group's, the first half's first, so that both lanes name them alike
+      const uint32_t mine = ((uint32_t)ku & 0xfffu) | (((uint32_t)kv & 0xfffu) << 12) | (many ? 1u << 24 : 0u);
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
+      const uint32_t first = axis ? other : mine, second = axis ? mine : other;
+      auto peak_of = [](uint32_t v) { return v == 0xfffu ? -1 : (int)v; };   // (K <= 1024: 0xfff is no peak index)
+      ku = peak_of(first & 0xfffu);
+      kv = peak_of((first >> 12) & 0xfffu);
+      many = ((first | second) >> 24) & 1u;
+      add_peak(peak_of(second & 0xfffu));
+      add_peak(peak_of((second >> 12) & 0xfffu));
     }
     if (many) ku = kv = -1;
     // the first two entries of the peaks' lists
@@ -485,15 +520,75 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
       }
     };
     if (ku >= 0) accumulate(ku, kfu, s, sc, true);
-    if (kv >= 0) accumulate(kv, kfv, sv, scv, false);   // an instance border: the planes come from L1 this time
-    // swap with the partner lane: afterwards every lane has both axes' sums of its half of the pixels
-    // (all register-array indices below are compile-time constants: the axis picks between two of them)
-    // per pixel, pick the sums of its own peak first (register pairs hold two pixels: blend the halves)
+    // An instance border: a group with a second peak.  Nearly every step of a large image has one such group, so the
+    // second pass over it is shared by the whole warp instead of being run by the group's two lanes while thirty wait:
+    // lane (pixel pair, axis, part of the axis' planes) re-reads its 32-bit pieces (cache hits), the parts are summed
+    // with shuffles and handed to the group's lanes in the layout of the first pass.
     {
-      uint32_t use_v = 0;
+      constexpr int NPQ = 16 / H2;               // parts that an axis' planes are split into
+      constexpr int PL = D2 / NPQ;               // planes per lane
+      static_assert(PL >= 1 && PL * NPQ == D2, "the planes divide among the lanes");
+      uint32_t border = __ballot_sync(0xffffffffu, kv >= 0 && axis == 0);
+      const int pp = lane & (H2 - 1), a2 = (lane / H2) & 1, pq = lane / (2 * H2);
+#pragma unroll 1
+      while (border) {
+        const int src_lane = __ffs(border) - 1;
+        border &= border - 1;
+        const int kvb = __shfl_sync(0xffffffffu, kv, src_lane);
+        const int kfb = __shfl_sync(0xffffffffu, kfv, src_lane);
+        const uint32_t gb = __shfl_sync(0xffffffffu, (uint32_t)(pix0 / VEC), src_lane);   // group index (< 2^28)
+        const int c0 = a2 * D2 + pq * PL;
+        const T* pb = e_img + (size_t)gb * VEC + 2 * pp + (size_t)c0 * plane;
+        const __half* rr = rows_ref + (size_t)kvb * D + c0;
+        const __half* rc = rows_cand + (size_t)kfb * D + c0;
+        __half2 v[PL];
 #pragma unroll
-      for (int j = 0; j < VEC; ++j)
-        if (kv >= 0 && kpix[j] == kv) use_v |= 1u << j;
+        for (int i = 0; i < PL; ++i) {
+          if constexpr (sizeof(T) == 2) {
+            const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pb + (size_t)i * plane));
+            v[i] = *reinterpret_cast<const __half2*>(&w);
+          } else {
+            const float2 f = __ldg(reinterpret_cast<const float2*>(pb + (size_t)i * plane));
+            v[i] = __floats2half2_rn(f.x, f.y);
+          }
+        }
+        __half2 acc = __float2half2_rn(0.0f), accc = acc;
+#pragma unroll
+        for (int i = 0; i < PL; ++i) {
+          const __half2 d = __hsub2(v[i], __half2half2(rr[i]));
+          acc = __hfma2(d, d, acc);
+          if constexpr (!SAME) {
+            const __half2 dc = __hsub2(v[i], __half2half2(rc[i]));
+            accc = __hfma2(dc, dc, accc);
+          }
+        }
+#pragma unroll
+        for (int off = 2 * H2; off < 32; off <<= 1) {
+          acc = __hadd2(acc, shfl_xor_h2(acc, off));
+          if constexpr (!SAME) accc = __hadd2(accc, shfl_xor_h2(accc, off));
+        }
+        // lane (pp, axis) of part 0 holds the sums of pixel pair pp on that axis
+        const bool mine = (lane >> 1) == (src_lane >> 1);
+#pragma unroll
+        for (int j = 0; j < H2; ++j) {
+          const __half2 t = shfl_h2(acc, axis * H2 + j);
+          if (mine) sv[j] = t;
+          if constexpr (!SAME) {
+            const __half2 tc = shfl_h2(accc, axis * H2 + j);
+            if (mine) scv[j] = tc;
+          }
+        }
+      }
+    }
+    // per pixel, pick the sums of its own peak first (register pairs hold two pixels: blend the halves).  The shuffle
+    // is executed by every lane: a group's two lanes share kv, the lanes of other groups do not.
+    {
+      uint32_t use_h = 0;
+#pragma unroll
+      for (int jj = 0; jj < H2; ++jj)
+        if (kv >= 0 && kpix[jj] == kv) use_h |= 1u << jj;
+      const uint32_t use_o = __shfl_xor_sync(0xffffffffu, use_h, 1);
+      const uint32_t use_v = axis ? (use_o | (use_h << H2)) : (use_h | (use_o << H2));
       if (use_v) {
 #pragma unroll
         for (int j = 0; j < H2; ++j) {
@@ -504,46 +599,44 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
         }
       }
     }
-    __half2 so[H2], sco[H2];
+    // swap with the partner lane: each lane keeps its own axis' sums of its half of the pixels and gets the partner's
+    // (the distances below are symmetric in the two axes, so which one is x does not matter)
+    constexpr int Q2 = H2 / 2;                  // half2 registers per half of the group (2 for binary16, 1 for binary32)
+    float2 own[Q2], oth[Q2], cwn[Q2], cth[Q2];
 #pragma unroll
-    for (int j = 0; j < H2; ++j) {
-      uint32_t w = *reinterpret_cast<uint32_t*>(&s[j]);
-      w = __shfl_xor_sync(0xffffffffu, w, 1);
-      so[j] = *reinterpret_cast<__half2*>(&w);
+    for (int i = 0; i < Q2; ++i) {
+      const __half2 send = axis ? s[i] : s[Q2 + i];
+      const __half2 keep = axis ? s[Q2 + i] : s[i];
+      own[i] = __half22float2(keep);
+      oth[i] = __half22float2(shfl_xor_h2(send, 1));
       if constexpr (!SAME) {
-        uint32_t wc = *reinterpret_cast<uint32_t*>(&sc[j]);
-        wc = __shfl_xor_sync(0xffffffffu, wc, 1);
-        sco[j] = *reinterpret_cast<__half2*>(&wc);
+        const __half2 sendc = axis ? sc[i] : sc[Q2 + i];
+        const __half2 keepc = axis ? sc[Q2 + i] : sc[i];
+        cwn[i] = __half22float2(keepc);
+        cth[i] = __half22float2(shfl_xor_h2(sendc, 1));
       } else {
-        sco[j] = so[j];
+        cwn[i] = own[i];
+        cth[i] = oth[i];
       }
     }
     int my_label[H2];
     uint32_t n_likely_hard = 0;
-    constexpr int Q2 = H2 / 2;                  // half2 registers per half of the group (2 for binary16, 1 for binary32)
 #pragma unroll
     for (int jj = 0; jj < H2; ++jj) {
-      const int j = axis * H2 + jj;              // the axis-0 lane finishes the first half, the axis-1 lane the second
-      // own sums of pixel jj (first half) and of pixel H2 + jj (second half), and the partner's
-      const float2 own_lo = __half22float2(s[jj / 2]), own_hi = __half22float2(s[Q2 + jj / 2]);
-      const float2 oth_lo = __half22float2(so[jj / 2]), oth_hi = __half22float2(so[Q2 + jj / 2]);
-      const float2 cwn_lo = __half22float2(sc[jj / 2]), cwn_hi = __half22float2(sc[Q2 + jj / 2]);
-      const float2 cth_lo = __half22float2(sco[jj / 2]), cth_hi = __half22float2(sco[Q2 + jj / 2]);
-      const float sx = axis == 0 ? ((jj & 1) ? own_lo.y : own_lo.x) : ((jj & 1) ? oth_hi.y : oth_hi.x);
-      const float sy = axis == 0 ? ((jj & 1) ? oth_lo.y : oth_lo.x) : ((jj & 1) ? own_hi.y : own_hi.x);
-      const float cx = axis == 0 ? ((jj & 1) ? cwn_lo.y : cwn_lo.x) : ((jj & 1) ? cth_hi.y : cth_hi.x);
-      const float cy = axis == 0 ? ((jj & 1) ? cth_lo.y : cth_lo.x) : ((jj & 1) ? cwn_hi.y : cwn_hi.x);
-      const int k0j = axis == 0 ? kpix[jj] : kpix[H2 + jj];
+      const int j = axis * H2 + jj;              // the pixel's place in the group
+      const float sa = (jj & 1) ? own[jj / 2].y : own[jj / 2].x, sb = (jj & 1) ? oth[jj / 2].y : oth[jj / 2].x;
+      const float ca = (jj & 1) ? cwn[jj / 2].y : cwn[jj / 2].x, cb = (jj & 1) ? cth[jj / 2].y : cth[jj / 2].x;
+      const int k0j = kpix[jj];
       int label = 0;
       bool slow = false;
-      if ((voted >> j) & 1u) {
+      if ((voted >> jj) & 1u) {
         slow = true;
         bool likely_hard = k0j < 0;
         if (k0j >= 0 && !many) {
           const uint2 e01 = k0j == ku ? e01u : e01v;
           const int kfj = (int)(e01.x & 0xfffu);
-          const float t = (fast_sqrt(sx) + fast_sqrt(sy)) * kHalfRel + kHalfAbs;
-          const float dub = SAME ? t : (fast_sqrt(cx) + fast_sqrt(cy)) * kHalfRel + kHalfAbs;
+          const float t = (fast_sqrt(sa) + fast_sqrt(sb)) * kHalfRel + kHalfAbs;
+          const float dub = SAME ? t : (fast_sqrt(ca) + fast_sqrt(cb)) * kHalfRel + kHalfAbs;
           const float reach = (dub + t) * kNearSlack;
           // the list's first entry is the candidate bounded above (with refined candidates that must be k0 itself:
           // an identical row with a lower index may precede it); the second entry decides whether the walk is over

@@ -114,6 +114,7 @@ struct PruneArgs {
   uint32_t* near_state = nullptr;
   uint32_t* slow_q = nullptr;
   int q_cap = 0;
+  int W = 0;               // image width (the streaming kernel walks the image in patches)
   void* ref_h = nullptr;
   void* cand_h = nullptr;
   uint32_t* hard_q = nullptr;
@@ -154,7 +155,7 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
     rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref_emb, peak_emb, pr->ref2, pr->cand2, pr->nbr,
                                        pr->cell_peak, pr->pix_cell, cells, count, labels, best, second, pr->near_state,
                                        k_limit + 1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h,
-                                       pr->hard_q);
+                                       pr->hard_q, pr->W);
     if (rc) return rc;
   }
   // (also with a limit of 0: an image without any peak still gets its all-zero label map from this kernel)
@@ -229,6 +230,7 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     pr.near_state = reinterpret_cast<uint32_t*>(ws + L.near_state);
     pr.slow_q = reinterpret_cast<uint32_t*>(ws + L.slow_q);
     pr.q_cap = L.q_cap;
+    pr.W = W;
     pr.hard_q = reinterpret_cast<uint32_t*>(ws + L.hard_q);
     pr.ref_h = ws + L.ref_h;
     pr.cand_h = ws + L.cand_h;

@@ -265,10 +265,10 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 constexpr int kVecGroupsMax = 256;   // groups per CTA: 256, 128 or 64 (template parameter GROUPS; the launcher takes the
                                      // largest that still gives a full wave of CTAs -- small images are latency-bound
                                      // and want many short CTAs, large ones want fewer fixed costs)
-constexpr int kVecLevelBatch = 4;  // harmonics whose plane loads are in flight together (2 loads each)
+constexpr int kVecLevelBatch = 2;  // harmonics whose plane loads are in flight together (2 loads each)
 
 template <typename T, int FT, int MODE, int GROUPS>
-__global__ void __launch_bounds__(kVoteThreads, 3)
+__global__ void __launch_bounds__(kVoteThreads, 4)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
                        int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
                        long long* __restrict__ sums, uint32_t* __restrict__ pix_cell) {
@@ -352,33 +352,36 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
     const T* src = e + span0 + (size_t)(ent & 0xffu) * VEC + (size_t)axis * 2 * F * plane;
 
     float p[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) p[j] = 0.0f;   // the first harmonic's step from 0 returns its own estimate u
     uint32_t okbits = (1u << VEC) - 1u;
     if (have) {
       float fin[VEC];
 #pragma unroll
       for (int j = 0; j < VEC; ++j) fin[j] = 0.0f;
-      // the plane loads of up to 8 harmonics (16 x 128 bits) are in flight together, kept raw in registers
+      // The plane loads of a batch of harmonics are in flight together, kept raw in registers.  The loop over the
+      // batches is not unrolled: the body for one batch (VEC pixels x LB harmonics) then stays in the instruction
+      // cache, which the fully unrolled chain of all F harmonics overflowed.
       constexpr int LB = F < kVecLevelBatch ? F : kVecLevelBatch;
-#pragma unroll
-      for (int l0 = 0; l0 < F; l0 += LB) {
+      const T* ptr = src;
+#pragma unroll 1
+      for (int l0 = 0; l0 < F; l0 += LB, ptr += (size_t)(2 * LB) * plane) {
         uint4 raw[2 * LB];
 #pragma unroll
-        for (int i = 0; i < 2 * LB; ++i)
-          raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(2 * l0 + i) * plane));
+        for (int i = 0; i < 2 * LB; ++i) raw[i] = __ldg(reinterpret_cast<const uint4*>(ptr + (size_t)i * plane));
 #pragma unroll
         for (int ll = 0; ll < LB; ++ll) {
-          const int l = l0 + ll;
           float s[VEC], c[VEC];
           unpack_vec<T>(raw[2 * ll], s);
           unpack_vec<T>(raw[2 * ll + 1], c);
 #pragma unroll
           for (int j = 0; j < VEC; ++j) fin[j] = fold_finite(fin[j], s[j], c[j]);
-          if (l < Fu) {
+          if (l0 + ll < Fu) {
             // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
 #pragma unroll
             for (int j = 0; j < VEC; j += 2) {
               const float2 u = atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
-              const float2 v = (l == 0) ? u : refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
+              const float2 v = refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
               p[j] = v.x;
               p[j + 1] = v.y;
             }
@@ -391,9 +394,6 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
         p[j] = __fmul_rn(p[j], unscale);
         if (fin[j] != fin[j]) okbits &= ~(1u << j);
       }
-    } else {
-#pragma unroll
-      for (int j = 0; j < VEC; ++j) p[j] = 0.0f;
     }
     // swap with the partner lane: afterwards every lane knows both coordinates of its half of the pixels
     const uint32_t ok_other = __shfl_xor_sync(0xffffffffu, okbits, 1);

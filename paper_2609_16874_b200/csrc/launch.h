@@ -77,7 +77,7 @@ int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                        const uint32_t* nbr, const int32_t* cell_peak, const uint32_t* pix_cell, int cells,
                        const int32_t* count, int32_t* labels, float* best, float* second, uint32_t* near_state, int k_min,
                        uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h,
-                       uint32_t* hard_q);
+                       uint32_t* hard_q, int W);
 
 // ---- second vote mode (launch_soft.cu).  acc: the per-image accumulators that the peak kernel folds into the
 // counters (participating / non-finite pixels), or NULL.

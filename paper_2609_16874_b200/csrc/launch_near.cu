@@ -52,6 +52,7 @@ struct NearArgs {
   uint32_t* status;
   const void *ref_h, *cand_h;
   uint32_t* hard_q;
+  int W;
 };
 
 template <typename T, int FT, bool WANT2>
@@ -82,7 +83,7 @@ int launch_stream_t(cudaStream_t st, const NearArgs& a) {
   // a warp takes 16 groups per step; a bounded grid (three CTAs per SM), shared among the images
   const long long n_steps = ((long long)a.HW / VEC + 15) / 16;
   const long long ctas = (n_steps + cpe::kStreamThreads / 32 - 1) / (cpe::kStreamThreads / 32);
-  const long long per_image = std::max(1, (3 * sm_count() + a.B - 1) / a.B);
+  const long long per_image = std::max(1, (cpe::stream_ctas_per_sm(FT) * sm_count() + a.B - 1) / a.B);
   dim3 grid((unsigned)std::min(ctas, per_image), (unsigned)a.B);
   CPE_CUDA(launch_dependent(plain_launch(a.p), kern, grid, cpe::kStreamThreads, (size_t)smem, st,
                             static_cast<const T*>(a.emb), a.fg, a.HW, a.p->max_instances,
@@ -138,9 +139,9 @@ int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int 
                        const uint32_t* nbr, const int32_t* cell_peak, const uint32_t* pix_cell, int cells,
                        const int32_t* count, int32_t* labels, float* best, float* second, uint32_t* near_state, int k_min,
                        uint32_t* slow_q, int q_cap, uint32_t* status, const void* ref_h, const void* cand_h,
-                       uint32_t* hard_q) {
+                       uint32_t* hard_q, int W) {
   const NearArgs a{emb, fg, B, HW, p, ref_emb, cand_emb, ref2, cand2, nbr, cell_peak, pix_cell, cells, count, labels, best,
-                   second, near_state, k_min, slow_q, q_cap, status, ref_h, cand_h, hard_q};
+                   second, near_state, k_min, slow_q, q_cap, status, ref_h, cand_h, hard_q, W};
   return p->dtype == CPE_F32 ? launch_near_f<float>(st, F, a) : launch_near_f<__half>(st, F, a);
 }
 

@@ -17,8 +17,8 @@ int launch_decode_vote_t(cudaStream_t st, const void* emb, const uint8_t* fg, in
                    (F == 4 || F == 8 || F == 16);
   if (vec) {
     const long long groups = (long long)HW / V;
-    // the largest span that still gives one full wave of CTAs (three resident per SM), else the smallest
-    const long long wave = 3LL * sm_count();
+    // the largest span that still gives one full wave of CTAs (four resident per SM), else the smallest
+    const long long wave = 4LL * sm_count();
     const int span = (groups + 255) / 256 * B >= wave ? 256 : (groups + 127) / 128 * B >= wave ? 128 : 64;
     dim3 grid((unsigned)((groups + span - 1) / span), (unsigned)B);
 #define CPE_LAUNCH_VOTE_G(FT_, RF_, G_)                                                                              \

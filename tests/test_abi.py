@@ -67,7 +67,11 @@ def test_argument_errors_are_reported_before_any_launch():
     mis = cb.make_params(cb.CPE_F32, 32, 32, workspace=256 * 1000 + 8, workspace_bytes=1 << 30)
     assert cb.cpe_decode(0, fake, 0, 1, 8, 8, 4, mis, fake, fake, fake) == cb.CPE_ERR_WORKSPACE
     for kw, code in [(dict(vote_threshold=-1), cb.CPE_ERR_PARAM), (dict(max_instances=0), cb.CPE_ERR_PARAM),
-                     (dict(levels=-2), cb.CPE_ERR_PARAM), (dict(tau=math.nan), cb.CPE_ERR_PARAM)]:
+                     (dict(levels=-2), cb.CPE_ERR_PARAM), (dict(tau=math.nan), cb.CPE_ERR_PARAM),
+                     (dict(flags=cb.CPE_FLAG_SOFT_VOTE, soft_threshold=-1.0), cb.CPE_ERR_PARAM),
+                     (dict(flags=cb.CPE_FLAG_SOFT_VOTE, soft_threshold=math.inf), cb.CPE_ERR_PARAM),
+                     (dict(flags=cb.CPE_FLAG_SOFT_VOTE, soft_threshold=math.nan), cb.CPE_ERR_PARAM),
+                     (dict(flags=cb.CPE_FLAG_SOFT_VOTE | cb.CPE_FLAG_REFINE, soft_threshold=1.0), cb.CPE_ERR_PARAM)]:
         q = cb.make_params(cb.CPE_F32, 32, 32, workspace=256 * 1000, workspace_bytes=1 << 30, **kw)
         assert cb.cpe_decode(0, fake, 0, 1, 8, 8, 4, q, fake, fake, fake) == code
     q = cb.make_params(7, 32, 32, workspace=256 * 1000, workspace_bytes=1 << 30)
