@@ -84,16 +84,17 @@ __device__ __forceinline__ void near_full_scan(const float2 (&e2)[D / 2], int K,
   }
 }
 
-// The same for one pixel by a whole warp (every lane passes the same pixel): lane l scores the peaks l, l + 32, ...
+// The same for one pixel by a whole warp (every lane passes the same pixel): a lane scores the peaks k_first,
+// k_first + k_stride, ... (lane, 32 for a warp on its own; several warps may share the peaks of one pixel)
 // with the pixel's values fetched by every lane (the same addresses: one transaction per load), then the lanes' results
 // are merged -- smaller distance first, lower k on equal distances, which is what the serial scan in ascending k gives.
 // A single thread scanning hundreds of peaks is a chain of dependent row fetches that takes as long as the rest of the
 // kernel; 32 lanes share it.
 template <typename T, int D, bool WANT2>
 __device__ __forceinline__ void near_full_scan_warp(const T* __restrict__ p, size_t plane, int K,
-                                                    const float* __restrict__ cand_img, float& d1, float& d2, int& k1) {
+                                                    const float* __restrict__ cand_img, float& d1, float& d2, int& k1,
+                                                    int k_first, int k_stride) {
   const float inf = __int_as_float(0x7f800000);
-  const int lane = threadIdx.x & 31;
   float2 e2[D / 2];
 #pragma unroll
   for (int c = 0; c < D / 2; ++c) {
@@ -103,7 +104,7 @@ __device__ __forceinline__ void near_full_scan_warp(const T* __restrict__ p, siz
   d1 = d2 = inf;
   k1 = 0x7fffffff;
   float bound2 = inf;
-  for (int k = lane; k < K; k += 32) {
+  for (int k = k_first; k < K; k += k_stride) {
     const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
     if (d < d1) { d2 = d1; d1 = d; k1 = k; }
     else if (d < d2) { d2 = d; }
@@ -224,7 +225,7 @@ assign_near_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, in
         const long long nn = __shfl_sync(0xffffffffu, n, src_lane);
         float w1, w2;
         int wk;
-        near_full_scan_warp<T, D, WANT2>(emb + (size_t)b * D * plane + nn, plane, K, cand_img, w1, w2, wk);
+        near_full_scan_warp<T, D, WANT2>(emb + (size_t)b * D * plane + nn, plane, K, cand_img, w1, w2, wk, (int)(threadIdx.x & 31), 32);
         if ((tid & 31) == src_lane) {
           d1 = w1;
           d2 = w2;
@@ -781,22 +782,63 @@ assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
   if (state[kNearGiveUp]) return;                // the filtered kernel redoes the whole image
   const int n_h = (int)min(state[kNearHardQueue], (uint32_t)q_cap);
   const float* cand_img = cand2 + (size_t)b * K_max * D;
-  const int lane = threadIdx.x & 31;
-  const int warp = blockIdx.x * (kNearThreads / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (kNearThreads / 32);
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  constexpr int kWarps = kNearThreads / 32;
   uint32_t n_rejected = 0, n_full = 0;
-  for (int i = warp; i < n_h; i += n_warps) {
-    const size_t n = hard_q[(size_t)b * q_cap + i];
-    float d1, d2;
-    int k1;
-    near_full_scan_warp<T, D, false>(emb + (size_t)b * D * plane + n, plane, K, cand_img, d1, d2, k1);
-    if (lane == 0) {
-      ++n_full;
-      int label = 0;
-      if (k1 >= 0) {
-        if (d1 < tau) label = k1 + 1;
-        else ++n_rejected;
+  auto finish = [&](size_t n, float d1, int k1) {
+    ++n_full;
+    int label = 0;
+    if (k1 >= 0) {
+      if (d1 < tau) label = k1 + 1;
+      else ++n_rejected;
+    }
+    labels[(size_t)b * plane + n] = label;
+  };
+  if (n_h <= (int)gridDim.x) {
+    // Few pixels (the usual case: a handful per image): a pixel's scan is a chain of K / 32 dependent row fetches for
+    // one warp, so a whole CTA shares it, thread t scoring the peaks t, t + 256, ...; the warps' results are merged
+    // with the same rule as the lanes' (smaller distance, then lower k).
+    __shared__ float s_d1[kWarps], s_d2[kWarps];
+    __shared__ int s_k1[kWarps];
+    for (int i = blockIdx.x; i < n_h; i += gridDim.x) {       // (at most one round)
+      const size_t n = hard_q[(size_t)b * q_cap + i];
+      float d1, d2;
+      int k1;
+      near_full_scan_warp<T, D, false>(emb + (size_t)b * D * plane + n, plane, K, cand_img, d1, d2, k1, (int)threadIdx.x,
+                                       kNearThreads);
+      if (lane == 0) {
+        s_d1[wid] = d1;
+        s_d2[wid] = d2;
+        s_k1[wid] = k1 < 0 ? 0x7fffffff : k1;
       }
-      labels[(size_t)b * plane + n] = label;
+      __syncthreads();
+      if (wid == 0) {
+        static_assert(kWarps <= 32, "one lane per warp result");
+        const float inf = __int_as_float(0x7f800000);
+        d1 = lane < kWarps ? s_d1[lane] : inf;
+        d2 = lane < kWarps ? s_d2[lane] : inf;
+        k1 = lane < kWarps ? s_k1[lane] : 0x7fffffff;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          const float od1 = __shfl_xor_sync(0xffffffffu, d1, off), od2 = __shfl_xor_sync(0xffffffffu, d2, off);
+          const int ok1 = __shfl_xor_sync(0xffffffffu, k1, off);
+          const bool other_wins = od1 < d1 || (od1 == d1 && ok1 < k1);
+          const float loser = other_wins ? d1 : od1;
+          if (other_wins) { d1 = od1; k1 = ok1; }
+          d2 = fminf(fminf(d2, od2), loser);
+        }
+        if (lane == 0) finish(n, d1, k1 == 0x7fffffff ? -1 : k1);
+      }
+      __syncthreads();
+    }
+  } else {
+    const int warp = blockIdx.x * kWarps + wid, n_warps = gridDim.x * kWarps;
+    for (int i = warp; i < n_h; i += n_warps) {
+      const size_t n = hard_q[(size_t)b * q_cap + i];
+      float d1, d2;
+      int k1;
+      near_full_scan_warp<T, D, false>(emb + (size_t)b * D * plane + n, plane, K, cand_img, d1, d2, k1, lane, 32);
+      if (lane == 0) finish(n, d1, k1);
     }
   }
   near_flush_counters(state, n_rejected, n_full * (uint32_t)K, 0u, n_full);

@@ -114,7 +114,17 @@ struct PruneArgs {
   uint32_t* near_state = nullptr;
   uint32_t* slow_q = nullptr;
   int q_cap = 0;
-  int W = 0;               // image width (the streaming kernel walks the image in patches)
+  int H = 0, W = 0;
+  // what the kernel that evaluates gamma of the peaks' mean estimates reads and writes
+  const uint32_t* votes = nullptr;
+  const long long* sums = nullptr;
+  const int32_t* peak_cell = nullptr;
+  float* gamma_out = nullptr;       // peak_emb with refined candidates, else ref_emb
+  float* out_centroids = nullptr;
+  int refine_out = 0;
+  const float *pal_w = nullptr, *pal_h = nullptr;
+  float* peak_emb = nullptr;
+  long long* sums_to_zero = nullptr;   // the list kernel leaves the sums zero for the next decode (NULL: kept)
   void* ref_h = nullptr;
   void* cand_h = nullptr;
   uint32_t* hard_q = nullptr;
@@ -146,8 +156,17 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   }
   int rc = CPE_OK;
   if (pr) {
+    // gamma of every peak's mean estimate (the bounds' reference points; the candidates too when they are refined),
+    // a thread per (peak, axis, harmonic) over as many CTAs as the largest image can need
+    const int k_cap = std::min(p->max_instances, cpe::kNearMaxPeaks);
+    const int ctas = std::max(1, std::min((k_cap * 2 * F + cpe::kRowsThreads - 1) / cpe::kRowsThreads, 4 * sm_count()));
+    CPE_CUDA(launch_dependent(plain_launch(p), cpe::peak_rows_kernel, dim3((unsigned)ctas, (unsigned)B), cpe::kRowsThreads, 0,
+                              st, pr->votes, pr->sums, p->bins_w, p->bins_h, p->max_instances, F, pr->H, pr->W,
+                              pr->peak_cell, count, pr->refine_out, pr->gamma_out, pr->out_centroids, pr->pal_w, pr->pal_h,
+                              pr->peak_emb));
+    CPE_CUDA(cudaGetLastError());
     rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->ref_h,
-                                      pr->cand_h, pr->nbr);
+                                      pr->cand_h, pr->nbr, pr->sums_to_zero, cells);
     if (rc) return rc;
   }
   if (ev_lists) CPE_CUDA(cudaEventRecord(ev_lists, st));
@@ -230,20 +249,35 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     pr.near_state = reinterpret_cast<uint32_t*>(ws + L.near_state);
     pr.slow_q = reinterpret_cast<uint32_t*>(ws + L.slow_q);
     pr.q_cap = L.q_cap;
+    pr.H = H;
     pr.W = W;
+    pr.votes = votes;
+    pr.sums = sums;
+    pr.peak_cell = peak_cell;
+    pr.refine_out = refine ? 1 : 0;
+    pr.gamma_out = refine ? peak_emb : reinterpret_cast<float*>(ws + L.ref_emb);
+    pr.out_centroids = out_centroids;
+    pr.pal_w = pal_w;
+    pr.pal_h = pal_h;
+    pr.peak_emb = peak_emb;
+    pr.sums_to_zero = keep_votes ? nullptr : sums;
     pr.hard_q = reinterpret_cast<uint32_t*>(ws + L.hard_q);
     pr.ref_h = ws + L.ref_h;
     pr.cand_h = ws + L.cand_h;
   }
   const bool one_peak_cta = L.words <= cpe::kPeakStageWords;
-  const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes;
-  if (sums && !sums_cleared_by_peaks) CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
+  // (with the pruned assignment the sums are read by a later kernel: they are cleared at the start instead)
+  const bool sums_cleared_by_peaks = sums && one_peak_cta && !keep_votes && !L.prune;
+  const bool sums_cleared_by_lists = sums && L.prune && !keep_votes;
+  if (sums && !sums_cleared_by_peaks && !sums_cleared_by_lists)
+    CPE_CUDA(cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st));
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_DECODE_VOTE], st));
   // From here on the vote map and the accumulators may hold this decode's votes.  If a later enqueue fails, the
   // kernel that would have left them zero for the next decode never runs: clear them here instead.
   auto fail_after_votes = [&](int code) {
     cudaMemsetAsync(ws + L.acc, 0, L.votes_end - L.acc, st);
+    if (sums) cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st);
     return code;
   };
   // Vote: by default the hard vote (each pixel's centroid estimate, one count).  With CPE_FLAG_SOFT_VOTE the map holds
@@ -275,8 +309,9 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     cudaError_t e = launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes,
                                      p->bins_w, p->bins_h, L.words, t_v, soft ? 1 : 0, bitmap, p->max_instances, F,
                                      H, W, pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids, out_count, acc,
-                                     counters, status, sums, sums_cleared_by_peaks ? 1 : 0, one_peak_cta ? 1 : 0,
-                                     refine ? 1 : 0, L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
+                                     counters, status, L.prune ? nullptr : sums, sums_cleared_by_peaks ? 1 : 0,
+                                     one_peak_cta ? 1 : 0, refine ? 1 : 0, L.prune ? 1 : 0,
+                                     L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
                                      L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr, pr.near_state);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return fail_after_votes(cuda_fail(e));

@@ -71,7 +71,8 @@ int launch_assign_filtered(cudaStream_t st, const void* emb, const uint8_t* fg, 
 // fewer than k_min peaks are left alone; near_state tells the filtered kernel, launched afterwards, which images it
 // is handed.
 int launch_peak_graph(cudaStream_t st, int B, int F, const cpe_params* p, const float* ref_emb, const float* cand_emb,
-                      const int32_t* count, int k_min, float* ref2, float* cand2, void* ref_h, void* cand_h, uint32_t* nbr);
+                      const int32_t* count, int k_min, float* ref2, float* cand2, void* ref_h, void* cand_h, uint32_t* nbr,
+                      long long* sums_to_zero, int cells);
 int launch_assign_near(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
                        const float* ref_emb, const float* cand_emb, const float* ref2, const float* cand2,
                        const uint32_t* nbr, const int32_t* cell_peak, const uint32_t* pix_cell, int cells,

@@ -9,7 +9,8 @@ namespace cpe {
 namespace host {
 
 int launch_peak_graph(cudaStream_t st, int B, int F, const cpe_params* p, const float* ref_emb, const float* cand_emb,
-                      const int32_t* count, int k_min, float* ref2, float* cand2, void* ref_h, void* cand_h, uint32_t* nbr) {
+                      const int32_t* count, int k_min, float* ref2, float* cand2, void* ref_h, void* cand_h, uint32_t* nbr,
+                      long long* sums_to_zero, int cells) {
   // one CTA per peak; no image has more than min(max_instances, kNearMaxPeaks) peaks to list
   const int k_cap = std::min(p->max_instances, cpe::kNearMaxPeaks);
   const int per_image = std::max(1, (8 * sm_count() + B - 1) / B);
@@ -18,7 +19,7 @@ int launch_peak_graph(cudaStream_t st, int B, int F, const cpe_params* p, const 
 #define CPE_GRAPH(FT_)                                                                                               \
   CPE_CUDA(launch_dependent(plain_launch(p), cpe::peak_graph_kernel<FT_>, grid, cpe::kGraphThreads, smem, st, ref_emb, \
                             cand_emb, count, p->max_instances, k_min, ref2, cand2,             \
-                            static_cast<__half*>(ref_h), static_cast<__half*>(cand_h), nbr))
+                            static_cast<__half*>(ref_h), static_cast<__half*>(cand_h), nbr, sums_to_zero, cells))
   switch (F) {
     case 4: CPE_GRAPH(4); break;
     case 8: CPE_GRAPH(8); break;

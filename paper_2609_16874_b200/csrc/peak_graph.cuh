@@ -7,7 +7,7 @@
 // some candidate has been scored exactly with distance U, every k with G_k - t > U is out, whatever the pixel.  G
 // depends on the peaks only: this kernel computes it for g = the reference point of peak k0 (gamma of the mean
 // estimate of the peak's 3x3 window of bins, the refined centroid) against all candidates of the image, and keeps the
-// kNbrCap smallest in ascending order, so that the assignment scans a list until G exceeds U + t and stops.
+// kNbrCap smallest in ascending order (a sort in shared memory), so that the assignment scans a list until G exceeds U + t and stops.
 //
 // A list entry is (Gq << 12) | k with Gq = floor(G * 2^16 * (1 - 2^-15)), i.e. G rounded DOWN by more than its own
 // rounding error (at most (2F + 3) units in the last place), as the bound needs; entries ascend as plain integers.
@@ -22,7 +22,7 @@
 
 namespace cpe {
 
-constexpr int kGraphThreads = 128;
+constexpr int kGraphThreads = 256;
 constexpr uint32_t kNbrEnd = 0xffffffffu;
 
 // One CTA per peak k0 (the grid strides over the peaks); its threads share the candidates.
@@ -31,15 +31,21 @@ __global__ void __launch_bounds__(kGraphThreads)
 peak_graph_kernel(const float* __restrict__ ref_emb, const float* __restrict__ cand_emb,
                   const int32_t* __restrict__ count_ptr, int K_max, int k_min, float* __restrict__ ref2,
                   float* __restrict__ cand2, __half* __restrict__ ref_h, __half* __restrict__ cand_h,
-                  uint32_t* __restrict__ nbr) {
+                  uint32_t* __restrict__ nbr, long long* __restrict__ sums_to_zero, int cells) {
   constexpr int D = 4 * FT, D2 = 2 * FT;
   __shared__ __align__(16) float s_ref[D];                    // plain order: x half, y half
   __shared__ __align__(16) uint32_t s_keys[kNearMaxPeaks];
   grid_dependency_sync();
   const int b = blockIdx.y;
+  const int tid = threadIdx.x;
+  // the per-bin sums have no reader left (the kernel before this one was the last): this CTA's share of them is left
+  // zero for the next decode, which then needs no clearing pass (sums_to_zero == NULL keeps them)
+  if (sums_to_zero) {
+    uint4* z = reinterpret_cast<uint4*>(sums_to_zero + (size_t)b * cells * 2);      // 16 bytes per bin
+    for (int i = blockIdx.x * kGraphThreads + tid; i < cells; i += gridDim.x * kGraphThreads) z[i] = make_uint4(0, 0, 0, 0);
+  }
   const int K = count_ptr[b];
   if (K < k_min || K > kNearMaxPeaks) return;
-  const int tid = threadIdx.x;
   const float* ref_img = ref_emb + (size_t)b * K_max * D;
   const float* cand_img = cand_emb + (size_t)b * K_max * D;
   const bool same = ref2 == cand2;
@@ -92,19 +98,32 @@ peak_graph_kernel(const float* __restrict__ ref_emb, const float* __restrict__ c
       s_keys[k] = key;
     }
     __syncthreads();
-    // the kNbrCap smallest keys in ascending order: a key's slot is the number of smaller keys (keys are distinct: k
-    // is part of them)
-    uint32_t* out = nbr + ((size_t)b * K_max + k0) * kNbrCap;
-    for (int k = tid; k < K; k += kGraphThreads) {
-      const uint32_t mine = s_keys[k];
-      int rank = 0;
-      for (int i = 0; i < Kpad; i += 4) {
-        const uint4 v = *reinterpret_cast<const uint4*>(&s_keys[i]);
-        rank += (v.x < mine) + (v.y < mine) + (v.z < mine) + (v.w < mine);
+    // the kNbrCap smallest keys in ascending order: a bitonic sort of the keys, padded with end marks to a power of two
+    // (keys are distinct -- k is part of them -- so the order is unique)
+    int n = kNbrCap;
+    while (n < K) n <<= 1;
+    for (int k = Kpad + tid; k < n; k += kGraphThreads) s_keys[k] = kNbrEnd;
+    __syncthreads();
+    // Thread t takes the pairs t, t + 256, ...: while the pair distance j is at most 32, the pairs of a warp lie in 64
+    // consecutive keys that no other warp touches, so those steps need no CTA-wide barrier.
+    for (int kk = 2; kk <= n; kk <<= 1) {
+      for (int j = kk >> 1; j > 0; j >>= 1) {
+        for (int t = tid; t < n / 2; t += kGraphThreads) {
+          const int i = 2 * t - (t & (j - 1));                 // the pair's lower index: bit j clear
+          const uint32_t a = s_keys[i], c = s_keys[i + j];
+          const bool ascending = (i & kk) == 0;
+          if ((a > c) == ascending) {
+            s_keys[i] = c;
+            s_keys[i + j] = a;
+          }
+        }
+        if (j > 32 || (j == 1 && kk >= 64)) __syncthreads();   // (the next step's j is kk: beyond the warp's keys)
+        else __syncwarp();
       }
-      if (rank < kNbrCap) out[rank] = mine;
     }
-    for (int j = K + tid; j < kNbrCap; j += kGraphThreads) out[j] = kNbrEnd;   // fewer candidates than entries
+    __syncthreads();
+    uint32_t* out = nbr + ((size_t)b * K_max + k0) * kNbrCap;
+    for (int r = tid; r < kNbrCap; r += kGraphThreads) out[r] = s_keys[r];
     __syncthreads();
   }
 }

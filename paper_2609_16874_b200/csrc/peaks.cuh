@@ -11,6 +11,31 @@ constexpr int kRefineChunk = 512;     // peaks whose refined positions are stage
 constexpr int kPeakStageWords = 8 * (kPeakThreads / 32);   // largest map (in bitmap words) that one CTA does alone
 constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared memory when one CTA does the image
 
+// Mean estimate of a peak on one axis, pooled over the 3x3 window of bins around it (`lin` is the peak's bin): the sum of
+// the fixed-point sums over 2^24 times the sum of the counts, in binary64.  `vote_at(i)` reads the count of bin i.
+template <typename VoteAt>
+__device__ __forceinline__ double window_mean(VoteAt vote_at, const long long* __restrict__ S, int lin, int bins_w,
+                                              int bins_h, int axis) {
+  const int cy = lin / bins_w, cx = lin - cy * bins_w;
+  long long s = 0, n = 0;
+#pragma unroll
+  for (int dy = -1; dy <= 1; ++dy) {
+#pragma unroll
+    for (int dx = -1; dx <= 1; ++dx) {
+      const int ny = cy + dy, nx = cx + dx;
+      if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
+      const int nlin = ny * bins_w + nx;
+      n += (long long)vote_at(nlin);
+      s += __ldcg(S + 2 * (size_t)nlin + axis);
+    }
+  }
+  return __ddiv_rn((double)s, __dmul_rn((double)n, 16777216.0));
+}
+// The refined centroid in pixel units: pixel centres sit at x = -1 + (2 col + 1) / W.
+__device__ __forceinline__ float mean_to_pixels(double m, int extent) {
+  return (float)__dmul_rn(__dadd_rn(__dmul_rn(__dadd_rn(m, 1.0), (double)extent), -1.0), 0.5);
+}
+
 // Phase 1 (every CTA): one thread per bin, one warp per 32 consecutive bins; the warp's ballot is one word
 // of the peak indicator bitmap (the paper's binary map H-bar, packed).  A bin is a peak iff V > T_v and it
 // beats each existing 8-neighbour: larger count, or equal count and lower linear index.
@@ -37,6 +62,9 @@ constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared me
 // its distance bounds are taken around.  `cell_peak` (with the pruned assignment): bin -> index of the peak whose 3x3
 // window holds it, -1 where there is none; `near_state`: that kernel's per-image words, zeroed here.
 //
+// `skip_rows`: the peaks' embeddings and centroids are left to peak_rows_kernel (launched next), which spreads them over
+// the GPU; this kernel's last CTA then ends with the peak list, the bin -> peak table and the counters.
+//
 // `staged` (only with one CTA per image; needs 4 * bins_w * bins_h bytes of dynamic shared memory): the CTA first
 // copies the whole vote map into shared memory with independent loads -- one round trip to L2 instead of one or two
 // per 32-bin word and warp iteration -- and keeps the bitmap and the head of the peak list there as well, so that
@@ -47,7 +75,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
              const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
              float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
              uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
-             long long* __restrict__ sums, int zero_sums, int staged, int refine_out,
+             long long* __restrict__ sums, int zero_sums, int staged, int refine_out, int skip_rows,
              float* __restrict__ ref_emb, int32_t* __restrict__ cell_peak, uint32_t* __restrict__ near_state) {
   extern __shared__ uint32_t s_map[];                 // [cells] when staged
   __shared__ uint32_t s_bm[kPeakStageWords];
@@ -124,8 +152,15 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   uint32_t* pv = peak_votes + (size_t)b * K_max;
   const int per = (words + kPeakThreads - 1) / kPeakThreads;
   const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+  // (eight words at a time, fetched before the first is used: a thread's words come one round trip apart otherwise)
   int local = 0;
-  for (int w = w0; w < w1; ++w) local += __popc(bitmap_at(w));
+  for (int w = w0; w < w1; w += 8) {
+    uint32_t v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w + u < w1) ? bitmap_at(w + u) : 0u;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) local += __popc(v[u]);
+  }
 
   __shared__ int s_warp[kPeakThreads / 32];
   __shared__ int s_total;
@@ -153,16 +188,22 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   int slot = s_warp[wid] + incl - local;
   const int total = s_total;
 
-  for (int w = w0; w < w1 && slot < K_max; ++w) {
-    uint32_t bits = bitmap_at(w);
-    while (bits && slot < K_max) {
-      const int bit = __ffs(bits) - 1;
-      bits &= bits - 1;
-      const int lin = w * 32 + bit;
-      pc[slot] = lin;
-      if (staged && slot < kPeakListStage) s_pc[slot] = lin;
-      pv[slot] = vote_at(lin);
-      ++slot;
+  for (int w = w0; w < w1 && slot < K_max && local > 0; w += 8) {     // (a slice without a peak is not read again)
+    uint32_t v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w + u < w1) ? bitmap_at(w + u) : 0u;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      uint32_t bits = v[u];
+      while (bits && slot < K_max) {
+        const int bit = __ffs(bits) - 1;
+        bits &= bits - 1;
+        const int lin = (w + u) * 32 + bit;
+        pc[slot] = lin;
+        if (staged && slot < kPeakListStage) s_pc[slot] = lin;
+        pv[slot] = vote_at(lin);
+        ++slot;
+      }
     }
   }
   const int count = min(total, K_max);
@@ -220,26 +261,9 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
       const int nk = min(kRefineChunk, count - k0);
       for (int i = tid; i < 2 * nk; i += kPeakThreads) {       // (peak, axis): pooled mean of the 3x3 window
         const int k = k0 + (i >> 1), axis = i & 1;
-        const int lin = cell_of(pc, k);
-        const int cy = lin / bins_w, cx = lin - cy * bins_w;
-        long long s = 0, n = 0;
-#pragma unroll
-        for (int dy = -1; dy <= 1; ++dy) {
-#pragma unroll
-          for (int dx = -1; dx <= 1; ++dx) {
-            const int ny = cy + dy, nx = cx + dx;
-            if (ny < 0 || ny >= bins_h || nx < 0 || nx >= bins_w) continue;
-            const int nlin = ny * bins_w + nx;
-            n += (long long)vote_at(nlin);
-            s += __ldcg(S + 2 * (size_t)nlin + axis);
-          }
-        }
-        const double m = __ddiv_rn((double)s, __dmul_rn((double)n, 16777216.0));
+        const double m = window_mean(vote_at, S, cell_of(pc, k), bins_w, bins_h, axis);
         s_mean[i] = m;
-        // pixel centres sit at x = -1 + (2 col + 1)/W
-        if (refine_out)
-          out_centroids[((size_t)b * K_max + k) * 2 + axis] =
-              (float)__dmul_rn(__dadd_rn(__dmul_rn(__dadd_rn(m, 1.0), (double)(axis ? H : W)), -1.0), 0.5);
+        if (refine_out) out_centroids[((size_t)b * K_max + k) * 2 + axis] = mean_to_pixels(m, axis ? H : W);
       }
       __syncthreads();
       for (int i = tid; i < 2 * F * nk; i += kPeakThreads) {   // (peak, axis, harmonic): sin and cos of pi 2^l mean
@@ -258,6 +282,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
       for (int i = tid; i < 2 * cells; i += kPeakThreads) S[i] = 0;
     if (refine_out) return;
   }
+  if (skip_rows) return;     // peak_rows_kernel writes the embeddings and the centroids
   for (int i = tid; i < count * D; i += kPeakThreads) {
     const int k = i / D, c = i - k * D;
     const int lin = cell_of(pc, k);
@@ -273,6 +298,57 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     float* o = out_centroids + ((size_t)b * K_max + k) * 2;
     o[0] = (float)(((x + 1.0) * (double)W - 1.0) * 0.5);
     o[1] = (float)(((y + 1.0) * (double)H - 1.0) * 0.5);
+  }
+}
+
+// gamma of the peaks' mean estimates as a kernel of its own, spread over the GPU: the binary64 sine and cosine of
+// 2F arguments per peak take the last CTA of peaks_kernel longer than everything else it does once an image has
+// hundreds of peaks.  A thread per (peak, axis, harmonic); `gm` [B][K_max][4F] receives gamma(mean) and, with
+// `refine_out`, out_centroids the means in pixel units (the same operations as in peaks_kernel).  F a power of two.
+constexpr int kRowsThreads = 128;
+__global__ void __launch_bounds__(kRowsThreads)
+peak_rows_kernel(const uint32_t* __restrict__ votes, const long long* __restrict__ sums, int bins_w, int bins_h, int K_max,
+                 int F, int H, int W, const int32_t* __restrict__ peak_cell, const int32_t* __restrict__ count_ptr,
+                 int refine_out, float* __restrict__ gm, float* __restrict__ out_centroids,
+                 const float* __restrict__ pal_w, const float* __restrict__ pal_h, float* __restrict__ peak_emb) {
+  grid_dependency_sync();
+  const int b = blockIdx.y;
+  const int cells = bins_w * bins_h;
+  const int count = count_ptr[b];
+  const uint32_t* V = votes + (size_t)b * cells;
+  const long long* S = sums + (size_t)b * cells * 2;
+  const int TP = 2 * F, D = 4 * F;                        // threads per peak (at most one warp)
+  const int lane = threadIdx.x & 31;
+  const int n_items = ((count * TP + 31) / 32) * 32;     // whole warps take part in the shuffle below
+  for (int i = blockIdx.x * kRowsThreads + threadIdx.x; i < n_items; i += gridDim.x * kRowsThreads) {
+    const int k = i / TP, r = i - k * TP;
+    const int axis = r / F, l = r - axis * F;
+    const bool have = k < count;
+    double m = 0.0;
+    const int lin = have ? peak_cell[(size_t)b * K_max + k] : 0;
+    if (have && l == 0) {
+      m = window_mean([&](int c) { return __ldcg(V + c); }, S, lin, bins_w, bins_h, axis);
+      if (refine_out) out_centroids[((size_t)b * K_max + k) * 2 + axis] = mean_to_pixels(m, axis ? H : W);
+    }
+    if (have && !refine_out) {
+      // the peak stays on its bin position: palette rows (Eq. 9) and the bin centre in pixel units
+      const int cy = lin / bins_w, cx = lin - cy * bins_w;
+      const int c = axis ? cy : cx, n = axis ? bins_h : bins_w;
+      const float2 pr = *reinterpret_cast<const float2*>((axis ? pal_h : pal_w) + (size_t)c * 2 * F + 2 * l);
+      *reinterpret_cast<float2*>(peak_emb + ((size_t)b * K_max + k) * D + axis * 2 * F + 2 * l) = pr;
+      if (l == 0) {
+        const double x = -1.0 + 2.0 * (double)(c + 1) / (double)(n + 1);
+        out_centroids[((size_t)b * K_max + k) * 2 + axis] = (float)(((x + 1.0) * (double)(axis ? H : W) - 1.0) * 0.5);
+      }
+    }
+    m = __shfl_sync(0xffffffffu, m, lane - l);             // from this (peak, axis)'s first thread
+    if (have) {
+      double sn, cs;
+      sincospi(scalbn(m, l), &sn, &cs);
+      float* o = gm + ((size_t)b * K_max + k) * D + axis * 2 * F + 2 * l;
+      o[0] = (float)sn;
+      o[1] = (float)cs;
+    }
   }
 }
 
