@@ -84,6 +84,11 @@ enum {
                                      withhold the arrival of each CTA's first tile, so that the consumers' bounded wait
                                      runs out, the kernel winds down and returns, and CPE_STATUS_TIMEOUT is set (the
                                      label map of that decode is incomplete)                                          */
+  CPE_FLAG_FUSE_PEAKS = 32768u,   /* small inputs (at most 2^20 pixels, vote maps of at most 8192 bins, no pruned
+                                     assignment): the voting kernel's last CTA of each image also searches the map
+                                     for the peaks, one kernel launch fewer per decode; same results.  Off by default:
+                                     the hand-over inside the kernel (ticket, fences) measured 2 to 4 us SLOWER per
+                                     decode than the separate launch it saves                                          */
   CPE_FLAG_SOFT_VOTE = 16384u,    /* vote as the paper prints it: the map is the real-valued histogram of Eq. 6,
                                      H(a, b) = sum over the participating pixels of exp(-d) with d of Eq. 4 (the sum
                                      that cpe_soft_votes computes, same accuracy), instead of the integer counts of the

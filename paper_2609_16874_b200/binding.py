@@ -38,6 +38,7 @@ CPE_FLAG_PRUNE_WALK_ONLY = 2048
 CPE_FLAG_TEST_STALL = 4096
 CPE_FLAG_PRUNE_ANY_SIZE = 8192
 CPE_FLAG_SOFT_VOTE = 16384
+CPE_FLAG_FUSE_PEAKS = 32768
 CPE_STATUS_PEAK_OVERFLOW, CPE_STATUS_NONFINITE, CPE_STATUS_INTERNAL, CPE_STATUS_TIMEOUT = 1, 2, 4, 8
 CPE_CNT_VOTING, CPE_CNT_NONFINITE, CPE_CNT_RAW_PEAKS, CPE_CNT_TRUNCATED, CPE_CNT_TAU_REJECTED = 0, 1, 2, 3, 4
 CPE_CNT_FILTER_PAIRS, CPE_CNT_RESCORED, CPE_CNT_FULL_SCORED, CPE_CNT_N = 5, 6, 7, 8

@@ -16,7 +16,6 @@
 #include "instance_masks.cuh"
 #include "launch.h"
 #include "layout.cuh"
-#include "peaks.cuh"
 
 namespace {
 thread_local int g_last_cuda = 0;
@@ -158,13 +157,9 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   if (pr) {
     // gamma of every peak's mean estimate (the bounds' reference points; the candidates too when they are refined),
     // a thread per (peak, axis, harmonic) over as many CTAs as the largest image can need
-    const int k_cap = std::min(p->max_instances, cpe::kNearMaxPeaks);
-    const int ctas = std::max(1, std::min((k_cap * 2 * F + cpe::kRowsThreads - 1) / cpe::kRowsThreads, 4 * sm_count()));
-    CPE_CUDA(launch_dependent(plain_launch(p), cpe::peak_rows_kernel, dim3((unsigned)ctas, (unsigned)B), cpe::kRowsThreads, 0,
-                              st, pr->votes, pr->sums, p->bins_w, p->bins_h, p->max_instances, F, pr->H, pr->W,
-                              pr->peak_cell, count, pr->refine_out, pr->gamma_out, pr->out_centroids, pr->pal_w, pr->pal_h,
-                              pr->peak_emb));
-    CPE_CUDA(cudaGetLastError());
+    rc = cpe::host::launch_peak_rows(st, B, F, p, pr->votes, pr->sums, pr->H, pr->W, pr->peak_cell, count, pr->refine_out,
+                                     pr->gamma_out, pr->out_centroids, pr->pal_w, pr->pal_h, pr->peak_emb);
+    if (rc) return rc;
     rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->ref_h,
                                       pr->cand_h, pr->nbr, pr->sums_to_zero, cells);
     if (rc) return rc;
@@ -280,41 +275,62 @@ int decode_impl(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int 
     if (sums) cudaMemsetAsync(ws + L.sums, 0, L.sums_end - L.sums, st);
     return code;
   };
+  // Stage 3's arguments (the voting kernel takes them along when it runs the search itself)
+  cpe::PeakArgs pk{};
+  pk.votes = votes;
+  pk.bins_w = p->bins_w;
+  pk.bins_h = p->bins_h;
+  pk.words = L.words;
+  pk.bitmap = bitmap;
+  pk.K_max = p->max_instances;
+  pk.F = F;
+  pk.H = H;
+  pk.W = W;
+  pk.pal_w = pal_w;
+  pk.pal_h = pal_h;
+  pk.peak_cell = peak_cell;
+  pk.peak_votes = peak_votes;
+  pk.peak_emb = peak_emb;
+  pk.out_centroids = out_centroids;
+  pk.out_count = out_count;
+  pk.acc = acc;
+  pk.counters = counters;
+  pk.status = status;
+  pk.sums = L.prune ? nullptr : sums;
+  pk.zero_sums = sums_cleared_by_peaks ? 1 : 0;
+  pk.staged = one_peak_cta ? 1 : 0;
+  pk.refine_out = refine ? 1 : 0;
+  pk.skip_rows = L.prune ? 1 : 0;
+  pk.ref_emb = L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr;
+  pk.cell_peak = L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr;
+  pk.near_state = pr.near_state;
   // Vote: by default the hard vote (each pixel's centroid estimate, one count).  With CPE_FLAG_SOFT_VOTE the map holds
   // the binary32 histogram of Eq. 6 instead: non-negative binary32 values order like their bit patterns and 0.0f is
   // all-zero bits, so the zeroing conventions and the peak kernel's comparisons carry over to it unchanged.
   const bool soft = (p->flags & CPE_FLAG_SOFT_VOTE) != 0;
-  uint32_t t_v = (uint32_t)p->vote_threshold;
+  pk.T_v = (uint32_t)p->vote_threshold;
+  pk.strict = soft ? 1 : 0;
+  bool peaks_done = false;
   if (soft) {
     if ((uintptr_t)emb % 16 || HW % 8) return CPE_ERR_ALIGN;
-    memcpy(&t_v, &p->soft_threshold, sizeof t_v);
+    memcpy(&pk.T_v, &p->soft_threshold, sizeof pk.T_v);
     // the soft-vote kernel only ever ORs into the status words; the peak kernel then ORs too
     CPE_CUDA(cudaMemsetAsync(status, 0, sizeof(uint32_t) * (size_t)B, st));
     rc = cpe::host::launch_soft_votes(st, emb, fg, B, HW, F, p, pal_w, pal_h, reinterpret_cast<float*>(votes), status, acc);
   } else {
+    // small maps without the pruned chain: the voting kernel's last CTA of an image searches the map itself
+    peaks_done = one_peak_cta && !L.prune && cpe::host::vote_can_fuse_peaks(B, HW, L.words, p);
     rc = cpe::host::launch_decode_vote(st, emb, fg, B, HW, F, p, votes, acc, sums,
-                                       L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr);
+                                       L.prune ? reinterpret_cast<uint32_t*>(ws + L.pix_cell) : nullptr,
+                                       peaks_done ? &pk : nullptr);
   }
   if (rc) return fail_after_votes(rc);
   if ((rc = debug_stage_check(st, "decode_vote"))) return rc;
 
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_PEAKS], st));
-  {
-    const int warps_per_cta = cpe::kPeakThreads / 32;
-    // small maps: one CTA per image does both phases without the cross-CTA hand-over
-    const int ctas = one_peak_cta ? 1 : (L.words + warps_per_cta - 1) / warps_per_cta;
-    dim3 grid((unsigned)ctas, (unsigned)B);
-    // one CTA per image: it works on a copy of the vote map in shared memory (at most 32 KB)
-    const size_t map_smem = one_peak_cta ? 4 * (size_t)L.cells : 0;
-    cudaError_t e = launch_dependent(plain_launch(p), cpe::peaks_kernel, grid, cpe::kPeakThreads, map_smem, st, votes,
-                                     p->bins_w, p->bins_h, L.words, t_v, soft ? 1 : 0, bitmap, p->max_instances, F,
-                                     H, W, pal_w, pal_h, peak_cell, peak_votes, peak_emb, out_centroids, out_count, acc,
-                                     counters, status, L.prune ? nullptr : sums, sums_cleared_by_peaks ? 1 : 0,
-                                     one_peak_cta ? 1 : 0, refine ? 1 : 0, L.prune ? 1 : 0,
-                                     L.prune ? reinterpret_cast<float*>(ws + L.ref_emb) : nullptr,
-                                     L.prune ? reinterpret_cast<int32_t*>(ws + L.cell_peak) : nullptr, pr.near_state);
-    if (e == cudaSuccess) e = cudaGetLastError();
-    if (e != cudaSuccess) return fail_after_votes(cuda_fail(e));
+  if (!peaks_done) {
+    rc = cpe::host::launch_peaks(st, B, p, pk);
+    if (rc) return fail_after_votes(rc);
   }
   if ((rc = debug_stage_check(st, "peaks"))) return rc;
   if (ev) CPE_CUDA(cudaEventRecord(ev[CPE_STAGE_LISTS], st));

@@ -11,6 +11,7 @@
 #pragma once
 
 #include "cpe_common.cuh"
+#include "peaks.cuh"
 
 namespace cpe {
 
@@ -46,6 +47,8 @@ constexpr float kRefineScale = 16777216.0f;  // 2^24
 
 // What a voting kernel records besides the vote map (template parameter MODE, a bit set):
 constexpr int kVoteSums = 1;    // the per-bin fixed-point sums of the estimates
+constexpr int kVotePeaks = 4;   // the last CTA of an image to finish also searches its (small) vote map for the peaks:
+                                // peaks_image with one CTA per image, instead of a launch of peaks_kernel
 constexpr int kVoteCells = 2;   // every participating pixel's bin (uint32 [B][H*W]; 0xffffffff: it did not vote), which the
                                 // pruned assignment looks its candidate list up with
 
@@ -70,6 +73,23 @@ __device__ __forceinline__ void vote_sums_add(long long* __restrict__ sums_img, 
                 (unsigned long long)(long long)sy);
     }
   }
+}
+
+// With kVotePeaks: called by every thread of a voting CTA after its votes and counts have gone to global memory.  The
+// last CTA of image b to get here (ticket counter, no waiting) runs the peak search on the finished map.
+template <int THREADS>
+__device__ __forceinline__ void vote_then_peaks(const PeakArgs& pa, int b, uint32_t* acc, uint32_t* s_map) {
+  __shared__ int s_vote_last;
+  __threadfence();              // this CTA's votes are visible device-wide before its ticket is taken
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t ticket = atomicAdd(&acc[b * kAccStride + kAccTicket], 1u);
+    s_vote_last = ticket == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_vote_last) return;
+  __threadfence();              // and the other CTAs' votes are visible to this one
+  peaks_image<THREADS>(pa, b, 0, 1, s_map);      // (leaves the ticket zero for the next decode)
 }
 
 // Compacts the participating pixels of the CTA's span into s_list (offsets within the span, ascending).
@@ -131,9 +151,11 @@ template <typename T, int FT, int MODE>
 __global__ void __launch_bounds__(kVoteThreads)
 decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int F_rt, int levels,
                    int bins_w, int bins_h, int vec_mask, uint32_t* __restrict__ votes,
-                   uint32_t* __restrict__ acc, long long* __restrict__ sums, uint32_t* __restrict__ pix_cell) {
+                   uint32_t* __restrict__ acc, long long* __restrict__ sums, uint32_t* __restrict__ pix_cell,
+                   const PeakArgs pa) {
   constexpr bool REFINE = (MODE & kVoteSums) != 0;
   constexpr bool CELLS = (MODE & kVoteCells) != 0;
+  extern __shared__ uint32_t s_vote_map[];       // with kVotePeaks: room for the vote map
   grid_dependency_sync();
   const int F = FT > 0 ? FT : F_rt;
   const int Fu = (levels > 0 && levels < F) ? levels : F;
@@ -251,6 +273,7 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
   }
   if (tid == 0 && s_voting) atomicAdd(&acc[b * kAccStride + kAccVoting], s_voting);
   if (tid == 0 && s_nonfinite) atomicAdd(&acc[b * kAccStride + kAccNonfinite], s_nonfinite);
+  if constexpr ((MODE & kVotePeaks) != 0) vote_then_peaks<kVoteThreads>(pa, b, acc, s_vote_map);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -265,15 +288,17 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 constexpr int kVecGroupsMax = 256;   // groups per CTA: 256, 128 or 64 (template parameter GROUPS; the launcher takes the
                                      // largest that still gives a full wave of CTAs -- small images are latency-bound
                                      // and want many short CTAs, large ones want fewer fixed costs)
-constexpr int kVecLevelBatch = 2;  // harmonics whose plane loads are in flight together (2 loads each)
+// harmonics whose plane loads are in flight together (2 loads each): what leaves room for four CTAs per SM
+template <typename T> __host__ __device__ constexpr int vec_level_batch() { return sizeof(T) == 4 ? 4 : 2; }
 
 template <typename T, int FT, int MODE, int GROUPS>
 __global__ void __launch_bounds__(kVoteThreads, 4)
 decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int HW, int levels, int bins_w,
                        int bins_h, uint32_t* __restrict__ votes, uint32_t* __restrict__ acc,
-                       long long* __restrict__ sums, uint32_t* __restrict__ pix_cell) {
+                       long long* __restrict__ sums, uint32_t* __restrict__ pix_cell, const PeakArgs pa) {
   constexpr bool REFINE = (MODE & kVoteSums) != 0;
   constexpr bool CELLS = (MODE & kVoteCells) != 0;
+  extern __shared__ uint32_t s_vote_map[];       // with kVotePeaks: room for the vote map
   grid_dependency_sync();
   constexpr int VEC = Elem<T>::kVec;
   constexpr int F = FT;
@@ -362,7 +387,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
       // The plane loads of a batch of harmonics are in flight together, kept raw in registers.  The loop over the
       // batches is not unrolled: the body for one batch (VEC pixels x LB harmonics) then stays in the instruction
       // cache, which the fully unrolled chain of all F harmonics overflowed.
-      constexpr int LB = F < kVecLevelBatch ? F : kVecLevelBatch;
+      constexpr int LB = F < vec_level_batch<T>() ? F : vec_level_batch<T>();
       const T* ptr = src;
 #pragma unroll 1
       for (int l0 = 0; l0 < F; l0 += LB, ptr += (size_t)(2 * LB) * plane) {
@@ -460,6 +485,7 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
   }
   if (tid == 0 && s_voting) atomicAdd(&acc[b * kAccStride + kAccVoting], s_voting);
   if (tid == 0 && s_nonfinite) atomicAdd(&acc[b * kAccStride + kAccNonfinite], s_nonfinite);
+  if constexpr ((MODE & kVotePeaks) != 0) vote_then_peaks<kVoteThreads>(pa, b, acc, s_vote_map);
 }
 
 }  // namespace cpe

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "cpe.h"
+#include "cpe_common.cuh"
 
 namespace cpe {
 namespace host {
@@ -57,9 +58,20 @@ cudaError_t launch_dependent(bool plain, void (*kern)(KArgs...), dim3 grid, int 
 
 inline bool plain_launch(const cpe_params* p) { return (p->flags & CPE_FLAG_NO_PDL) != 0; }
 
-// ---- stage 1+2 (launch_vote.cu).  sums: per-bin fixed-point sums or NULL; pix_cell: per-pixel bin or NULL.
+// ---- stage 1+2 (launch_vote.cu).  sums: per-bin fixed-point sums or NULL; pix_cell: per-pixel bin or NULL;
+// fused_peaks: not NULL = the last CTA of each image also runs the peak search (stage 3) on its small map, and
+// launch_peaks is not called.
 int launch_decode_vote(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,
-                       uint32_t* votes, uint32_t* acc, long long* sums, uint32_t* pix_cell);
+                       uint32_t* votes, uint32_t* acc, long long* sums, uint32_t* pix_cell,
+                       const cpe::PeakArgs* fused_peaks);
+// Whether launch_decode_vote can take stage 3 along for this problem.
+bool vote_can_fuse_peaks(int B, int HW, int words, const cpe_params* p);
+
+// ---- stage 3 (launch_vote.cu): the peak search, and (pruned assignment) the kernel that writes the peaks' rows
+int launch_peaks(cudaStream_t st, int B, const cpe_params* p, const cpe::PeakArgs& a);
+int launch_peak_rows(cudaStream_t st, int B, int F, const cpe_params* p, const uint32_t* votes, const long long* sums, int H,
+                     int W, const int32_t* peak_cell, const int32_t* count, int refine_out, float* gamma_out,
+                     float* out_centroids, const float* pal_w, const float* pal_h, float* peak_emb);
 
 // ---- stage 4+5, tensor-core filtered kernels (launch_filter.cu): images with at least k_min peaks.
 int launch_assign_filtered(cudaStream_t st, const void* emb, const uint8_t* fg, int B, int HW, int F, const cpe_params* p,

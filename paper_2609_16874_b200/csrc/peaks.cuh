@@ -8,7 +8,6 @@ namespace cpe {
 
 constexpr int kPeakThreads = 1024;   // wide CTAs: the last one of an image does the whole compaction
 constexpr int kRefineChunk = 512;     // peaks whose refined positions are staged in shared memory at a time
-constexpr int kPeakStageWords = 8 * (kPeakThreads / 32);   // largest map (in bitmap words) that one CTA does alone
 constexpr int kPeakListStage = 1024;  // peak-list entries mirrored in shared memory when one CTA does the image
 
 // Mean estimate of a peak on one axis, pooled over the 3x3 window of bins around it (`lin` is the peak's bin): the sum of
@@ -69,19 +68,34 @@ __device__ __forceinline__ float mean_to_pixels(double m, int extent) {
 // copies the whole vote map into shared memory with independent loads -- one round trip to L2 instead of one or two
 // per 32-bin word and warp iteration -- and keeps the bitmap and the head of the peak list there as well, so that
 // the dependent steps of this latency-bound kernel stay on the SM.
-__global__ void __launch_bounds__(kPeakThreads)
-peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int words, uint32_t T_v, int strict,
-             uint32_t* __restrict__ bitmap, int K_max, int F, int H, int W, const float* __restrict__ pal_w,
-             const float* __restrict__ pal_h, int32_t* __restrict__ peak_cell, uint32_t* __restrict__ peak_votes,
-             float* __restrict__ peak_emb, float* __restrict__ out_centroids, int32_t* __restrict__ out_count,
-             uint32_t* __restrict__ acc, uint32_t* __restrict__ counters, uint32_t* __restrict__ status,
-             long long* __restrict__ sums, int zero_sums, int staged, int refine_out, int skip_rows,
-             float* __restrict__ ref_emb, int32_t* __restrict__ cell_peak, uint32_t* __restrict__ near_state) {
-  extern __shared__ uint32_t s_map[];                 // [cells] when staged
+// The search for image b by CTA `cta` of `n_ctas` (THREADS threads each); s_map: [cells] words of shared memory when
+// a.staged.  peaks_kernel calls it with its grid's coordinates; the voting kernel's last CTA of an image calls it with
+// n_ctas = 1 when the map is small (one launch fewer).
+template <int THREADS>
+__device__ __forceinline__ void peaks_image(const PeakArgs& a, int b, int cta, int n_ctas, uint32_t* s_map) {
+  const uint32_t* __restrict__ votes = a.votes;
+  const int bins_w = a.bins_w, bins_h = a.bins_h, words = a.words;
+  const uint32_t T_v = a.T_v;
+  const int strict = a.strict;
+  uint32_t* __restrict__ bitmap = a.bitmap;
+  const int K_max = a.K_max, F = a.F, H = a.H, W = a.W;
+  const float* __restrict__ pal_w = a.pal_w;
+  const float* __restrict__ pal_h = a.pal_h;
+  int32_t* __restrict__ peak_cell = a.peak_cell;
+  uint32_t* __restrict__ peak_votes = a.peak_votes;
+  float* __restrict__ peak_emb = a.peak_emb;
+  float* __restrict__ out_centroids = a.out_centroids;
+  int32_t* __restrict__ out_count = a.out_count;
+  uint32_t* __restrict__ acc = a.acc;
+  uint32_t* __restrict__ counters = a.counters;
+  uint32_t* __restrict__ status = a.status;
+  long long* __restrict__ sums = a.sums;
+  const int zero_sums = a.zero_sums, staged = a.staged, refine_out = a.refine_out, skip_rows = a.skip_rows;
+  float* __restrict__ ref_emb = a.ref_emb;
+  int32_t* __restrict__ cell_peak = a.cell_peak;
+  uint32_t* __restrict__ near_state = a.near_state;
   __shared__ uint32_t s_bm[kPeakStageWords];
   __shared__ int s_pc[kPeakListStage];
-  grid_dependency_sync();
-  const int b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int cells = bins_w * bins_h;
   const uint32_t* V = votes + (size_t)b * cells;
@@ -93,15 +107,15 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     acc_nonfinite = __ldcg(&acc[b * kAccStride + kAccNonfinite]);
   }
   if (staged) {
-    for (int i = tid; i < cells; i += kPeakThreads) s_map[i] = __ldcg(V + i);
+    for (int i = tid; i < cells; i += THREADS) s_map[i] = __ldcg(V + i);
     __syncthreads();
   }
   auto vote_at = [&](int i) -> uint32_t { return staged ? s_map[i] : __ldg(V + i); };
   auto bitmap_at = [&](int w) -> uint32_t { return staged ? s_bm[w] : __ldcg(bm + w); };
   auto cell_of = [&](const int32_t* list, int k) -> int { return (staged && k < kPeakListStage) ? s_pc[k] : list[k]; };
 
-  // ---- phase 1 (a CTA takes the words blockIdx.x*32 + wid, then strides by the grid: one CTA per image for small maps)
-  for (int warp = blockIdx.x * (kPeakThreads / 32) + wid; warp < words; warp += gridDim.x * (kPeakThreads / 32)) {
+  // ---- phase 1 (a CTA takes the words cta*32 + wid, then strides by the grid: one CTA per image for small maps)
+  for (int warp = cta * (THREADS / 32) + wid; warp < words; warp += n_ctas * (THREADS / 32)) {
     const int lin = warp * 32 + lane;
     bool peak = false;
     if (lin < cells) {
@@ -132,13 +146,13 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   }
 
   // ---- which CTA of this image is the last one?  (with one CTA per image there is nothing to ask)
-  if (gridDim.x > 1) {
+  if (n_ctas > 1) {
     __shared__ int s_last;
     __threadfence();          // this CTA's bitmap words are visible device-wide before its ticket is taken
     __syncthreads();
     if (tid == 0) {
       const uint32_t ticket = atomicAdd(&acc[b * kAccStride + kAccTicket], 1u);
-      s_last = ticket == gridDim.x - 1;
+      s_last = ticket == (uint32_t)(n_ctas - 1);
     }
     __syncthreads();
     if (!s_last) return;
@@ -150,7 +164,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   // ---- phase 2
   int32_t* pc = peak_cell + (size_t)b * K_max;
   uint32_t* pv = peak_votes + (size_t)b * K_max;
-  const int per = (words + kPeakThreads - 1) / kPeakThreads;
+  const int per = (words + THREADS - 1) / THREADS;
   const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
   // (eight words at a time, fetched before the first is used: a thread's words come one round trip apart otherwise)
   int local = 0;
@@ -162,7 +176,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     for (int u = 0; u < 8; ++u) local += __popc(v[u]);
   }
 
-  __shared__ int s_warp[kPeakThreads / 32];
+  __shared__ int s_warp[THREADS / 32];
   __shared__ int s_total;
   int incl = local;
 #pragma unroll
@@ -172,16 +186,17 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
   }
   if (lane == 31) s_warp[wid] = incl;
   __syncthreads();
-  if (wid == 0) {                      // exclusive scan of the 32 warp totals by the first warp
-    static_assert(kPeakThreads / 32 == 32, "one lane per warp total");
-    const int mine = s_warp[lane];
+  if (wid == 0) {                      // exclusive scan of the warp totals by the first warp
+    constexpr int NW = THREADS / 32;
+    static_assert(NW <= 32, "one lane per warp total");
+    const int mine = lane < NW ? s_warp[lane] : 0;
     int inc = mine;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, inc, d);
       if (lane >= d) inc += t;
     }
-    s_warp[lane] = inc - mine;
+    if (lane < NW) s_warp[lane] = inc - mine;
     if (lane == 31) s_total = inc;
   }
   __syncthreads();
@@ -239,7 +254,7 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     // every bin of a peak's 3x3 window names that peak (two peaks are never neighbours, so a peak's own bin is in no
     // other window; a bin between two peaks gets either)
     int32_t* cp = cell_peak + (size_t)b * cells;
-    for (int k = tid; k < count; k += kPeakThreads) {
+    for (int k = tid; k < count; k += THREADS) {
       const int lin = cell_of(pc, k);
       const int cy = lin / bins_w, cx = lin - cy * bins_w;
 #pragma unroll
@@ -259,14 +274,14 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     long long* S = sums + (size_t)b * cells * 2;
     for (int k0 = 0; k0 < count; k0 += kRefineChunk) {
       const int nk = min(kRefineChunk, count - k0);
-      for (int i = tid; i < 2 * nk; i += kPeakThreads) {       // (peak, axis): pooled mean of the 3x3 window
+      for (int i = tid; i < 2 * nk; i += THREADS) {       // (peak, axis): pooled mean of the 3x3 window
         const int k = k0 + (i >> 1), axis = i & 1;
         const double m = window_mean(vote_at, S, cell_of(pc, k), bins_w, bins_h, axis);
         s_mean[i] = m;
         if (refine_out) out_centroids[((size_t)b * K_max + k) * 2 + axis] = mean_to_pixels(m, axis ? H : W);
       }
       __syncthreads();
-      for (int i = tid; i < 2 * F * nk; i += kPeakThreads) {   // (peak, axis, harmonic): sin and cos of pi 2^l mean
+      for (int i = tid; i < 2 * F * nk; i += THREADS) {   // (peak, axis, harmonic): sin and cos of pi 2^l mean
         const int kk = i / (2 * F), r = i - kk * 2 * F;
         const int axis = r / F, l = r - axis * F;
         double sn, cs;
@@ -279,17 +294,17 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     }
     // small maps (this CTA does the whole image): the sums have no reader left and are left zero for the next decode
     if (zero_sums)
-      for (int i = tid; i < 2 * cells; i += kPeakThreads) S[i] = 0;
+      for (int i = tid; i < 2 * cells; i += THREADS) S[i] = 0;
     if (refine_out) return;
   }
   if (skip_rows) return;     // peak_rows_kernel writes the embeddings and the centroids
-  for (int i = tid; i < count * D; i += kPeakThreads) {
+  for (int i = tid; i < count * D; i += THREADS) {
     const int k = i / D, c = i - k * D;
     const int lin = cell_of(pc, k);
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     pe[i] = (c < 2 * F) ? pal_w[cx * 2 * F + c] : pal_h[cy * 2 * F + (c - 2 * F)];
   }
-  for (int k = tid; k < count; k += kPeakThreads) {
+  for (int k = tid; k < count; k += THREADS) {
     const int lin = cell_of(pc, k);
     const int cy = lin / bins_w, cx = lin - cy * bins_w;
     // bin position -1 + 2i/(n+1), i = c+1 (Eq. 9); pixel centres sit at x = -1 + (2 col + 1)/W
@@ -299,6 +314,13 @@ peaks_kernel(const uint32_t* __restrict__ votes, int bins_w, int bins_h, int wor
     o[0] = (float)(((x + 1.0) * (double)W - 1.0) * 0.5);
     o[1] = (float)(((y + 1.0) * (double)H - 1.0) * 0.5);
   }
+}
+
+__global__ void __launch_bounds__(kPeakThreads)
+peaks_kernel(const PeakArgs a) {
+  extern __shared__ uint32_t s_peak_map[];            // [cells] when a.staged
+  grid_dependency_sync();
+  peaks_image<kPeakThreads>(a, (int)blockIdx.y, (int)blockIdx.x, (int)gridDim.x, s_peak_map);
 }
 
 // gamma of the peaks' mean estimates as a kernel of its own, spread over the GPU: the binary64 sine and cosine of

@@ -216,3 +216,35 @@ def test_refined_edge_cases_empty_truncated_nonfinite_and_border_peaks():
     assert set((cells % bw).tolist()) <= {0, bw - 1} and set((cells // bw).tolist()) <= {0, bh - 1}
     gpu = run_refined(emb, fg, bw, bh, T_v=8, K_max=8)
     compare_refined(gpu, ora)
+
+
+FUSE_CASES = [
+    ("c1", dict()),                                                        # vector-load vote kernel, fp32
+    ("c1", dict(H=67, W=93)),                                              # scalar-load vote kernel
+    ("c2", dict(H=192, W=256, K=12)),
+    ("c3", dict(H=99, W=121, K=8, bins_w=64, bins_h=32)),                  # fp16, scalar path
+    ("c4", dict(B=3, H=160, W=168, K=30, bins_w=40, bins_h=40)),           # batch: one ticket per image
+    ("c5", dict(H=256, W=256, K=40, bins_w=96, bins_h=80)),                # F = 16, 7680 bins
+]
+
+
+@pytest.mark.parametrize("name,over", FUSE_CASES, ids=[f"{n}-{i}" for i, (n, _) in enumerate(FUSE_CASES)])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_peak_search_inside_the_voting_kernel_gives_the_same_decode(name, over, mode):
+    """CPE_FLAG_FUSE_PEAKS: the last voting CTA of an image runs stage 3.  Refined and plain decodes against the oracle,
+    twice in a row (the ticket and the accumulators must be left zero), with an image without participating pixels."""
+    from gpu_util import compare_front, run_gpu
+    cfg = wl.scaled(wl.CONFIGS[name], **over)
+    fr = wl.make_frame(cfg, 1)
+    emb, fg = fr["emb"], fr["fg"].copy()
+    if cfg.B > 1:
+        fg[1] = 0
+    ora = oracle.decode_refined(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    gpu = run_refined(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, mode=mode, flags=cb.CPE_FLAG_FUSE_PEAKS)
+    compare_refined(gpu, ora)
+    plain = oracle.decode(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max)
+    for keep in (True, False):
+        g = run_gpu(emb, fg, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau, cfg.K_max, 0, True, mode, keep_votes=keep,
+                    flags=cb.CPE_FLAG_FUSE_PEAKS)
+        compare_front(g, plain, cfg.F, cfg.bins_w, cfg.bins_h)
+        compare_labels(g["labels"], g["best"], g["second"], plain["labels"], plain["best"], plain["second"])
