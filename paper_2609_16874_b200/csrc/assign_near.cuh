@@ -765,8 +765,8 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
   near_flush_counters(state, n_rejected, n_pairs, n_multi, n_full);
 }
 
-// The pixels that the walk left over: every peak, one warp per pixel (near_full_scan_warp), the queue dealt out
-// warp by warp so that a run of such pixels spreads over the whole grid.
+// The pixels that the walk left over are scored against every peak: a whole CTA per pixel while there are fewer pixels
+// than CTAs, else a thread per pixel with the rows staged in shared memory.
 template <typename T, int FT>
 __global__ void __launch_bounds__(kNearThreads)
 assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const float* __restrict__ cand2,
@@ -832,13 +832,51 @@ assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
       __syncthreads();
     }
   } else {
-    const int warp = blockIdx.x * kWarps + wid, n_warps = gridDim.x * kWarps;
-    for (int i = warp; i < n_h; i += n_warps) {
-      const size_t n = hard_q[(size_t)b * q_cap + i];
-      float d1, d2;
-      int k1;
-      near_full_scan_warp<T, D, false>(emb + (size_t)b * D * plane + n, plane, K, cand_img, d1, d2, k1, lane, 32);
-      if (lane == 0) finish(n, d1, k1);
+    // Many pixels (an instance without a peak of its own sends all of its pixels here): the all-pairs scheme, a thread
+    // per pixel with the pixel's values in registers while the candidate rows pass through shared memory in chunks.
+    // Peaks in ascending k with a strict comparison: the lowest k keeps an exact tie, as in the scans above.
+    constexpr int kChunk = 32;
+    __shared__ __align__(16) float s_rows[kChunk * D];
+    const float inf = __int_as_float(0x7f800000);
+    for (int base = blockIdx.x * kNearThreads; base < n_h; base += gridDim.x * kNearThreads) {   // uniform per CTA
+      const int i = base + (int)threadIdx.x;
+      const bool have = i < n_h;
+      const size_t n = have ? hard_q[(size_t)b * q_cap + i] : 0;
+      float2 e2[D / 2];
+      if (have) {
+        const T* p = emb + (size_t)b * D * plane + n;
+#pragma unroll
+        for (int c = 0; c < D / 2; ++c) {
+          e2[c].x = Elem<T>::load1(p + (size_t)c * plane);
+          e2[c].y = Elem<T>::load1(p + (size_t)(D / 2 + c) * plane);
+        }
+      }
+      float d1 = inf, bound2 = inf;
+      int k1 = -1;
+      for (int k0 = 0; k0 < K; k0 += kChunk) {
+        const int kn = min(kChunk, K - k0);
+        __syncthreads();
+        for (int j = threadIdx.x; j < kn * (D / 4); j += kNearThreads)
+          reinterpret_cast<float4*>(s_rows)[j] = __ldg(reinterpret_cast<const float4*>(cand_img + (size_t)k0 * D) + j);
+        __syncthreads();
+        if (have) {
+          int kk = 0;
+          for (; kk + 4 <= kn; kk += 4) {
+            float d[4];
+            score_direct4<D>(e2, reinterpret_cast<const float2*>(s_rows + kk * D), bound2, d);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (d[j] < d1) { d1 = d[j]; k1 = k0 + kk + j; }
+            bound2 = d1 * d1 * (1.0f + 1e-6f);
+          }
+          for (; kk < kn; ++kk) {
+            const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(s_rows + kk * D), bound2);
+            if (d < d1) { d1 = d; k1 = k0 + kk; }
+            bound2 = d1 * d1 * (1.0f + 1e-6f);
+          }
+        }
+      }
+      if (have) finish(n, d1, k1);
     }
   }
   near_flush_counters(state, n_rejected, n_full * (uint32_t)K, 0u, n_full);
