@@ -381,9 +381,15 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
     for (int j = 0; j < VEC; ++j) p[j] = 0.0f;   // the first harmonic's step from 0 returns its own estimate u
     uint32_t okbits = (1u << VEC) - 1u;
     if (have) {
+      // validity accumulators: binary32 inputs fold |s| + |c| per pixel (fold_finite); binary16 inputs are finite iff
+      // every element is (their sums cannot overflow binary32), so the raw pairs go through a packed multiply by zero
+      // that turns an infinity or a NaN into a NaN that sticks -- half the instructions
       float fin[VEC];
+      __half2 fin2[VEC / 2];
 #pragma unroll
       for (int j = 0; j < VEC; ++j) fin[j] = 0.0f;
+#pragma unroll
+      for (int j = 0; j < VEC / 2; ++j) fin2[j] = __float2half2_rn(0.0f);
       // The plane loads of a batch of harmonics are in flight together, kept raw in registers.  The loop over the
       // batches is not unrolled: the body for one batch (VEC pixels x LB harmonics) then stays in the instruction
       // cache, which the fully unrolled chain of all F harmonics overflowed.
@@ -399,8 +405,19 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
           float s[VEC], c[VEC];
           unpack_vec<T>(raw[2 * ll], s);
           unpack_vec<T>(raw[2 * ll + 1], c);
+          if constexpr (sizeof(T) == 2) {
+            const uint32_t ws[4] = {raw[2 * ll].x, raw[2 * ll].y, raw[2 * ll].z, raw[2 * ll].w};
+            const uint32_t wc[4] = {raw[2 * ll + 1].x, raw[2 * ll + 1].y, raw[2 * ll + 1].z, raw[2 * ll + 1].w};
+            const __half2 zero2 = __float2half2_rn(0.0f);
 #pragma unroll
-          for (int j = 0; j < VEC; ++j) fin[j] = fold_finite(fin[j], s[j], c[j]);
+            for (int j = 0; j < VEC / 2; ++j) {
+              fin2[j] = __hfma2(*reinterpret_cast<const __half2*>(&ws[j]), zero2, fin2[j]);
+              fin2[j] = __hfma2(*reinterpret_cast<const __half2*>(&wc[j]), zero2, fin2[j]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) fin[j] = fold_finite(fin[j], s[j], c[j]);
+          }
           if (l0 + ll < Fu) {
             // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
 #pragma unroll
@@ -417,7 +434,9 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
 #pragma unroll
       for (int j = 0; j < VEC; ++j) {
         p[j] = __fmul_rn(p[j], unscale);
-        if (fin[j] != fin[j]) okbits &= ~(1u << j);
+        bool bad = fin[j] != fin[j];
+        if constexpr (sizeof(T) == 2) bad = (j & 1) ? __hisnan(__high2half(fin2[j / 2])) : __hisnan(__low2half(fin2[j / 2]));
+        if (bad) okbits &= ~(1u << j);
       }
     }
     // swap with the partner lane: afterwards every lane knows both coordinates of its half of the pixels
