@@ -136,7 +136,7 @@ def algorithmic_bytes(cfg, fg_pixels: int, pruned: bool):
 STAGE_KERNELS = {
     "decode_vote": "decode_vote_vec_kernel",
     "peaks": "peaks_kernel",
-    "lists": "peak_graph_kernel",
+    "lists": "peak_rows_kernel + peak_graph_kernel",
     "assign": "assign_near_stream_kernel + assign_near_walk_kernel + assign_near_hard_kernel (pruned) / "
               "assign_kernel (few peaks) / assign_filter_kernel (handed on)",
 }
