@@ -467,6 +467,17 @@ def run_ours(args, cfg):
             line["launch_floor"] = measure_launch_floor(wl.CONFIGS["c2"], 200, 10, dev)
         except Exception as exc:
             line["launch_floor"] = {"error": repr(exc)}
+        try:   # the decode with the paper's own vote (Eq. 5-6, strict maxima, Eq. 7-8)
+            sd = {}
+            for n in ("c1", "c2"):
+                thr = soft_threshold_for(wl.CONFIGS[n], dev)
+                r = measure_other(wl.CONFIGS[n], 40, 5, dev, soft_threshold=thr)
+                r["workload"] += ("; vote mode: soft (CPE_FLAG_SOFT_VOTE, soft_threshold %.4g = 0.3 x the histogram's "
+                                  "maximum on frame 0: side lobes of the sinusoidal weights reach a quarter of a main lobe)" % thr)
+                sd[n] = r
+            line["soft_vote_decode"] = sd
+        except Exception as exc:
+            line["soft_vote_decode"] = {"error": repr(exc)}
         try:
             line["soft_votes"] = {n: measure_soft_votes(wl.CONFIGS[n], 40, 5, dev) for n in ("c2", "c3")}
         except Exception as exc:
@@ -483,7 +494,21 @@ def run_ours(args, cfg):
     dist_util.shutdown()
 
 
-def measure_other(cfg, steps, warmup, dev, refine=False, k_max=None, flags=0):
+def soft_threshold_for(cfg, dev):
+    """A peak threshold for the soft-vote decode of this workload: 0.3 of the histogram's maximum on frame 0 (the
+    threshold is the caller's parameter; the paper's is "predefined")."""
+    import torch
+    from paper_2609_16874_b200 import binding as cb
+    fr = wl.make_frame(cfg, 0)
+    dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, device=dev)
+    h = dec.soft_votes(torch.from_numpy(fr["emb"]).to(dev), torch.from_numpy(fr["fg"]).to(dev))
+    torch.cuda.synchronize(dev)
+    thr = 0.3 * float(h.max().item())
+    dec.close()
+    return thr
+
+
+def measure_other(cfg, steps, warmup, dev, refine=False, k_max=None, flags=0, soft_threshold=None):
     """Graph-replay timing of one more workload (no host leg, no CPU baseline): p50, MP/s, per-stage times.
     `refine`: with sub-cell refined centroids (CPE_FLAG_REFINE); `k_max`: max_instances other than the workload's."""
     import torch
@@ -495,7 +520,7 @@ def measure_other(cfg, steps, warmup, dev, refine=False, k_max=None, flags=0):
     flush = (torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
              if cfg.emb_bytes < 2 * L2_BYTES and n_frames * cfg.emb_bytes < 2 * L2_BYTES else None)
     dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, cfg.T_v, cfg.tau,
-                     k_max if k_max else cfg.K_max, device=dev, refine=refine, flags=flags)
+                     k_max if k_max else cfg.K_max, device=dev, refine=refine, flags=flags, soft_threshold=soft_threshold)
     pruned = cb.cpe_get_intermediate(dec.params, cb.CPE_INT_PRUNE_STATE, cfg.B, cfg.H, cfg.W, cfg.F)[0] == cb.CPE_OK
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
