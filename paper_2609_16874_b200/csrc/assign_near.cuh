@@ -169,7 +169,22 @@ assign_near_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, in
   const int tid = threadIdx.x;
   const size_t plane = (size_t)HW;
   const int K = count_ptr[b];
-  if (K < k_min) return;                       // few peaks: the all-pairs kernel's image
+  if (K < k_min) {
+    // Not this kernel's image -- unless it has no peak at all and this chain serves every image (k_min = 1): then
+    // every pixel's label is 0 and its scores are +inf.
+    if (K == 0 && k_min == 1) {
+      const float inf0 = __int_as_float(0x7f800000);
+      for (long long n = (long long)blockIdx.x * kNearThreads + tid; n < HW; n += (long long)gridDim.x * kNearThreads) {
+        const size_t o = (size_t)b * plane + n;
+        labels[o] = 0;
+        if (WANT2) {
+          best[o] = inf0;
+          second[o] = inf0;
+        }
+      }
+    }
+    return;
+  }
   uint32_t* state = near_state + b * kNearStride;
   if (K > kNearMaxPeaks) {                      // no lists were made: the filtered kernel's image
     if (tid == 0 && blockIdx.x == 0) state[kNearGiveUp] = 1u;
@@ -323,7 +338,16 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const size_t plane = (size_t)HW;
   const int K = count_ptr[b];
-  if (K < k_min) return;                       // few peaks: the all-pairs kernel's image
+  if (K < k_min) {
+    // Not this kernel's image -- unless it has no peak at all and this chain serves every image (k_min = 1): then
+    // every pixel's label is 0 (the label map is 16-byte aligned and H*W a multiple of four here).
+    if (K == 0 && k_min == 1) {
+      int4* z = reinterpret_cast<int4*>(labels + (size_t)b * plane);
+      for (long long i = (long long)blockIdx.x * kStreamThreads + tid; i < (long long)HW / 4; i += (long long)gridDim.x * kStreamThreads)
+        z[i] = make_int4(0, 0, 0, 0);
+    }
+    return;
+  }
   uint32_t* state = near_state + b * kNearStride;
   if (K > kNearMaxPeaks) {                      // no lists were made: the filtered kernel's image
     if (tid == 0 && blockIdx.x == 0) state[kNearGiveUp] = 1u;

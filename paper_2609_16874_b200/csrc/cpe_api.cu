@@ -160,7 +160,7 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
     rc = cpe::host::launch_peak_rows(st, B, F, p, pr->votes, pr->sums, pr->H, pr->W, pr->peak_cell, count, pr->refine_out,
                                      pr->gamma_out, pr->out_centroids, pr->pal_w, pr->pal_h, pr->peak_emb);
     if (rc) return rc;
-    rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, k_limit + 1, pr->ref2, pr->cand2, pr->ref_h,
+    rc = cpe::host::launch_peak_graph(st, B, F, p, pr->ref_emb, peak_emb, count, 1, pr->ref2, pr->cand2, pr->ref_h,
                                       pr->cand_h, pr->nbr, pr->sums_to_zero, cells);
     if (rc) return rc;
   }
@@ -168,16 +168,20 @@ int launch_assign(cudaStream_t st, const void* emb, const uint8_t* fg, int B, in
   if (pr) {
     rc = cpe::host::launch_assign_near(st, emb, fg, B, HW, F, p, pr->ref_emb, peak_emb, pr->ref2, pr->cand2, pr->nbr,
                                        pr->cell_peak, pr->pix_cell, cells, count, labels, best, second, pr->near_state,
-                                       k_limit + 1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h,
-                                       pr->hard_q, pr->W);
+                                       1, pr->slow_q, pr->q_cap, status, pr->ref_h, pr->cand_h, pr->hard_q, pr->W);
     if (rc) return rc;
+    // The pruned chain serves every image, whatever its number of peaks (an image without any gets its all-zero label
+    // map from it): no all-pairs launch.  The filtered kernel follows for the images that were handed on, and it
+    // leaves the vote map zero.
+    return cpe::host::launch_assign_filtered(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
+                                             status, votes_to_zero, cells, 1, acc, pr->near_state);
   }
   // (also with a limit of 0: an image without any peak still gets its all-zero label map from this kernel)
   rc = launch_assign_exact<T>(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters, nullptr,
                               cells, k_limit);
   if (rc) return rc;
   return cpe::host::launch_assign_filtered(st, emb, fg, B, HW, F, p, peak_emb, count, labels, best, second, counters,
-                                           status, votes_to_zero, cells, k_limit + 1, acc, pr ? pr->near_state : nullptr);
+                                           status, votes_to_zero, cells, k_limit + 1, acc, nullptr);
 }
 
 // Debug builds only (-DCPE_DEBUG_SYNC): wait after every stage and name the stage whose kernel failed (never

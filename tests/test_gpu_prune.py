@@ -157,7 +157,8 @@ def test_pruned_assignment_edge_cases():
     check_pruned(fr["emb"], np.zeros_like(fr["fg"]), cfg.bins_w, cfg.bins_h)
     check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, K_max=1)
     check_pruned(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, K_max=3, refine=True)
-    # a batch whose images go three ways: no peaks, few (all pairs), many (pruned)
+    # a batch with no, few and many peaks per image: the pruned chain serves all three (an image without peaks is
+    # zero-filled, not walked)
     H, W, F, bw, bh = 96, 128, 4, 64, 48
     rng = np.random.default_rng(8)
     emb = np.empty((3, 4 * F, H, W), np.float16)
@@ -169,4 +170,4 @@ def test_pruned_assignment_edge_cases():
         fg[b] = 1
     gpu, ora = check_pruned(emb, fg, bw, bh, flags=ANY_SIZE, expect_handed_on=[False, False, False])
     assert ora["count"].tolist() == [0, 5, 60]
-    assert gpu["prune_state"][2, 0] > 0 and gpu["prune_state"][1, 0] == 0      # only the third image was walked
+    assert gpu["prune_state"][2, 0] > 0 and gpu["prune_state"][1, 0] > 0 and gpu["prune_state"][0, 0] == 0
