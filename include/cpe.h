@@ -74,8 +74,8 @@ enum {
   CPE_FLAG_MMA_ASSIGN = 256u,     /* filtered assignment: the mma.sync kernel for every image (comparisons)          */
   CPE_FLAG_NO_PRUNE = 512u,       /* do not prune the candidates of Eq. 7 (see cpe_decode): every image with more peaks
                                      than the all-pairs range goes to the tensor-core filtered kernels; same results  */
-  CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment for every image, however few peaks it has and however small
-                                     the input is; same results                                                       */
+  CPE_FLAG_PRUNE_ALL = 1024u,     /* the pruned assignment however small the input is and whatever max_instances is
+                                     (it serves every image of a decode, also those with few peaks); same results     */
   CPE_FLAG_PRUNE_ANY_SIZE = 8192u,/* the pruned assignment also for inputs of fewer than 2^19 pixels (by default those
                                      go without it: its extra launches cost more than it saves there); same results    */
   CPE_FLAG_PRUNE_WALK_ONLY = 2048u, /* pruned assignment: the one-thread-per-pixel kernel also where the streaming kernel
@@ -213,6 +213,18 @@ int cpe_init_workspace(cpe_stream_t stream, int B, int H, int W, int F, const cp
  *      candidate centroids, listed by ascending linear bin index (Sec. 3.2, local-maxima search);
  *   3. every participating pixel gets label 1 + argmin_k ||xhat - P_w(a_k)|| + ||yhat - P_h(b_k)||
  *      (Eq. 4, Eq. 7; lowest k on ties) if that distance is below tau (Eq. 8), else 0.
+ *
+ * How step 3 is computed does not change its result (every pair that is scored is scored in the same fixed order of
+ * binary32 operations): on inputs of at least 2^19 pixels whose max_instances exceeds the all-pairs range (32 peaks,
+ * 16 for F > 8) the candidates of Eq. 7 are pruned.  Around a reference point g (gamma of the mean estimate of a
+ * peak's 3x3 window of bins) the triangle inequality gives |d_k - G_k| <= t, with G_k the Eq. 4 distance from g to
+ * candidate k and t the pixel's distance to g; every peak gets the list of its nearest candidates by G, a pixel is
+ * looked up through the bin it voted for, and only candidates that the bound cannot exclude are scored (usually one).
+ * Images that the bounds cannot prune, or with more than 1024 peaks, are handed to a tensor-core filtered kernel
+ * (binary16 contraction with rigorous error bounds, exact re-scoring of what survives), which also serves smaller
+ * inputs with more peaks than the all-pairs range; all pairs are scored on the plain ALUs otherwise.  The pruned
+ * path needs the larger workspace that cpe_workspace_size reports for it (4 bytes per pixel for the bins, two queues
+ * of H*W/4 entries per image, the lists) and F in {4, 8, 16}.
  *
  * emb, fg_mask      device, see Conventions.  emb aligned to its element size (16 bytes and
  *                   H*W a multiple of 16/elemsize select the vectorised kernels).
