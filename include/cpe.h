@@ -249,6 +249,17 @@ const char* cpe_strerror(int code);
 /* The CUDA runtime error number behind the calling thread's last CPE_ERR_CUDA (0 if none). */
 int cpe_last_cuda_error(void);
 
+/*
+ * Self-test of the voting kernel's division.  For binary16 input the quotient min(|s|,|c|) / max(|s|,|c|) inside the
+ * per-pixel estimate (the atan2 of the coarse-to-fine phase unwrapping) is formed by a reciprocal estimate, one Newton
+ * step and one residual correction in packed binary32 instead of two IEEE divisions; the estimate's bins are only
+ * bit-exact if that quotient is the IEEE one.  This call checks it for EVERY pair of binary16 values 0 <= a <= b
+ * (b = 0 is replaced by the kernel's floor 2^-30), about 5 x 10^8 quotients, and stores the number of results whose
+ * bits differ from IEEE division in *out_mismatches (device, 8-byte aligned; 0 on a correct build).  Enqueues a memset
+ * and one kernel on `stream`.
+ */
+int cpe_selftest_half_division(cpe_stream_t stream, unsigned long long* out_mismatches);
+
 /* ------------------------------------------------------------------ CUDA-graph helper ------- */
 
 /*

@@ -54,6 +54,7 @@ EXPORTS = (
     "cpe_profile_decode", "cpe_host_ctx_create", "cpe_host_decode", "cpe_host_submit", "cpe_host_wait",
     "cpe_host_ctx_traffic", "cpe_host_ctx_destroy",
     "cpe_decode_static", "cpe_soft_votes", "cpe_instance_masks", "cpe_channels_last_to_planar",
+    "cpe_selftest_half_division",
 )
 
 
@@ -117,6 +118,8 @@ def load() -> ctypes.CDLL:
     lib.cpe_strerror.restype = ctypes.c_char_p
     lib.cpe_last_cuda_error.argtypes = []
     lib.cpe_last_cuda_error.restype = ci
+    lib.cpe_selftest_half_division.argtypes = [vp, vp]
+    lib.cpe_selftest_half_division.restype = ci
     lib.cpe_graph_create.argtypes = [vp, vp, vp, ci, ci, ci, ci, pp, vp, vp, vp, ctypes.POINTER(vp)]
     lib.cpe_graph_create.restype = ci
     lib.cpe_graph_launch.argtypes = [vp, vp]
@@ -166,6 +169,10 @@ def cpe_strerror(code: int) -> str:
 
 def cpe_last_cuda_error() -> int:
     return int(load().cpe_last_cuda_error())
+
+
+def cpe_selftest_half_division(stream, out_mismatches: int) -> int:
+    return int(load().cpe_selftest_half_division(stream, out_mismatches))
 
 
 def cpe_workspace_size(B, H, W, F, params: cpe_params) -> int:

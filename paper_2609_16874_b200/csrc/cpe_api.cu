@@ -762,6 +762,36 @@ extern "C" int cpe_decode_static(cpe_stream_t stream, const void* emb, const uin
   return decode_impl(st, emb, fg_mask, B, H, W, F, &p, out_labels, out_centroids, out_count, nullptr);
 }
 
+namespace cpe {
+// Self-test of div2_half_operands: CTA i takes the denominator with binary16 bit pattern i (0 .. 0x7bff: zero and every
+// positive finite value), its threads all numerators up to it; counts the results whose bits differ from __fdiv_rn's.
+__global__ void half_division_selftest_kernel(unsigned long long* __restrict__ mismatches) {
+  const uint32_t bi = blockIdx.x;
+  if (bi > 0x7bffu) return;
+  const float floor_b = 9.31322574615478515625e-10f;
+  const float b = fmaxf(__half2float(__ushort_as_half((unsigned short)bi)), floor_b);
+  unsigned long long n = 0;
+  for (uint32_t ai = 2 * threadIdx.x; ai <= bi; ai += 2 * blockDim.x) {
+    const float a0 = __half2float(__ushort_as_half((unsigned short)ai));
+    const float a1 = __half2float(__ushort_as_half((unsigned short)min(ai + 1u, bi)));
+    const float2 got = div2_half_operands(make_float2(a0, a1), make_float2(b, b));
+    n += __float_as_uint(got.x) != __float_as_uint(__fdiv_rn(a0, b));
+    n += __float_as_uint(got.y) != __float_as_uint(__fdiv_rn(a1, b));
+  }
+  if (n) atomicAdd(mismatches, n);
+}
+}  // namespace cpe
+
+extern "C" int cpe_selftest_half_division(cpe_stream_t stream, unsigned long long* out_mismatches) {
+  if (!out_mismatches) return CPE_ERR_NULL;
+  if ((uintptr_t)out_mismatches % 8) return CPE_ERR_ALIGN;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  CPE_CUDA(cudaMemsetAsync(out_mismatches, 0, sizeof(unsigned long long), st));
+  cpe::half_division_selftest_kernel<<<0x7c00, 256, 0, st>>>(out_mismatches);
+  CPE_CUDA(cudaGetLastError());
+  return CPE_OK;
+}
+
 extern "C" int cpe_soft_votes(cpe_stream_t stream, const void* emb, const uint8_t* fg_mask, int B, int H, int W, int F,
                    const cpe_params* params, float* out_hist) {
   if (!emb || !out_hist) return CPE_ERR_NULL;

@@ -422,7 +422,9 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
             // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
 #pragma unroll
             for (int j = 0; j < VEC; j += 2) {
-              const float2 u = atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
+              // (binary16 input: the variant whose two divisions run as packed instructions, bit-identical for such operands)
+              const float2 u = sizeof(T) == 2 ? atan2_ht_pair_h(s[j], c[j], s[j + 1], c[j + 1])
+                                              : atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
               const float2 v = refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
               p[j] = v.x;
               p[j + 1] = v.y;

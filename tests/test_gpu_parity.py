@@ -409,3 +409,14 @@ def test_small_max_instances_takes_the_three_kernel_chain():
             assert ((lab == ora["labels"]) | near_tie).all()
         dec.close()
     assert nodes[32] == 3 and nodes[33] > nodes[32], nodes
+
+
+def test_packed_division_of_the_voting_kernel_is_the_ieee_quotient_for_every_binary16_pair():
+    """The voting kernel divides binary16-valued operands with a reciprocal estimate and one correction in packed
+    binary32; the library's self-test compares it with IEEE division for all 5e8 pairs 0 <= a <= b."""
+    import torch
+    out = torch.full((1,), 123, dtype=torch.int64, device="cuda")
+    rc = cb.cpe_selftest_half_division(torch.cuda.current_stream().cuda_stream, out.data_ptr())
+    assert rc == cb.CPE_OK
+    torch.cuda.synchronize()
+    assert int(out.item()) == 0
