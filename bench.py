@@ -472,7 +472,7 @@ def run_ours(args, cfg):
             for n in ("c1", "c2"):
                 thr = soft_threshold_for(wl.CONFIGS[n], dev)
                 r = measure_other(wl.CONFIGS[n], 40, 5, dev, soft_threshold=thr)
-                r["workload"] += ("; vote mode: soft (CPE_FLAG_SOFT_VOTE, soft_threshold %.4g = 0.15 x the histogram's "
+                r["workload"] += ("; vote mode: soft (CPE_FLAG_SOFT_VOTE, soft_threshold %.4g = 0.3 x the histogram's "
                                   "maximum on frame 0; a global threshold cuts small instances and lets side lobes of large "
                                   "ones through: see instances_found)" % thr)
                 sd[n] = r
@@ -496,7 +496,7 @@ def run_ours(args, cfg):
 
 
 def soft_threshold_for(cfg, dev):
-    """A peak threshold for the soft-vote decode of this workload: 0.15 of the histogram's maximum on frame 0 (the
+    """A peak threshold for the soft-vote decode of this workload: 0.3 of the histogram's maximum on frame 0 (the
     threshold is the caller's parameter; the paper's is "predefined")."""
     import torch
     from paper_2609_16874_b200 import binding as cb
@@ -504,7 +504,7 @@ def soft_threshold_for(cfg, dev):
     dec = cb.Decoder(cfg.B, cfg.H, cfg.W, cfg.F, cfg.dtype, cfg.bins_w, cfg.bins_h, device=dev)
     h = dec.soft_votes(torch.from_numpy(fr["emb"]).to(dev), torch.from_numpy(fr["fg"]).to(dev))
     torch.cuda.synchronize(dev)
-    thr = 0.15 * float(h.max().item())
+    thr = 0.3 * float(h.max().item())
     dec.close()
     return thr
 
