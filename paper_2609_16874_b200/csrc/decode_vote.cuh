@@ -350,20 +350,17 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
   const uint32_t act = __ballot_sync(0xffffffffu, bits != 0);
   if (lane == 0) s_scan[wid] = __popc(act);
   __syncthreads();
-  if (tid == 0) {
-    int run = 0;
+  // every thread adds up the warps' counts itself (eight shared-memory reads): no serial step, one barrier fewer
+  int before = 0, total = 0;
 #pragma unroll
-    for (int w = 0; w < kVoteThreads / 32; ++w) {
-      const int t = s_scan[w];
-      s_scan[w] = run;
-      run += t;
-    }
-    s_scan[kVoteThreads / 32] = run;
+  for (int w = 0; w < kVoteThreads / 32; ++w) {
+    const int t = s_scan[w];
+    if (w < wid) before += t;
+    total += t;
   }
+  if (bits) s_grp[before + __popc(act & ((1u << lane) - 1u))] = (uint16_t)(tid | (bits << 8));
   __syncthreads();
-  if (bits) s_grp[s_scan[wid] + __popc(act & ((1u << lane) - 1u))] = (uint16_t)(tid | (bits << 8));
-  __syncthreads();
-  const int n_items = 2 * s_scan[kVoteThreads / 32];
+  const int n_items = 2 * total;
 
   const float half_w = (float)(bins_w + 1) * 0.5f, half_h = (float)(bins_h + 1) * 0.5f;
   uint32_t nonfinite = 0, voted = 0;
