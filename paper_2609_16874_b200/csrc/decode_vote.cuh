@@ -288,8 +288,8 @@ decode_vote_scalar_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
 constexpr int kVecGroupsMax = 256;   // groups per CTA: 256, 128 or 64 (template parameter GROUPS; the launcher takes the
                                      // largest that still gives a full wave of CTAs -- small images are latency-bound
                                      // and want many short CTAs, large ones want fewer fixed costs)
-// harmonics whose plane loads are in flight together (2 loads each): what leaves room for four CTAs per SM
-template <typename T> __host__ __device__ constexpr int vec_level_batch() { return sizeof(T) == 4 ? 4 : 2; }
+// harmonics whose plane loads are in flight together (2 loads each); four CTAs per SM at 64 registers
+template <typename T> __host__ __device__ constexpr int vec_level_batch() { return 4; }
 
 template <typename T, int FT, int MODE, int GROUPS>
 __global__ void __launch_bounds__(kVoteThreads, 4)
