@@ -67,25 +67,8 @@ __device__ __forceinline__ void near_walk(const float2 (&e2)[D / 2], int k0, int
   hard = (j == kNbrCap && K > kNbrCap) || (!WANT2 && j == kWalkMax);
 }
 
-// Every peak, in ascending k (a hard pixel).
-template <int D, bool WANT2>
-__device__ __forceinline__ void near_full_scan(const float2 (&e2)[D / 2], int K, const float* __restrict__ cand_img,
-                                               float& d1, float& d2, int& k1) {
-  const float inf = __int_as_float(0x7f800000);
-  d1 = d2 = inf;
-  k1 = -1;
-  float bound2 = inf;
-  for (int k = 0; k < K; ++k) {
-    const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(cand_img + (size_t)k * D), bound2);
-    if (d < d1) { d2 = d1; d1 = d; k1 = k; }
-    else if (d < d2) { d2 = d; }
-    const float bound = WANT2 ? d2 : d1;
-    bound2 = bound * bound * (1.0f + 1e-6f);
-  }
-}
-
-// The same for one pixel by a whole warp (every lane passes the same pixel): a lane scores the peaks k_first,
-// k_first + k_stride, ... (lane, 32 for a warp on its own; several warps may share the peaks of one pixel)
+// Every peak of an image for one pixel (a hard pixel), by a whole warp (every lane passes the same pixel): a lane
+// scores the peaks k_first, k_first + k_stride, ... (lane, 32 for a warp on its own; several warps may share one pixel)
 // with the pixel's values fetched by every lane (the same addresses: one transaction per load), then the lanes' results
 // are merged -- smaller distance first, lower k on equal distances, which is what the serial scan in ascending k gives.
 // A single thread scanning hundreds of peaks is a chain of dependent row fetches that takes as long as the rest of the
