@@ -626,7 +626,10 @@ assign_mma_body(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int H
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               as[mt][i] = ax[mt][i] + ay[i];
-              any = any || (as[mt][i] <= thr[mt * 2 + (i >> 1)]);
+              // the test of pass_mask below, evaluated here already: on workloads whose candidates all lie at about
+              // the same distance the coarser S <= thr alone passes for nearly every pair
+              const float S = as[mt][i], A = ax[mt][i];
+              any = any || (fmaf(2.0f, fminf(A, S - A), S) <= thr[mt * 2 + (i >> 1)]);
             }
           }
           if (__any_sync(0xffffffffu, any)) {
