@@ -29,7 +29,7 @@ constexpr int kSvTiles = 2;         // pixel tile buffers
 constexpr int kSvCols = 512;        // tensor-memory columns: D_x [0,128), D_y [128,256), H block [256,384)
 
 struct SvSmem {
-  int tiles, pw, ph, ex, ey, ring, ringbits, rnx, rny, rflags, misc, total;
+  int tiles, pw, ph, ex, ey, exl, eyl, ring, ringbits, rnx, rny, rflags, misc, total;
 };
 __host__ __device__ inline SvSmem sv_smem_layout(int KA) {
   SvSmem s;
@@ -39,6 +39,9 @@ __host__ __device__ inline SvSmem sv_smem_layout(int KA) {
   s.ph = off;       off += 2 * kSvBins * KA * 2;
   s.ex = off;       off += kTcRows * kSvBins * 2;                   // E_x tile, operand layout of GEMM 2
   s.ey = off;       off += kTcRows * kSvBins * 2;
+  // low parts of the two E tiles (F <= 8 only: with F > 8 the pixel tiles leave no room for them)
+  s.exl = off;      off += KA == 16 ? kTcRows * kSvBins * 2 : 0;
+  s.eyl = off;      off += KA == 16 ? kTcRows * kSvBins * 2 : 0;
   s.ring = off;     off += kTcRing * 4;
   s.ringbits = off; off += kTcRing;
   s.rnx = off;      off += kSvTiles * kTcRows * 4;
@@ -68,6 +71,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
   constexpr uint32_t kPalLbo = kSvBins * 16;        // ... in a palette block
   constexpr uint32_t kELbo = (kSvBins / 8) * 128;   // ... (along the pixels) in an E tile
   constexpr bool kSplitPixel = sizeof(T) == 4;      // binary32 pixels carry a low part
+  constexpr bool kSplitE = KA == 16;                // the weights go to GEMM 2 as binary16 high + low parts
   extern __shared__ __align__(1024) unsigned char sv_smem[];
   const SvSmem L = sv_smem_layout(KA);
   __half* s_tiles = reinterpret_cast<__half*>(sv_smem + L.tiles);
@@ -75,6 +79,8 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
   __half* s_ph = reinterpret_cast<__half*>(sv_smem + L.ph);
   __half* s_ex = reinterpret_cast<__half*>(sv_smem + L.ex);
   __half* s_ey = reinterpret_cast<__half*>(sv_smem + L.ey);
+  __half* s_exl = reinterpret_cast<__half*>(sv_smem + L.exl);      // (only with kSplitE)
+  __half* s_eyl = reinterpret_cast<__half*>(sv_smem + L.eyl);
   uint32_t* s_ring = reinterpret_cast<uint32_t*>(sv_smem + L.ring);
   uint8_t* s_ringbits = reinterpret_cast<uint8_t*>(sv_smem + L.ringbits);
   float* s_rnx = reinterpret_cast<float*>(sv_smem + L.rnx);               // per tile buffer and row: ||xhat||^2
@@ -115,7 +121,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < kSvTiles * 2 * kPartHalves / 2; i += kSvThreads) reinterpret_cast<uint32_t*>(s_tiles)[i] = 0u;
-  for (int i = tid; i < kTcRows * kSvBins; i += kSvThreads) {      // E_x and E_y are contiguous
+  for (int i = tid; i < (kSplitE ? 2 : 1) * kTcRows * kSvBins; i += kSvThreads) {      // E_x, E_y (and their low parts) are contiguous
     reinterpret_cast<uint32_t*>(s_ex)[i] = 0u;
   }
   // -2 P rows of this block, split into binary16 high and low parts; K-major core matrices: (bin n, slot s) at
@@ -327,6 +333,8 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     const uint64_t d_ph = tc_desc((uint32_t)__cvta_generic_to_shared(s_ph), kPalLbo, 128u);
     const uint64_t d_ex = tc_desc((uint32_t)__cvta_generic_to_shared(s_ex), kELbo, 128u);
     const uint64_t d_ey = tc_desc((uint32_t)__cvta_generic_to_shared(s_ey), kELbo, 128u);
+    const uint64_t d_exl = tc_desc((uint32_t)__cvta_generic_to_shared(s_exl), kELbo, 128u);
+    const uint64_t d_eyl = tc_desc((uint32_t)__cvta_generic_to_shared(s_eyl), kELbo, 128u);
     constexpr uint64_t kLoPal = (uint64_t)((kSvBins * KA * 2) >> 4);        // low part of a palette block
     constexpr uint64_t kLoTile = (uint64_t)((kPartHalves * 2) >> 4);        // low part of a pixel tile
     uint32_t t = 0;
@@ -340,19 +348,33 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
     // approximations (sqrt, 2^x: about 2^-22 relative each) are far inside the binary16 rounding that follows; the
     // flush-to-zero forms are single instructions (a subnormal argument or result is below anything binary16 holds:
     // its smallest subnormal is e^-16.6).  A row without a pixel is masked after packing.  `ck` = c log2(e)^2.
-    auto weights8 = [&](const float* v, float ck, bool live) -> uint4 {
-      uint32_t w[4];
+    // With kSplitE a weight w goes to GEMM 2 as two binary16 numbers, hi = fl16(w) and lo = fl16(w - hi), and the product
+    // of two weights as hi hi + hi lo + lo hi (what is dropped, lo lo, is 2^-22 of it): the histogram is then good to
+    // about 1e-5 instead of the 1e-3 of a single binary16 rounding.  The weights are also scaled by 2^14 (added to the
+    // exponent argument, so it costs nothing), which keeps the low parts of small weights out of binary16's subnormal
+    // range; the block is scaled back by 2^-28 when it is added to the histogram.
+    constexpr float kEScale = kSplitE ? 14.0f : 0.0f;
+    auto weights8 = [&](const float* v, float ck, bool live, uint4& lo_out) -> uint4 {
+      uint32_t w[4], wl[4];
       const uint32_t keep = live ? 0xffffffffu : 0u;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float d0, d1, e0, e1;
         asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d0) : "f"(fabsf(fmaf(v[2 * i], log2e_sq, ck))));
         asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(d1) : "f"(fabsf(fmaf(v[2 * i + 1], log2e_sq, ck))));
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-d0));
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-d1));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(kEScale - d0));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(kEScale - d1));
         const __half2 h = __floats2half2_rn(e0, e1);
         w[i] = *reinterpret_cast<const uint32_t*>(&h) & keep;
+        if constexpr (kSplitE) {
+          const float2 hf = __half22float2(h);
+          const __half2 l = __floats2half2_rn(e0 - hf.x, e1 - hf.y);
+          wl[i] = *reinterpret_cast<const uint32_t*>(&l) & keep;
+        } else {
+          wl[i] = 0u;
+        }
       }
+      lo_out = make_uint4(wl[0], wl[1], wl[2], wl[3]);
       return make_uint4(w[0], w[1], w[2], w[3]);
     };
 
@@ -414,14 +436,18 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       // (p / 8) * kELbo + (n / 8) * 128 + (p % 8) * 16 + (n % 8) * 2 bytes
       {
         unsigned char* e_row = reinterpret_cast<unsigned char*>(axis_y ? s_ey : s_ex) + (row >> 3) * kELbo + (row & 7) * 16;
+        unsigned char* e_row_lo = reinterpret_cast<unsigned char*>(axis_y ? s_eyl : s_exl) + (row >> 3) * kELbo + (row & 7) * 16;
         // only the bins that exist (in steps of 32): the rest of the E tiles stays zero
         const int nbins = axis_y ? nb : na;
         for (int c0 = 0; c0 < nbins; c0 += 32) {
           float v[32];
           tc_ld32(t_lane + (uint32_t)(axis_y * 128 + c0), v);
 #pragma unroll
-          for (int g = 0; g < 4; ++g)
-            *reinterpret_cast<uint4*>(e_row + ((c0 >> 3) + g) * 128) = weights8(v + 8 * g, c_row, live);
+          for (int g = 0; g < 4; ++g) {
+            uint4 lo;
+            *reinterpret_cast<uint4*>(e_row + ((c0 >> 3) + g) * 128) = weights8(v + 8 * g, c_row, live, lo);
+            if constexpr (kSplitE) *reinterpret_cast<uint4*>(e_row_lo + ((c0 >> 3) + g) * 128) = lo;
+          }
         }
       }
       // the next tile's row data (the producers are a tile ahead), before the barrier that frees D and publishes E
@@ -436,6 +462,10 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
         for (int ks = 0; ks < kTcRows / 16; ++ks) {
           const uint64_t o = (uint64_t)((ks * 2u * kELbo) >> 4);
           tc_mma(tmem + 256u, d_ex + o, d_ey + o, kSvIdesc2, t > 0 || ks > 0);
+          if constexpr (kSplitE) {
+            tc_mma(tmem + 256u, d_ex + o, d_eyl + o, kSvIdesc2, true);
+            tc_mma(tmem + 256u, d_exl + o, d_ey + o, kSvIdesc2, true);
+          }
         }
         tc_commit(mb_e);
         if (!(flags & kRfEnd)) issue_gemm1((int)((t + 1) % kSvTiles));
@@ -459,7 +489,8 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
         if (a < bins_w) {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (b0 + c0 + j < bins_h) atomicAdd(h_img + (size_t)(b0 + c0 + j) * bins_w + a, v[j]);
+            if (b0 + c0 + j < bins_h)
+              atomicAdd(h_img + (size_t)(b0 + c0 + j) * bins_w + a, kSplitE ? v[j] * 3.7252902984619140625e-9f : v[j]);   // 2^-28
         }
       }
     }

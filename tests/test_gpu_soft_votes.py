@@ -8,9 +8,15 @@ from paper_2609_16874_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-# Per bin: binary16 rounding of E_x and of E_y (2^-11 each) before the second contraction, binary32 accumulation and
-# atomics (~1e-6), first contraction good to ~1e-6 in the squared distance (operands split into two binary16 parts).
-REL = 2e-3
+# Per bin, F <= 8: the weights enter the second contraction as binary16 high + low parts (what is dropped is 2^-22 of a
+# product), binary32 accumulation and atomics (~1e-6), first contraction good to ~1e-6 in the squared distance (operands
+# split into two binary16 parts), special-function square root and 2^x (2^-22 each): 1e-4 holds with a factor of ten
+# to spare (measured 5e-6 .. 9e-6).  F > 8 (no room for the low parts): one binary16 rounding of E_x and of E_y, 2^-11 each.
+REL_SPLIT, REL_SINGLE = 1e-4, 2e-3
+
+
+def rel_of(emb):
+    return REL_SPLIT if emb.shape[1] // 4 <= 8 else REL_SINGLE
 
 
 def run_soft(emb, fg, bins_w, bins_h):
@@ -41,7 +47,7 @@ def check(emb, fg, bins_w, bins_h, cells=None):
         want = oracle.soft_votes(emb, fg, bins_w, bins_h, sample_cells=cells)
         g = got.reshape(got.shape[0], -1)[:, cells].astype(np.float64)
     err = np.abs(g - want)
-    assert (err <= REL * want + 1e-30).all(), (float((err / np.maximum(want, 1e-300)).max()), float(want.max()))
+    assert (err <= rel_of(emb) * want + 1e-30).all(), (float((err / np.maximum(want, 1e-300)).max()), float(want.max()))
     return got, want
 
 
@@ -82,10 +88,14 @@ def test_soft_votes_skip_nonfinite_and_out_of_range_pixels():
     check(h, None, 16, 16)
 
 
-def test_soft_votes_full_size_c2_on_sampled_bins():
-    cfg = wl.CONFIGS["c2"]
+@pytest.mark.parametrize("name,n_random", [("c2", 24), ("c3", 10), ("c4", 10)])
+def test_soft_votes_full_size_on_sampled_bins(name, n_random):
+    """Full-size c2, c3 and c4 (F = 8: the 1e-4 bound): random bins and the eight bins with the most hard votes of image 0
+    (where the instances are), each summed over every participating pixel by the oracle."""
+    cfg = wl.CONFIGS[name]
     fr = wl.make_frame(cfg, 0)
     rng = np.random.default_rng(9)
-    cells = np.unique(np.concatenate([rng.integers(0, cfg.bins_w * cfg.bins_h, 24),
-                                      np.argsort(oracle.votes(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h)["votes"].ravel())[-8:]]))
+    oracle.set_threads(oracle.max_threads())
+    hard = oracle.votes(fr["emb"][:1], fr["fg"][:1], cfg.bins_w, cfg.bins_h)["votes"][0]
+    cells = np.unique(np.concatenate([rng.integers(0, cfg.bins_w * cfg.bins_h, n_random), np.argsort(hard.ravel())[-8:]]))
     check(fr["emb"], fr["fg"], cfg.bins_w, cfg.bins_h, cells=cells.astype(np.int32))
