@@ -26,6 +26,7 @@ constexpr int kSvThreads = 384;     // warps 0-3: pixel rows, x axis (and MMA is
                                     // warps 8-11: the same pixel rows, y axis
 constexpr int kSvBins = 128;        // bins per block side
 constexpr int kSvTiles = 2;         // pixel tile buffers
+constexpr int kSvFlushTiles = 8;    // tiles accumulated in tensor memory between two flushes of the H block
 constexpr int kSvCols = 512;        // tensor-memory columns: D_x [0,128), D_y [128,256), H block [256,384)
 
 struct SvSmem {
@@ -410,6 +411,32 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       return true;
     };
 
+    // The H block goes to the histogram (thread = bin a, the tensor-memory lane; columns = bins b) every kSvFlushTiles
+    // tiles and at the end.  The tensor pipe adds into its binary32 accumulator with a small systematic loss per
+    // addition (measured: about 2^-23 of the running sum, all of one sign), so a block that ran over a CTA's whole
+    // share of a large image (a hundred tiles, thousands of additions) came out 1.7e-4 low; restarting it every
+    // eight tiles bounds the loss at 192 additions (2.3e-5) and leaves the long sum to the round-to-nearest atomics.
+    uint32_t t_flushed = 0;
+    auto flush_block = [&]() {
+      const bool ok = mbar_wait(mb_e, (t - 1) & 1u, s_abort);   // GEMM 2 of tile t - 1 is done
+      if (!__all_sync(0xffffffffu, ok)) { bad = true; return; }
+      tc_fence_after();
+      const int a = a0 + row;
+      float* h_img = hist + (size_t)img * bins_w * bins_h;
+      // the two threads of a row share its columns
+      for (int c0 = axis_y * (kSvBins / 2); c0 < (axis_y + 1) * (kSvBins / 2); c0 += 32) {
+        float v[32];
+        tc_ld32(t_lane + 256u + (uint32_t)c0, v);
+        if (a < bins_w) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (b0 + c0 + j < bins_h)
+              atomicAdd(h_img + (size_t)(b0 + c0 + j) * bins_w + a, kSplitE ? v[j] * 3.7252902984619140625e-9f : v[j]);   // 2^-28
+        }
+      }
+      t_flushed = t;
+    };
+
     // The loop is software-pipelined by one tile: the thread that issues GEMM 2 of tile t issues GEMM 1 of tile t + 1
     // right behind it, so the tensor pipe runs them back to back while the row threads are between two epilogues,
     // and one wait (GEMM 1 done: the MMAs complete in issue order, so GEMM 2 of the tile before is done as well)
@@ -461,7 +488,7 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
 #pragma unroll
         for (int ks = 0; ks < kTcRows / 16; ++ks) {
           const uint64_t o = (uint64_t)((ks * 2u * kELbo) >> 4);
-          tc_mma(tmem + 256u, d_ex + o, d_ey + o, kSvIdesc2, t > 0 || ks > 0);
+          tc_mma(tmem + 256u, d_ex + o, d_ey + o, kSvIdesc2, t > t_flushed || ks > 0);
           if constexpr (kSplitE) {
             tc_mma(tmem + 256u, d_ex + o, d_eyl + o, kSvIdesc2, true);
             tc_mma(tmem + 256u, d_exl + o, d_ey + o, kSvIdesc2, true);
@@ -472,28 +499,10 @@ soft_vote_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg, int 
       }
       __syncwarp();
       ++t;
+      // the reads of the block are ordered before the next GEMM 2 (which starts it afresh) by the next tile's barrier
+      if (t - t_flushed == (uint32_t)kSvFlushTiles && !(flags & kRfEnd)) flush_block();
     }
-    // ---- the block goes to the histogram: thread = bin a (tensor-memory lane), columns = bins b
-    if (!bad && t > 0) {
-      const bool ok = mbar_wait(mb_e, (t - 1) & 1u, s_abort);
-      if (!__all_sync(0xffffffffu, ok)) bad = true;
-    }
-    if (!bad && t > 0) {
-      tc_fence_after();
-      const int a = a0 + row;
-      float* h_img = hist + (size_t)img * bins_w * bins_h;
-      // the two threads of a row share its columns
-      for (int c0 = axis_y * (kSvBins / 2); c0 < (axis_y + 1) * (kSvBins / 2); c0 += 32) {
-        float v[32];
-        tc_ld32(t_lane + 256u + (uint32_t)c0, v);
-        if (a < bins_w) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (b0 + c0 + j < bins_h)
-              atomicAdd(h_img + (size_t)(b0 + c0 + j) * bins_w + a, kSplitE ? v[j] * 3.7252902984619140625e-9f : v[j]);   // 2^-28
-        }
-      }
-    }
+    if (!bad && t > t_flushed) flush_block();
     if (bad) {
       *s_abort = 1;
       am_ok(false, 13u, status);
