@@ -37,7 +37,8 @@ __device__ __forceinline__ float score_direct(const float2 (&e2)[D / 2], const f
 
 // Four peaks at once: four independent chains keep the FMA pipe busy (one chain alone waits on its own latency).
 // Peaks beyond `kn` must not be passed (the caller pads the shared-memory chunk with copies of a valid peak).
-template <int D>
+// ROW2 = distance between two of the four rows, in float2 units.
+template <int D, int ROW2 = D / 2>
 __device__ __forceinline__ void score_direct4(const float2 (&e2)[D / 2], const float2* __restrict__ pk2, float bound2,
                                               float (&d)[4]) {
   float2 s[4];
@@ -47,7 +48,7 @@ __device__ __forceinline__ void score_direct4(const float2 (&e2)[D / 2], const f
   for (int c = 0; c < D / 2; c += 2) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const float4 q = *reinterpret_cast<const float4*>(pk2 + j * (D / 2) + c);
+      const float4 q = *reinterpret_cast<const float4*>(pk2 + j * ROW2 + c);
       float2 t = sub2_rn(e2[c], make_float2(q.x, q.y));
       s[j] = fma2_rn(t, t, s[j]);
       t = sub2_rn(e2[c + 1], make_float2(q.z, q.w));

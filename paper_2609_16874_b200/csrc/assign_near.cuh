@@ -773,7 +773,7 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
 }
 
 // The pixels that the walk left over are scored against every peak: a whole CTA per pixel while there are fewer pixels
-// than CTAs, else a thread per pixel with the rows staged in shared memory.
+// than CTAs, else eight lanes per pixel with the rows staged in shared memory.
 template <typename T, int FT>
 __global__ void __launch_bounds__(kNearThreads)
 assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const float* __restrict__ cand2,
@@ -839,14 +839,20 @@ assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
       __syncthreads();
     }
   } else {
-    // Many pixels (an instance without a peak of its own sends all of its pixels here): the all-pairs scheme, a thread
-    // per pixel with the pixel's values in registers while the candidate rows pass through shared memory in chunks.
-    // Peaks in ascending k with a strict comparison: the lowest k keeps an exact tie, as in the scans above.
-    constexpr int kChunk = 32;
-    __shared__ __align__(16) float s_rows[kChunk * D];
+    // Many pixels (an instance without a peak of its own sends all of its pixels here): the all-pairs scheme with
+    // eight lanes per pixel.  The candidate rows pass through shared memory in chunks of 32; lane s of a pixel scores
+    // the rows s, s + 8, s + 16, s + 24 of a chunk against the pixel's values in its registers (a row is padded to
+    // D + 4 floats, so the eight rows that a warp reads at a time sit in different banks), and the eight results are
+    // merged like the lanes' of the warp-wide scan: smaller distance first, lower k on equal distances -- what the
+    // serial scan in ascending k with a strict comparison gives.  (One thread per pixel scoring every peak left most
+    // of the GPU idle: a few thousand threads, each a chain of a hundred dependent scores.)
+    constexpr int kChunk = 32, kSlices = 8, kRow = D + 4;
+    constexpr int kPixPerCta = kNearThreads / kSlices;
+    __shared__ __align__(16) float s_rows[kChunk * kRow];
     const float inf = __int_as_float(0x7f800000);
-    for (int base = blockIdx.x * kNearThreads; base < n_h; base += gridDim.x * kNearThreads) {   // uniform per CTA
-      const int i = base + (int)threadIdx.x;
+    const int slice = lane & (kSlices - 1);
+    for (int base = blockIdx.x * kPixPerCta; base < n_h; base += gridDim.x * kPixPerCta) {   // uniform per CTA
+      const int i = base + (int)(threadIdx.x / kSlices);
       const bool have = i < n_h;
       const size_t n = have ? hard_q[(size_t)b * q_cap + i] : 0;
       float2 e2[D / 2];
@@ -859,31 +865,34 @@ assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
         }
       }
       float d1 = inf, bound2 = inf;
-      int k1 = -1;
+      int k1 = 0x7fffffff;
       for (int k0 = 0; k0 < K; k0 += kChunk) {
         const int kn = min(kChunk, K - k0);
         __syncthreads();
-        for (int j = threadIdx.x; j < kn * (D / 4); j += kNearThreads)
-          reinterpret_cast<float4*>(s_rows)[j] = __ldg(reinterpret_cast<const float4*>(cand_img + (size_t)k0 * D) + j);
+        // (rows past the last peak are copies of the chunk's first row: scored, never taken)
+        for (int j = threadIdx.x; j < kChunk * (D / 4); j += kNearThreads) {
+          const int r = j / (D / 4), q = j % (D / 4);
+          reinterpret_cast<float4*>(s_rows + r * kRow)[q] =
+              __ldg(reinterpret_cast<const float4*>(cand_img + (size_t)(k0 + (r < kn ? r : 0)) * D) + q);
+        }
         __syncthreads();
         if (have) {
-          int kk = 0;
-          for (; kk + 4 <= kn; kk += 4) {
-            float d[4];
-            score_direct4<D>(e2, reinterpret_cast<const float2*>(s_rows + kk * D), bound2, d);
+          float d[4];
+          score_direct4<D, kSlices * kRow / 2>(e2, reinterpret_cast<const float2*>(s_rows + slice * kRow), bound2, d);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (d[j] < d1) { d1 = d[j]; k1 = k0 + kk + j; }
-            bound2 = d1 * d1 * (1.0f + 1e-6f);
-          }
-          for (; kk < kn; ++kk) {
-            const float d = score_direct<D>(e2, reinterpret_cast<const float2*>(s_rows + kk * D), bound2);
-            if (d < d1) { d1 = d; k1 = k0 + kk; }
-            bound2 = d1 * d1 * (1.0f + 1e-6f);
-          }
+          for (int j = 0; j < 4; ++j)
+            if (slice + kSlices * j < kn && d[j] < d1) { d1 = d[j]; k1 = k0 + slice + kSlices * j; }
+          bound2 = d1 * d1 * (1.0f + 1e-6f);
         }
       }
-      if (have) finish(n, d1, k1);
+      // (every lane of the warp takes part: lanes without a pixel carry +inf)
+#pragma unroll
+      for (int off = 1; off < kSlices; off <<= 1) {
+        const float od1 = __shfl_xor_sync(0xffffffffu, d1, off);
+        const int ok1 = __shfl_xor_sync(0xffffffffu, k1, off);
+        if (od1 < d1 || (od1 == d1 && ok1 < k1)) { d1 = od1; k1 = ok1; }
+      }
+      if (have && slice == 0) finish(n, d1, k1 == 0x7fffffff ? -1 : k1);
     }
   }
   near_flush_counters(state, n_rejected, n_full * (uint32_t)K, 0u, n_full);

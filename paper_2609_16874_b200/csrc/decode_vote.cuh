@@ -379,14 +379,14 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
     uint32_t okbits = (1u << VEC) - 1u;
     if (have) {
       // validity accumulators: binary32 inputs fold |s| + |c| per pixel (fold_finite); binary16 inputs are finite iff
-      // every element is (their sums cannot overflow binary32), so the raw pairs go through a packed multiply by zero
-      // that turns an infinity or a NaN into a NaN that sticks -- half the instructions
+      // every element is (their sums cannot overflow binary32), so a running packed maximum of the absolute values in
+      // the form that propagates NaNs is enough: one instruction per two pixels and harmonic
       float fin[VEC];
-      __half2 fin2[VEC / 2];
+      __half2 rmax[VEC / 2];
 #pragma unroll
       for (int j = 0; j < VEC; ++j) fin[j] = 0.0f;
 #pragma unroll
-      for (int j = 0; j < VEC / 2; ++j) fin2[j] = __float2half2_rn(0.0f);
+      for (int j = 0; j < VEC / 2; ++j) rmax[j] = __float2half2_rn(0.0f);
       // The plane loads of a batch of harmonics are in flight together, kept raw in registers.  The loop over the
       // batches is not unrolled: the body for one batch (VEC pixels x LB harmonics) then stays in the instruction
       // cache, which the fully unrolled chain of all F harmonics overflowed.
@@ -399,32 +399,38 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
         for (int i = 0; i < 2 * LB; ++i) raw[i] = __ldg(reinterpret_cast<const uint4*>(ptr + (size_t)i * plane));
 #pragma unroll
         for (int ll = 0; ll < LB; ++ll) {
-          float s[VEC], c[VEC];
-          unpack_vec<T>(raw[2 * ll], s);
-          unpack_vec<T>(raw[2 * ll + 1], c);
           if constexpr (sizeof(T) == 2) {
+            // two pixels at a time, from the packed pairs as they were loaded (atan2_ht_pair_hw)
             const uint32_t ws[4] = {raw[2 * ll].x, raw[2 * ll].y, raw[2 * ll].z, raw[2 * ll].w};
             const uint32_t wc[4] = {raw[2 * ll + 1].x, raw[2 * ll + 1].y, raw[2 * ll + 1].z, raw[2 * ll + 1].w};
-            const __half2 zero2 = __float2half2_rn(0.0f);
 #pragma unroll
             for (int j = 0; j < VEC / 2; ++j) {
-              fin2[j] = __hfma2(*reinterpret_cast<const __half2*>(&ws[j]), zero2, fin2[j]);
-              fin2[j] = __hfma2(*reinterpret_cast<const __half2*>(&wc[j]), zero2, fin2[j]);
+              const __half2 ys = *reinterpret_cast<const __half2*>(&ws[j]), xs = *reinterpret_cast<const __half2*>(&wc[j]);
+              const __half2 ay = __habs2(ys), ax = __habs2(xs);
+              const __half2 mxn = __hmax2_nan(ax, ay);
+              rmax[j] = __hmax2_nan(rmax[j], mxn);
+              if (l0 + ll < Fu) {
+                const float2 u = atan2_ht_pair_hw(ys, xs, ay, ax, mxn);
+                const float2 v = refine_scaled_pair(make_float2(p[2 * j], p[2 * j + 1]), u);
+                p[2 * j] = v.x;
+                p[2 * j + 1] = v.y;
+              }
             }
           } else {
+            float s[VEC], c[VEC];
+            unpack_vec<T>(raw[2 * ll], s);
+            unpack_vec<T>(raw[2 * ll + 1], c);
 #pragma unroll
             for (int j = 0; j < VEC; ++j) fin[j] = fold_finite(fin[j], s[j], c[j]);
-          }
-          if (l0 + ll < Fu) {
-            // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
+            if (l0 + ll < Fu) {
+              // two pixels at a time: the polynomial and the coarse-to-fine step as packed instructions
 #pragma unroll
-            for (int j = 0; j < VEC; j += 2) {
-              // (binary16 input: the variant whose two divisions run as packed instructions, bit-identical for such operands)
-              const float2 u = sizeof(T) == 2 ? atan2_ht_pair_h(s[j], c[j], s[j + 1], c[j + 1])
-                                              : atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
-              const float2 v = refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
-              p[j] = v.x;
-              p[j + 1] = v.y;
+              for (int j = 0; j < VEC; j += 2) {
+                const float2 u = atan2_ht_pair(s[j], c[j], s[j + 1], c[j + 1]);
+                const float2 v = refine_scaled_pair(make_float2(p[j], p[j + 1]), u);
+                p[j] = v.x;
+                p[j + 1] = v.y;
+              }
             }
           }
         }
@@ -434,7 +440,8 @@ decode_vote_vec_kernel(const T* __restrict__ emb, const uint8_t* __restrict__ fg
       for (int j = 0; j < VEC; ++j) {
         p[j] = __fmul_rn(p[j], unscale);
         bool bad = fin[j] != fin[j];
-        if constexpr (sizeof(T) == 2) bad = (j & 1) ? __hisnan(__high2half(fin2[j / 2])) : __hisnan(__low2half(fin2[j / 2]));
+        if constexpr (sizeof(T) == 2)   // the running maximum is infinite or a NaN: exponent field all ones
+          bad = ((*reinterpret_cast<const uint32_t*>(&rmax[j / 2]) >> (16 * (j & 1))) & 0x7c00u) == 0x7c00u;
         if (bad) okbits &= ~(1u << j);
       }
     }
