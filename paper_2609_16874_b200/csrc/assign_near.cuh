@@ -775,7 +775,7 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
 // The pixels that the walk left over are scored against every peak: a whole CTA per pixel while there are fewer pixels
 // than CTAs, else eight lanes per pixel with the rows staged in shared memory.
 template <typename T, int FT>
-__global__ void __launch_bounds__(kNearThreads)
+__global__ void __launch_bounds__(kNearThreads, FT == 16 ? 1 : 4)   // (a CTA is a chain of latencies: many resident ones)
 assign_near_hard_kernel(const T* __restrict__ emb, int HW, int K_max, const float* __restrict__ cand2,
                         const int32_t* __restrict__ count_ptr, float tau, int32_t* __restrict__ labels,
                         uint32_t* __restrict__ near_state, const uint32_t* __restrict__ hard_q, int q_cap, int k_min) {
