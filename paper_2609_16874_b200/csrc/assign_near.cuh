@@ -19,8 +19,9 @@
 // the voting kernel does -- a thread takes (8-pixel group, axis), 128-bit plane loads, background never fetched --
 // and only certifies, from cheap upper bounds of t and of the distance to the first candidate of k0's list, that the
 // second list entry is already out of reach (nearly every pixel when the candidates sit on the voted centroids):
-// the label is then final.  The other pixels go to a queue in global memory, which assign_near_walk_kernel decides
-// exactly, one thread per pixel.  assign_near_kernel is that walk for every pixel: any alignment, and scores.
+// the label is then final.  The other pixels are decided exactly by a walk of the list, one thread per pixel: a warp's
+// first few by the warp itself once it has streamed its share, the rest through a queue in global memory by
+// assign_near_walk_kernel.  assign_near_kernel is that walk for every pixel: any alignment, and scores.
 #pragma once
 
 #include "assign.cuh"
@@ -30,6 +31,7 @@
 namespace cpe {
 
 constexpr int kNearThreads = 256;
+constexpr int kWarpQueue = 64;         // pixels that a warp of the streaming kernel keeps for its own walks
 constexpr float kNearSlack = 1.00002f;
 constexpr int kNearWalkMax = 12;     // list entries one thread walks before the pixel goes to the warp-wide scan
 
@@ -110,8 +112,11 @@ __device__ __forceinline__ void near_full_scan_warp(const T* __restrict__ p, siz
 // totals and decides whether the image is handed on.  Returns the stop flag.
 // (Hard pixels come in clusters -- an instance whose peak a stronger neighbour suppressed --, so the ratio is only
 // looked at once an eighth of the image has been visited.)
-__device__ __forceinline__ uint32_t near_account(uint32_t* state, uint32_t visited, uint32_t n_hard, uint32_t min_proc) {
-  const uint32_t proc = atomicAdd(&state[kNearProcessed], visited) + visited;
+// (proc_floor: the caller's own estimate of the pixels visited so far by everybody, for callers that report pixels
+// without hard ones only now and then -- the counter alone would then lag behind the hard pixels' count.)
+__device__ __forceinline__ uint32_t near_account(uint32_t* state, uint32_t visited, uint32_t n_hard, uint32_t min_proc,
+                                                 uint32_t proc_floor = 0u) {
+  const uint32_t proc = max(atomicAdd(&state[kNearProcessed], visited) + visited, proc_floor);
   if (!n_hard) return *reinterpret_cast<volatile uint32_t*>(&state[kNearGiveUp]);
   const uint32_t hd = atomicAdd(&state[kNearHard], n_hard) + n_hard;
   uint32_t stop = *reinterpret_cast<volatile uint32_t*>(&state[kNearGiveUp]);
@@ -297,9 +302,10 @@ constexpr float kHalfRel = 1.01f, kHalfAbs = 0.008f;
 // Upper bounds need no exact arithmetic: the sums of squares are accumulated in packed binary16 (two pixels per
 // instruction, no widening of the loaded values) and inflated by their worst-case error.  A certified pixel gets the
 // first candidate's label; every other pixel -- not certified, no peak for its bin, tau finite (the exact distance is
-// then needed) -- is appended to the image's queue in global memory (`slow_q`, capacity q_cap; its fill is
-// near_state[kNearQueue]) and decided exactly by assign_near_walk_kernel afterwards.  A queue that overflows hands the
-// image to the filtered kernel, like too many hard pixels do.
+// then needed) -- is decided exactly by a walk of its list: the first kWarpQueue of a warp by the warp itself when its
+// share of the image is done, the rest (and all of them when tau is finite) appended to the image's queue in global
+// memory (`slow_q`, capacity q_cap; its fill is near_state[kNearQueue]) for assign_near_walk_kernel.  A queue that
+// overflows hands the image to the filtered kernel, like too many hard pixels do.
 //
 // Dynamic shared memory (`smem_rows_bytes`): binary16 copies of the reference rows [K][D] and, unless SAME, of the
 // candidate rows; an image whose rows do not fit reads them from global memory (`ref_h` / `cand_h`, [K][D] binary16,
@@ -311,8 +317,13 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
                           const uint32_t* __restrict__ nbr, const int32_t* __restrict__ cell_peak,
                           const uint32_t* __restrict__ pix_cell, int cells, const int32_t* __restrict__ count_ptr, float tau,
                           int32_t* __restrict__ labels, uint32_t* __restrict__ near_state, uint32_t* __restrict__ slow_q,
-                          int q_cap, int k_min, int smem_rows_bytes) {
+                          int q_cap, int k_min, int smem_rows_bytes, const float* __restrict__ ref2,
+                          const float* __restrict__ cand2, uint32_t* __restrict__ hard_q) {
   extern __shared__ __align__(16) unsigned char near_smem[];
+  // A warp keeps the first kWarpQueue pixels that it cannot certify to itself and walks their lists when its share of
+  // the image is done (a lane per pixel, as assign_near_walk_kernel does for the rest): the walks are chains of
+  // dependent fetches, which hide behind the other warps' streaming instead of waiting for a kernel of their own.
+  __shared__ uint32_t s_wq[kStreamThreads / 32][kWarpQueue];
   grid_dependency_sync();
   constexpr int VEC = Elem<T>::kVec;           // pixels per 128-bit load
   constexpr int H2 = VEC / 2;
@@ -364,7 +375,9 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
   const bool certify = !(tau < __int_as_float(0x7f800000));   // with a finite tau every pixel needs its exact distance
   const uint32_t min_proc = max(8192u, (uint32_t)HW / 8u);
   uint32_t n_pairs = 0;
+  uint32_t wq_n = 0;                            // fill of this warp's own queue (uniform over the warp)
   uint32_t visited = 0, hard_acc = 0;          // lane 0: not yet added to the image's totals
+  uint32_t visited_all = 0;                     // pixels this warp has been through
   const int axis = lane & 1;                    // lanes 2j and 2j+1 share a group
   const long long n_groups = (long long)HW / VEC;
   const long long n_steps = (n_groups + 15) / 16;
@@ -665,7 +678,10 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
       my_label[jj] = label;
       // queue the pixel: one atomic per warp and round
       const uint32_t sm = __ballot_sync(0xffffffffu, slow);
-      if (sm) {
+      if (sm && certify && wq_n + (uint32_t)__popc(sm) <= (uint32_t)kWarpQueue) {
+        if (slow) s_wq[wid][wq_n + (uint32_t)__popc(sm & ((1u << lane) - 1u))] = (uint32_t)(pix0 + j);
+        wq_n += (uint32_t)__popc(sm);
+      } else if (sm) {
         uint32_t base = 0;
         if (lane == 0) base = atomicAdd(&state[kNearQueue], (uint32_t)__popc(sm));
         base = __shfl_sync(0xffffffffu, base, 0);
@@ -686,16 +702,66 @@ assign_near_stream_kernel(const T* __restrict__ emb, const uint8_t* __restrict__
     // ---- hand the image on if too many pixels cannot be closed by the bounds (before the walks are paid for)
     const uint32_t nh = __reduce_add_sync(0xffffffffu, n_likely_hard);
     visited += 16u * VEC;
+    visited_all += 16u * VEC;
     hard_acc += nh;
     uint32_t stop = 0;
     if (lane == 0 && (hard_acc || visited >= 4096u)) {
-      stop = near_account(state, visited, hard_acc, min_proc);
+      // hard pixels are reported at once, the others now and then: the share is taken of what all warps have visited
+      // by now, estimated from this warp's own progress (the warps walk the image in step)
+      const uint32_t everybody = (uint32_t)min((unsigned long long)visited_all * (unsigned long long)n_warps, (unsigned long long)HW);
+      stop = near_account(state, visited, hard_acc, min_proc, everybody);
       visited = hard_acc = 0;
     }
     if (__shfl_sync(0xffffffffu, stop, 0)) return;     // the filtered kernel redoes the whole image
   }
   if (lane == 0 && visited) near_account(state, visited, hard_acc, min_proc);
-  near_flush_counters(state, 0u, n_pairs, 0u, 0u);
+
+  // ---- this warp's own queue: exact walks, a lane per pixel
+  uint32_t n_multi = 0;
+  __syncwarp();
+  if (wq_n) {
+    const float* ref_img = ref2 + (size_t)b * K_max * D;
+    const float* cand_img = cand2 + (size_t)b * K_max * D;
+    for (uint32_t i0 = 0; i0 < wq_n; i0 += 32u) {
+      const bool have = i0 + lane < wq_n;
+      const size_t n = have ? s_wq[wid][i0 + lane] : 0;
+      float d1 = __int_as_float(0x7f800000), d2 = d1;
+      int k1 = -1;
+      bool hard = false;
+      uint32_t scored = 0;
+      if (have) {
+        const uint32_t cell = __ldg(pc_img + n);
+        int k0 = (cell != 0xffffffffu && (int)cell < cells) ? __ldg(cp_img + cell) : -1;
+        if (k0 >= K) k0 = -1;
+        hard = k0 < 0;
+        if (!hard) {
+          const T* p = e_img + n;
+          float2 e2[D / 2];
+#pragma unroll
+          for (int c = 0; c < D / 2; ++c) {
+            e2[c].x = Elem<T>::load1(p + (size_t)c * plane);
+            e2[c].y = Elem<T>::load1(p + (size_t)(D / 2 + c) * plane);
+          }
+          near_walk<D, false>(e2, k0, K, SAME, ref_img, cand_img, nbr_img, d1, d2, k1, hard, scored);
+        }
+      }
+      const uint32_t hm = __ballot_sync(0xffffffffu, hard);
+      if (hm) {
+        uint32_t hbase = 0;
+        if (lane == 0) hbase = atomicAdd(&state[kNearHardQueue], (uint32_t)__popc(hm));
+        hbase = __shfl_sync(0xffffffffu, hbase, 0);
+        const uint32_t at = hbase + (uint32_t)__popc(hm & ((1u << lane) - 1u));
+        if (hard && at < (uint32_t)q_cap) hard_q[(size_t)b * q_cap + at] = (uint32_t)n;
+        if (lane == 0 && hbase + (uint32_t)__popc(hm) > (uint32_t)q_cap) atomicExch(&state[kNearGiveUp], 1u);
+      }
+      if (have && !hard) {
+        if (scored > 1) ++n_multi;
+        n_pairs += scored;
+        lab_img[n] = k1 >= 0 ? k1 + 1 : 0;        // (tau is infinite here: nothing is rejected)
+      }
+    }
+  }
+  near_flush_counters(state, 0u, n_pairs, n_multi, 0u);
 }
 
 // The walk of the pixels that the streaming kernel queued, one thread per pixel.
@@ -756,7 +822,10 @@ assign_near_walk_kernel(const T* __restrict__ emb, int HW, int K_max, const floa
       uint32_t hbase = 0;
       if (lane == 0) hbase = atomicAdd(&state[kNearHardQueue], (uint32_t)__popc(hm));
       hbase = __shfl_sync(0xffffffffu, hbase, 0);
-      if (hard) hard_q[(size_t)b * q_cap + hbase + (uint32_t)__popc(hm & ((1u << lane) - 1u))] = (uint32_t)n;
+      // (the streaming kernel's warps append here too: the bound is checked, and an overflow hands the image on)
+      const uint32_t at = hbase + (uint32_t)__popc(hm & ((1u << lane) - 1u));
+      if (hard && at < (uint32_t)q_cap) hard_q[(size_t)b * q_cap + at] = (uint32_t)n;
+      if (lane == 0 && hbase + (uint32_t)__popc(hm) > (uint32_t)q_cap) atomicExch(&state[kNearGiveUp], 1u);
     }
     if (have && !hard) {
       if (scored > 1) ++n_multi;

@@ -90,7 +90,7 @@ int launch_stream_t(cudaStream_t st, const NearArgs& a) {
                             static_cast<const T*>(a.emb), a.fg, a.HW, a.p->max_instances,
                             static_cast<const __half*>(a.ref_h), static_cast<const __half*>(a.cand_h), a.nbr, a.cell_peak,
                             a.pix_cell, a.cells, a.count, a.p->tau, a.labels, a.near_state, a.slow_q, a.q_cap, a.k_min,
-                            smem));
+                            smem, a.ref2, a.cand2, a.hard_q));
   CPE_CUDA(cudaGetLastError());
   // the pixels it queued
   const long long walk_ctas = std::max(1, ((FT == 16 ? 2 : 3) * sm_count() + a.B - 1) / a.B);
